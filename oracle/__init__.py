@@ -1,0 +1,206 @@
+"""ctypes front end of the CPU oracle (``qarl_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: importable from ``tests/``, the smoke check and the benchmark's
+CPU-baseline leg.  The product path (the CUDA library and its Python binding) never imports
+this package, and this package never imports the product path.
+
+bf16 tensors travel as numpy ``uint16`` arrays of bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from .build import build as _build
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build())
+        L = _lib
+        i64, p = C.c_int64, C.c_void_p
+        L.oracle_bf16_rne.restype = C.c_uint16
+        L.oracle_bf16_rne.argtypes = [C.c_float]
+        L.oracle_e4m3_decode.restype = C.c_double
+        L.oracle_e4m3_decode.argtypes = [C.c_uint8]
+        L.oracle_e4m3_encode.restype = C.c_uint8
+        L.oracle_e4m3_encode.argtypes = [C.c_float]
+        L.oracle_e4m3_encode_array.restype = None
+        L.oracle_e4m3_encode_array.argtypes = [p, i64, p]
+        L.oracle_bf16_rne_array.restype = None
+        L.oracle_bf16_rne_array.argtypes = [p, i64, p]
+        L.oracle_quantize_weight.restype = C.c_int
+        L.oracle_quantize_weight.argtypes = [p, i64, i64, i64, p, p]
+        L.oracle_quantize_act.restype = C.c_int
+        L.oracle_quantize_act.argtypes = [p, i64, i64, i64, p, p]
+        L.oracle_linear_q.restype = C.c_int
+        L.oracle_linear_q.argtypes = [p, p, i64, i64, p, p, i64, p, p]
+        L.oracle_linear.restype = C.c_int
+        L.oracle_linear.argtypes = [p, i64, i64, p, p, i64, p, p]
+        L.oracle_permute.restype = C.c_int
+        L.oracle_permute.argtypes = [p, i64, i64, i64, p, p, p]
+        L.oracle_swiglu.restype = None
+        L.oracle_swiglu.argtypes = [p, i64, i64, p]
+        L.oracle_combine.restype = None
+        L.oracle_combine.argtypes = [p, p, p, i64, i64, i64, p]
+        L.oracle_moe.restype = C.c_int
+        L.oracle_moe.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p]
+        L.oracle_num_threads.restype = C.c_int
+        L.oracle_num_threads.argtypes = []
+    return _lib
+
+
+def _ptr(a: np.ndarray | None):
+    if a is None:
+        return None
+    assert a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle returned status {code}")
+        self.code = code
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def e4m3_decode_table() -> np.ndarray:
+    """All 256 code values as float64 (NaN at 0x7F / 0xFF)."""
+    return np.array([lib().oracle_e4m3_decode(c) for c in range(256)], dtype=np.float64)
+
+
+def e4m3_encode(v) -> np.ndarray:
+    v = _c(v, np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    lib().oracle_e4m3_encode_array(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def bf16_rne(v) -> np.ndarray:
+    v = _c(v, np.float32)
+    out = np.empty(v.shape, dtype=np.uint16)
+    lib().oracle_bf16_rne_array(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def quantize_weight(w_bits: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
+    """w bf16 bits [E, N, K] or [N, K] -> (codes u8 same shape, scales f32 [.., N/128, K/128])."""
+    w = _c(w_bits, np.uint16)
+    squeeze = w.ndim == 2
+    if squeeze:
+        w = w[None]
+    E, N, K = w.shape
+    codes = np.empty((E, N, K), dtype=np.uint8)
+    scales = np.empty((E, N // 128, K // 128), dtype=np.float32)
+    rc = lib().oracle_quantize_weight(_ptr(w), E, N, K, _ptr(codes), _ptr(scales))
+    if rc:
+        raise OracleError(rc)
+    return (codes[0], scales[0]) if squeeze else (codes, scales)
+
+
+def quantize_act(x_bits: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
+    """x bf16 bits [M, K] -> (codes u8 [M, K], scales f32 [M, K/128])."""
+    x = _c(x_bits, np.uint16)
+    M, K = x.shape
+    codes = np.empty((M, K), dtype=np.uint8)
+    scales = np.empty((M, K // 128), dtype=np.float32)
+    rc = lib().oracle_quantize_act(_ptr(x), M, K, K, _ptr(codes), _ptr(scales))
+    if rc:
+        raise OracleError(rc)
+    return codes, scales
+
+
+def linear_q(xc, xs, wc, ws) -> tuple[np.ndarray, np.ndarray]:
+    """Block-scaled linear from codes and scales -> (y fp32 [M, N], y bf16 bits [M, N])."""
+    xc, xs, wc, ws = _c(xc, np.uint8), _c(xs, np.float32), _c(wc, np.uint8), _c(ws, np.float32)
+    M, K = xc.shape
+    N = wc.shape[0]
+    assert wc.shape[1] == K
+    y32 = np.empty((M, N), dtype=np.float32)
+    y16 = np.empty((M, N), dtype=np.uint16)
+    rc = lib().oracle_linear_q(_ptr(xc), _ptr(xs), M, K, _ptr(wc), _ptr(ws), N, _ptr(y32), _ptr(y16))
+    if rc:
+        raise OracleError(rc)
+    return y32, y16
+
+
+def linear(x_bits, wc, ws) -> tuple[np.ndarray, np.ndarray]:
+    """y = blockscaled(quantize_act(x), W) -> (y fp32, y bf16 bits)."""
+    x, wc, ws = _c(x_bits, np.uint16), _c(wc, np.uint8), _c(ws, np.float32)
+    M, K = x.shape
+    N = wc.shape[0]
+    y32 = np.empty((M, N), dtype=np.float32)
+    y16 = np.empty((M, N), dtype=np.uint16)
+    rc = lib().oracle_linear(_ptr(x), M, K, _ptr(wc), _ptr(ws), N, _ptr(y32), _ptr(y16))
+    if rc:
+        raise OracleError(rc)
+    return y32, y16
+
+
+def permute(ids, E: int) -> tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """ids int32 [M, k] -> (offsets [E+1], sorted_pair [M*k], pos_of_pair [M*k])."""
+    ids = _c(ids, np.int32)
+    M, k = ids.shape
+    offsets = np.empty(E + 1, dtype=np.int32)
+    sorted_pair = np.empty(M * k, dtype=np.int32)
+    pos = np.empty(M * k, dtype=np.int32)
+    rc = lib().oracle_permute(_ptr(ids), M, k, E, _ptr(offsets), _ptr(sorted_pair), _ptr(pos))
+    if rc:
+        raise OracleError(rc)
+    return offsets, sorted_pair, pos
+
+
+def swiglu(gate_up_bits) -> np.ndarray:
+    """gate_up bf16 bits [P, 2I] -> h bf16 bits [P, I]."""
+    gu = _c(gate_up_bits, np.uint16)
+    P, I2 = gu.shape
+    h = np.empty((P, I2 // 2), dtype=np.uint16)
+    lib().oracle_swiglu(_ptr(gu), P, I2 // 2, _ptr(h))
+    return h
+
+
+def combine(y32, ids, wts) -> np.ndarray:
+    """y32 fp32 [M*k, H] by flat pair id, ids/wts [M, k] -> out bf16 bits [M, H]."""
+    y32, ids, wts = _c(y32, np.float32), _c(ids, np.int32), _c(wts, np.float32)
+    M, k = ids.shape
+    H = y32.shape[1]
+    out = np.empty((M, H), dtype=np.uint16)
+    lib().oracle_combine(_ptr(y32), _ptr(ids), _ptr(wts), M, k, H, _ptr(out))
+    return out
+
+
+def moe(x_bits, ids, wts, w13c, w13s, w2c, w2s, dumps: bool = False):
+    """One routed MoE FFN layer.  Returns out bf16 bits [M, H], or (out, dict of dumps)
+    with gate_up [P,2I], h [P,I], h_codes [P,I], h_scales [P,I/128], y32 [P,H] by pair id."""
+    x, ids, wts = _c(x_bits, np.uint16), _c(ids, np.int32), _c(wts, np.float32)
+    w13c, w13s = _c(w13c, np.uint8), _c(w13s, np.float32)
+    w2c, w2s = _c(w2c, np.uint8), _c(w2s, np.float32)
+    M, H = x.shape
+    k = ids.shape[1]
+    E, I2, _ = w13c.shape
+    I = I2 // 2
+    P = M * k
+    out = np.empty((M, H), dtype=np.uint16)
+    d = {}
+    if dumps:
+        d = dict(gate_up=np.empty((P, 2 * I), np.uint16), h=np.empty((P, I), np.uint16),
+                 h_codes=np.empty((P, I), np.uint8), h_scales=np.empty((P, I // 128), np.float32),
+                 y32=np.empty((P, H), np.float32))
+    rc = lib().oracle_moe(_ptr(x), _ptr(ids), _ptr(wts), M, H, I, E, k,
+                          _ptr(w13c), _ptr(w13s), _ptr(w2c), _ptr(w2s), _ptr(out),
+                          _ptr(d.get("gate_up")), _ptr(d.get("h")), _ptr(d.get("h_codes")),
+                          _ptr(d.get("h_scales")), _ptr(d.get("y32")))
+    if rc:
+        raise OracleError(rc)
+    return (out, d) if dumps else out

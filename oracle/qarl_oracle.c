@@ -1,0 +1,415 @@
+/*
+ * CPU oracle for the block-scaled FP8 quantized forward (QaRL, Sec. 2.2 and Sec. 3.1).
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It is a plain, slow, obviously-correct restatement of what
+ * the quantized forward computes, written from the paper's formulas and the e4m3 format
+ * definition.  It shares no code with the CUDA path and must never be called from it; only
+ * the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Parity status: every function below is pinned by tests that do not call this file's own
+ * formulas (library casts, closed forms, brute force, exact-arithmetic special cases) except
+ * one: the ORDER in which block partial sums are promoted and in which the top-k
+ * contributions are added (oracle_linear_q's kb-ascending chain, oracle_combine's
+ * ascending-expert chain) is "parity unpinned" by the paper -- App. C only requires that
+ * some fixed order be used.  The order chosen here is stated beside each function.
+ *
+ * Build: gcc -O2 -fopenmp -ffp-contract=off -fno-fast-math -shared -fPIC (see oracle/build.py).
+ * OpenMP is used over independent rows / experts only, never inside a reduction whose
+ * order is specified.
+ *
+ * Notation follows the paper: s = max|W| / alpha, W_q = [W / s]_FP8, W^ = s * W_q,
+ * Y ~= (s_x s_w) (X_q W_q), alpha = 448 for e4m3 (Sec. 2.2, "Floating-point quantization").
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define QBLOCK 128            /* block edge: 128x128 weight blocks, 1x128 activation groups */
+#define E4M3_ALPHA 448.0f     /* Sec. 2.2: alpha = 448 for e4m3 => the no-infinity variant  */
+#define AMAX_FLOOR 0x1p-40f   /* reading for an all-zero block (paper is silent)            */
+
+/* ---------------------------------------------------------------------------------------
+ * bf16 helpers.  bf16 is the upper half of an IEEE fp32.
+ * ------------------------------------------------------------------------------------- */
+static inline float bf16_to_f32(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* fp32 -> bf16, round to nearest, ties to even. */
+uint16_t oracle_bf16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u); /* NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+float oracle_bf16_to_f32(uint16_t b) { return bf16_to_f32(b); }
+
+/* ---------------------------------------------------------------------------------------
+ * e4m3 ("fn": no infinities, max finite 448 -- fixed by alpha = 448 in Sec. 2.2).
+ * code = s eeee mmm.  e = 0: (-1)^s * m * 2^-9.  1 <= e <= 15: (-1)^s * (1 + m/8) * 2^(e-7).
+ * 0x7F and 0xFF are NaN.
+ * ------------------------------------------------------------------------------------- */
+double oracle_e4m3_decode(uint8_t c) {
+    int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    if (e == 15 && m == 7) return NAN;
+    double v = (e == 0) ? ldexp((double)m, -9) : ldexp(1.0 + m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* The code's value as an integer count of 2^-9 (exact; |.| <= 448 * 512 = 229376). */
+static inline int32_t e4m3_units(uint8_t c) {
+    int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    int32_t v = (e == 0) ? m : ((8 + m) << (e - 1));
+    return s ? -v : v;
+}
+
+/* fp32 -> e4m3: round to nearest on the e4m3 grid, ties to the even mantissa code,
+ * magnitudes above 448 saturate to +-448, the sign is kept (also for zero / underflow).
+ * The paper only writes [.]_FPk ("casting"); rounding and overflow mode are this reading. */
+uint8_t oracle_e4m3_encode(float f) {
+    if (isnan(f)) return 0x7f;
+    uint8_t sign = signbit(f) ? 0x80 : 0x00;
+    double a = fabs((double)f);
+    if (a > 448.0) return sign | 0x7e;
+    if (a < 0x1p-6) {
+        /* subnormal grid, spacing 2^-9; q = 8 lands on the smallest normal (code 0x08) */
+        int q = (int)nearbyint(ldexp(a, 9));
+        return sign | (uint8_t)q;
+    }
+    int ex;
+    (void)frexp(a, &ex);          /* a = f * 2^ex, f in [0.5, 1) => floor(log2 a) = ex - 1 */
+    int e_unb = ex - 1;
+    int q = (int)nearbyint(ldexp(a, 3 - e_unb));   /* in [8, 16] */
+    if (q == 16) { q = 8; e_unb += 1; }
+    return sign | (uint8_t)(((e_unb + 7) << 3) | (q - 8));
+}
+
+/* Array forms of the two casts (for exhaustive tests). */
+void oracle_e4m3_encode_array(const float *v, int64_t n, uint8_t *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_e4m3_encode(v[i]);
+}
+
+void oracle_bf16_rne_array(const float *v, int64_t n, uint16_t *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_bf16_rne(v[i]);
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Scale and code of one block (Sec. 2.2): s = max|W| / 448, W_q = [W / s]_FP8.
+ * Readings where the paper is silent or ambiguous:
+ *   - an all-zero block uses amax_c = max(amax, 2^-40);
+ *   - W / s is evaluated as W * inv with inv = fl(448 / amax_c), one fp32 multiply per
+ *     element; the stored scale is still s = fl(amax_c / 448).
+ * ------------------------------------------------------------------------------------- */
+static inline float block_scale(float amax, float *inv) {
+    float amax_c = amax > AMAX_FLOOR ? amax : AMAX_FLOOR;
+    *inv = E4M3_ALPHA / amax_c;
+    return amax_c / E4M3_ALPHA;
+}
+
+/* W bf16 [E, N, K] -> codes u8 [E, N, K], scales f32 [E, N/128, K/128]; 128x128 blocks. */
+int oracle_quantize_weight(const uint16_t *w, int64_t E, int64_t N, int64_t K,
+                           uint8_t *codes, float *scales) {
+    if (N % QBLOCK || K % QBLOCK) return -2;
+    int64_t nb = N / QBLOCK, kb = K / QBLOCK;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t e = 0; e < E; ++e)
+        for (int64_t bn = 0; bn < nb; ++bn)
+            for (int64_t bk = 0; bk < kb; ++bk) {
+                const uint16_t *base = w + (e * N + bn * QBLOCK) * K + bk * QBLOCK;
+                float amax = 0.0f;
+                for (int r = 0; r < QBLOCK; ++r)
+                    for (int c = 0; c < QBLOCK; ++c) {
+                        float a = fabsf(bf16_to_f32(base[(int64_t)r * K + c]));
+                        if (a > amax) amax = a;
+                    }
+                float inv;
+                float s = block_scale(amax, &inv);
+                scales[(e * nb + bn) * kb + bk] = s;
+                uint8_t *cb = codes + (e * N + bn * QBLOCK) * K + bk * QBLOCK;
+                for (int r = 0; r < QBLOCK; ++r)
+                    for (int c = 0; c < QBLOCK; ++c) {
+                        float v = bf16_to_f32(base[(int64_t)r * K + c]) * inv;
+                        cb[(int64_t)r * K + c] = oracle_e4m3_encode(v);
+                    }
+            }
+    return 0;
+}
+
+/* X bf16 [M, K] (row stride ldx elements) -> codes u8 [M, K], scales f32 [M, K/128];
+ * 1x128 groups along K. */
+int oracle_quantize_act(const uint16_t *x, int64_t M, int64_t K, int64_t ldx,
+                        uint8_t *codes, float *scales) {
+    if (K % QBLOCK) return -2;
+    int64_t kb = K / QBLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t g = 0; g < kb; ++g) {
+            const uint16_t *base = x + m * ldx + g * QBLOCK;
+            float amax = 0.0f;
+            for (int c = 0; c < QBLOCK; ++c) {
+                float a = fabsf(bf16_to_f32(base[c]));
+                if (a > amax) amax = a;
+            }
+            float inv;
+            float s = block_scale(amax, &inv);
+            scales[m * kb + g] = s;
+            for (int c = 0; c < QBLOCK; ++c)
+                codes[m * K + g * QBLOCK + c] = oracle_e4m3_encode(bf16_to_f32(base[c]) * inv);
+        }
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Block-scaled linear (Eq. "Y ~= (s_x s_w)(X_q W_q)" of Sec. 2.2, applied per 128-wide
+ * K-block, accumulating in higher precision = fp32):
+ *   y[m,n] = sum_kb  fl(s_x[m,kb] * s_w[n/128,kb]) * p[m,n,kb],
+ *   p = the EXACT dot product of the 128 code values of the block, rounded once to fp32.
+ * Order (parity unpinned by the paper, App. C only asks for a fixed one): acc starts at
+ * 0.0f and takes acc = fmaf(sc, p, acc) for kb = 0, 1, 2, ... ascending.
+ * The block sum is exact: each code is an integer multiple of 2^-9, so products are
+ * integers in units of 2^-18 and 128 of them stay below 2^43.
+ *
+ * w_row_block_of(n): scale row for weight row n is n / 128.
+ * Outputs: y32 (fp32, may be NULL) and y16 (bf16 bits, may be NULL), both [M, N].
+ * ------------------------------------------------------------------------------------- */
+static void linear_rows(const uint8_t *xc, const float *xs, int64_t M, int64_t K,
+                        const uint8_t *wc, const float *ws, int64_t N,
+                        float *y32, uint16_t *y16, int64_t ldy) {
+    int64_t kb = K / QBLOCK;
+    /* decode the weight codes once: int32 units of 2^-9 */
+    int32_t *wi = (int32_t *)malloc((size_t)N * K * sizeof(int32_t));
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N * K; ++i) wi[i] = e4m3_units(wc[i]);
+    int32_t *xi = (int32_t *)malloc((size_t)(M > 0 ? M : 1) * K * sizeof(int32_t));
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M * K; ++i) xi[i] = e4m3_units(xc[i]);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            float acc = 0.0f;
+            const int32_t *xr = xi + m * K;
+            const int32_t *wr = wi + n * K;
+            for (int64_t b = 0; b < kb; ++b) {
+                int64_t isum = 0;
+                for (int c = 0; c < QBLOCK; ++c)
+                    isum += (int64_t)xr[b * QBLOCK + c] * (int64_t)wr[b * QBLOCK + c];
+                float p = (float)ldexp((double)isum, -18);   /* exact, then one rounding */
+                float sc = xs[m * kb + b] * ws[(n / QBLOCK) * kb + b];
+                acc = fmaf(sc, p, acc);
+            }
+            if (y32) y32[m * ldy + n] = acc;
+            if (y16) y16[m * ldy + n] = oracle_bf16_rne(acc);
+        }
+    free(xi);
+    free(wi);
+}
+
+int oracle_linear_q(const uint8_t *xc, const float *xs, int64_t M, int64_t K,
+                    const uint8_t *wc, const float *ws, int64_t N,
+                    float *y32, uint16_t *y16) {
+    if (N % QBLOCK || K % QBLOCK) return -2;
+    linear_rows(xc, xs, M, K, wc, ws, N, y32, y16, N);
+    return 0;
+}
+
+/* y = blockscaled(quantize_act(x), W): the dense projection as one call. */
+int oracle_linear(const uint16_t *x, int64_t M, int64_t K,
+                  const uint8_t *wc, const float *ws, int64_t N,
+                  float *y32, uint16_t *y16) {
+    if (N % QBLOCK || K % QBLOCK) return -2;
+    uint8_t *xc = (uint8_t *)malloc((size_t)(M > 0 ? M : 1) * K);
+    float *xs = (float *)malloc((size_t)(M > 0 ? M : 1) * (K / QBLOCK) * sizeof(float));
+    oracle_quantize_act(x, M, K, K, xc, xs);
+    linear_rows(xc, xs, M, K, wc, ws, N, y32, y16, N);
+    free(xc);
+    free(xs);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Expert permutation (the grouping step of the routed MoE; not in the paper's text, fixed
+ * by the problem statement): flat pair id p = t*k + j; pairs stably sorted by expert id
+ * (ties by ascending p).  offsets[e] = first sorted position of expert e, offsets[E] = P.
+ * Returns -8 for an id outside [0, E) or the same expert twice in one token.
+ * ------------------------------------------------------------------------------------- */
+int oracle_permute(const int32_t *ids, int64_t M, int64_t k, int64_t E,
+                   int32_t *offsets, int32_t *sorted_pair, int32_t *pos_of_pair) {
+    int64_t P = M * k;
+    for (int64_t t = 0; t < M; ++t)
+        for (int64_t j = 0; j < k; ++j) {
+            int32_t e = ids[t * k + j];
+            if (e < 0 || e >= E) return -8;
+            for (int64_t j2 = 0; j2 < j; ++j2)
+                if (ids[t * k + j2] == e) return -8;
+        }
+    int64_t *count = (int64_t *)calloc((size_t)E + 1, sizeof(int64_t));
+    for (int64_t p = 0; p < P; ++p) count[ids[p]]++;
+    int64_t run = 0;
+    for (int64_t e = 0; e < E; ++e) {
+        offsets[e] = (int32_t)run;
+        run += count[e];
+    }
+    offsets[E] = (int32_t)run;
+    int64_t *cursor = (int64_t *)malloc((size_t)E * sizeof(int64_t));
+    for (int64_t e = 0; e < E; ++e) cursor[e] = offsets[e];
+    for (int64_t p = 0; p < P; ++p) {     /* ascending p => stable */
+        int64_t pos = cursor[ids[p]]++;
+        if (sorted_pair) sorted_pair[pos] = (int32_t)p;
+        if (pos_of_pair) pos_of_pair[p] = (int32_t)pos;
+    }
+    free(count);
+    free(cursor);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * SwiGLU on bf16 operands: h = bf16( silu(g) * u ), silu(g) = g / (1 + exp(-g)), evaluated
+ * in double and rounded once to fp32, then to bf16.  g and u are the bf16-rounded gate / up
+ * projections (every tensor crossing an op boundary is bf16 -- a reading; the paper does
+ * not discuss the activation).  gate_up is [P, 2I] with gate in columns 0..I-1.
+ * ------------------------------------------------------------------------------------- */
+void oracle_swiglu(const uint16_t *gate_up, int64_t P, int64_t I, uint16_t *h) {
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < P; ++p)
+        for (int64_t i = 0; i < I; ++i) {
+            double g = (double)bf16_to_f32(gate_up[p * 2 * I + i]);
+            double u = (double)bf16_to_f32(gate_up[p * 2 * I + I + i]);
+            double v = g / (1.0 + exp(-g)) * u;
+            h[p * I + i] = oracle_bf16_rne((float)v);
+        }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Top-k weighted combine.  For token t the k contributions are visited in ASCENDING EXPERT
+ * ID (a canonical order that does not depend on the caller's slot order; parity unpinned
+ * by the paper):  c_j = bf16( fl(w[t,j] * y32_j) );  sum = 0.0f; sum += float(c_j);
+ * out = bf16(sum).   y32 is [P, H] indexed by flat pair id p = t*k + j.
+ * ------------------------------------------------------------------------------------- */
+void oracle_combine(const float *y32, const int32_t *ids, const float *wts,
+                    int64_t M, int64_t k, int64_t H, uint16_t *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t) {
+        int64_t order[64];
+        for (int64_t j = 0; j < k; ++j) order[j] = j;
+        for (int64_t a = 1; a < k; ++a) {            /* insertion sort by expert id */
+            int64_t v = order[a], b = a;
+            while (b > 0 && ids[t * k + order[b - 1]] > ids[t * k + v]) {
+                order[b] = order[b - 1];
+                --b;
+            }
+            order[b] = v;
+        }
+        for (int64_t c = 0; c < H; ++c) {
+            float sum = 0.0f;
+            for (int64_t a = 0; a < k; ++a) {
+                int64_t j = order[a];
+                float cj = bf16_to_f32(oracle_bf16_rne(wts[t * k + j] * y32[(t * k + j) * H + c]));
+                sum = sum + cj;
+            }
+            out[t * H + c] = oracle_bf16_rne(sum);
+        }
+    }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * One routed MoE FFN layer on quantized weights, per pair p = (t, j) with expert e:
+ *   x_q          = quantize_act(x[t])                         (1x128 groups along H)
+ *   gate_up[p]   = bf16( blockscaled(x_q, W13_e) )            [2I]
+ *   h[p]         = swiglu(gate_up[p])                         [I], bf16
+ *   h_q          = quantize_act(h[p])                         (1x128 groups along I)
+ *   y32[p]       = blockscaled(h_q, W2_e)                     [H], fp32
+ *   out[t]       = combine over the token's k pairs
+ * w13 codes [E, 2I, H] (rows 0..I-1 gate, I..2I-1 up; scale blocks over the concatenated
+ * [2I, H] matrix), w2 codes [E, H, I].
+ * Optional dumps (NULL to skip), all indexed by flat pair id p = t*k + j:
+ *   d_gate_up bf16 [P, 2I], d_h bf16 [P, I], d_hc u8 [P, I], d_hs f32 [P, I/128],
+ *   d_y32 f32 [P, H].
+ * ------------------------------------------------------------------------------------- */
+int oracle_moe(const uint16_t *x, const int32_t *ids, const float *wts,
+               int64_t M, int64_t H, int64_t I, int64_t E, int64_t k,
+               const uint8_t *w13c, const float *w13s, const uint8_t *w2c, const float *w2s,
+               uint16_t *out, uint16_t *d_gate_up, uint16_t *d_h, uint8_t *d_hc, float *d_hs,
+               float *d_y32) {
+    if (H % QBLOCK || I % QBLOCK || k > 64) return -2;
+    int64_t P = M * k;
+    int32_t *offsets = (int32_t *)malloc(((size_t)E + 1) * sizeof(int32_t));
+    int32_t *sorted = (int32_t *)malloc((size_t)(P > 0 ? P : 1) * sizeof(int32_t));
+    int rc = oracle_permute(ids, M, k, E, offsets, sorted, NULL);
+    if (rc) { free(offsets); free(sorted); return rc; }
+
+    int64_t hb = H / QBLOCK, ib = I / QBLOCK;
+    size_t Pn = (size_t)(P > 0 ? P : 1), Mn = (size_t)(M > 0 ? M : 1);
+    uint8_t *xc = (uint8_t *)malloc(Mn * H);
+    float *xs = (float *)malloc(Mn * hb * sizeof(float));
+    oracle_quantize_act(x, M, H, H, xc, xs);
+
+    uint16_t *gate_up = d_gate_up ? d_gate_up : (uint16_t *)malloc(Pn * 2 * I * sizeof(uint16_t));
+    uint16_t *h = d_h ? d_h : (uint16_t *)malloc(Pn * I * sizeof(uint16_t));
+    uint8_t *hc = d_hc ? d_hc : (uint8_t *)malloc(Pn * I);
+    float *hs = d_hs ? d_hs : (float *)malloc(Pn * ib * sizeof(float));
+    float *y32 = d_y32 ? d_y32 : (float *)malloc(Pn * H * sizeof(float));
+
+    /* gate_up, one expert group at a time (rows gathered into a contiguous scratch) */
+    for (int64_t e = 0; e < E; ++e) {
+        int64_t g0 = offsets[e], g1 = offsets[e + 1], G = g1 - g0;
+        if (G == 0) continue;
+        uint8_t *gc = (uint8_t *)malloc((size_t)G * H);
+        float *gs = (float *)malloc((size_t)G * hb * sizeof(float));
+        uint16_t *gy = (uint16_t *)malloc((size_t)G * 2 * I * sizeof(uint16_t));
+        for (int64_t r = 0; r < G; ++r) {
+            int64_t t = sorted[g0 + r] / k;
+            memcpy(gc + r * H, xc + t * H, (size_t)H);
+            memcpy(gs + r * hb, xs + t * hb, (size_t)hb * sizeof(float));
+        }
+        linear_rows(gc, gs, G, H, w13c + e * 2 * I * H, w13s + e * (2 * I / QBLOCK) * hb,
+                    2 * I, NULL, gy, 2 * I);
+        for (int64_t r = 0; r < G; ++r)
+            memcpy(gate_up + (int64_t)sorted[g0 + r] * 2 * I, gy + r * 2 * I,
+                   (size_t)2 * I * sizeof(uint16_t));
+        free(gc); free(gs); free(gy);
+    }
+    oracle_swiglu(gate_up, P, I, h);
+    oracle_quantize_act(h, P, I, I, hc, hs);
+    for (int64_t e = 0; e < E; ++e) {
+        int64_t g0 = offsets[e], g1 = offsets[e + 1], G = g1 - g0;
+        if (G == 0) continue;
+        uint8_t *gc = (uint8_t *)malloc((size_t)G * I);
+        float *gs = (float *)malloc((size_t)G * ib * sizeof(float));
+        float *gy = (float *)malloc((size_t)G * H * sizeof(float));
+        for (int64_t r = 0; r < G; ++r) {
+            int64_t p = sorted[g0 + r];
+            memcpy(gc + r * I, hc + p * I, (size_t)I);
+            memcpy(gs + r * ib, hs + p * ib, (size_t)ib * sizeof(float));
+        }
+        linear_rows(gc, gs, G, I, w2c + e * H * I, w2s + e * hb * ib, H, gy, NULL, H);
+        for (int64_t r = 0; r < G; ++r)
+            memcpy(y32 + (int64_t)sorted[g0 + r] * H, gy + r * H, (size_t)H * sizeof(float));
+        free(gc); free(gs); free(gy);
+    }
+    oracle_combine(y32, ids, wts, M, k, H, out);
+
+    if (!d_gate_up) free(gate_up);
+    if (!d_h) free(h);
+    if (!d_hc) free(hc);
+    if (!d_hs) free(hs);
+    if (!d_y32) free(y32);
+    free(xc); free(xs); free(offsets); free(sorted);
+    return 0;
+}
+
+/* Number of OpenMP threads the oracle will use (reported beside its timing). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_num_threads(void) { return 1; }
+#endif
