@@ -1,0 +1,139 @@
+/*
+ * qarl.h -- C ABI of the B200-native block-scaled FP8 quantized forward.
+ *
+ * The library implements the quantized forward that a low-bit rollout decoder and the
+ * rollout-aligned training-side forward share (QaRL, Sec. 3.1, components 1 and 2):
+ *   Quant (Sec. 2.2, floating-point quantization):  s = max|W| / alpha,  W_q = [W / s]_FP8,
+ *                                                    alpha = 448 (e4m3);
+ *   low-bit GEMM with rescale (Sec. 2.2):            Y ~= (s_x s_w) (X_q W_q),
+ * applied with one fp32 scale per 128x128 weight block and per 1x128 activation group, on
+ * dense projections and on the routed-expert FFN (gate_up -> SwiGLU -> re-quantize -> down ->
+ * top-k weighted combine).  The K reduction order is fixed (App. C, batch-invariant kernel):
+ * every output row is bitwise identical whatever M, batch composition or tile schedule.
+ *
+ * Conventions for every call
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library never
+ *     allocates, frees or keeps caller memory in these calls.  `stream` is a cudaStream_t
+ *     passed as void*; all work is enqueued on it and the call returns without synchronizing.
+ *   - bf16 tensors are row-major arrays of 16-bit patterns; codes are e4m3 ("fn": no
+ *     infinities, max 448) bytes; scales are fp32.
+ *   - Pointers must be 16-byte aligned; N, K, H, I must be multiples of 128.  M >= 0 is
+ *     arbitrary; M = 0 enqueues nothing and returns QARL_OK.
+ *   - Errors the host can see (null pointer, bad shape, misalignment, small workspace) are
+ *     returned before anything is launched.  Errors only the device can see (an expert id
+ *     outside [0, E), an expert repeated within one token, a bounded wait that expired) set
+ *     the context's device status word; the outputs of that call are unspecified and the
+ *     error is reported by qarl_poll_device_status.
+ *   - A context belongs to one device and may be used from one host thread at a time.
+ *   - There is no CPU fallback: without an sm_100 device qarl_create fails.
+ */
+#ifndef QARL_H_
+#define QARL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qarl_ctx qarl_ctx; /* opaque */
+
+typedef enum {
+  QARL_OK = 0,
+  QARL_ERR_INVALID_ARG = -1,         /* null pointer, negative size, k out of range        */
+  QARL_ERR_UNSUPPORTED_SHAPE = -2,   /* N, K, H or I not a multiple of 128, sizes too big  */
+  QARL_ERR_MISALIGNED = -3,          /* a pointer or row stride is not 16-byte aligned     */
+  QARL_ERR_WORKSPACE_TOO_SMALL = -4,
+  QARL_ERR_UNSUPPORTED_DEVICE = -5,  /* not compute capability 10.x                        */
+  QARL_ERR_CUDA = -6,                /* a CUDA runtime / driver call failed                */
+  QARL_ERR_DEVICE_TIMEOUT = -7,      /* a bounded device-side wait expired                 */
+  QARL_ERR_BAD_EXPERT_ID = -8        /* id outside [0,E) or repeated within a token        */
+} qarl_status;
+
+/* Create a context on CUDA device `device` (host call; allocates a few bytes of device
+ * memory for the status word).  Fails with QARL_ERR_UNSUPPORTED_DEVICE unless the device
+ * has compute capability 10.x.  *out is set to NULL on failure. */
+int qarl_create(qarl_ctx** out, int device);
+void qarl_destroy(qarl_ctx* ctx);
+/* Static string for a status code (never NULL). */
+const char* qarl_status_string(int status);
+/* Synchronizes `stream`, then returns and clears the device status word (QARL_OK if no
+ * device-side error was recorded since the last poll). */
+int qarl_poll_device_status(qarl_ctx* ctx, void* stream);
+/* Text of the last CUDA error the context saw (host memory owned by the context). */
+const char* qarl_last_cuda_error(qarl_ctx* ctx);
+
+/* Sec. 2.2 Quant, 128x128 blocks (Sec. 3.1 item 2: done on the fly from the bf16 masters).
+ * in : w_bf16  device bf16 [E, N, K] row-major (E = 1 for a dense weight).
+ * out: codes   device u8   [E, N, K];  scales device f32 [E, N/128, K/128].
+ * Per block: amax = max|w|, s = max(amax, 2^-40) / 448, code = e4m3_rne_sat(w * (448 / max(amax, 2^-40))). */
+int qarl_quantize_weight(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
+                         uint8_t* codes, float* scales, void* stream);
+
+/* Sec. 2.2 Quant, 1x128 groups along K.
+ * in : x_bf16 device bf16 [M, K] with row stride ldx elements (ldx >= K, ldx % 8 == 0).
+ * out: codes  device u8 [M, K] (dense);  scales device f32 [M, K/128]. */
+int qarl_quantize_act(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                      uint8_t* codes, float* scales, void* stream);
+
+/* Sec. 2.2 low-bit GEMM with rescale, per 128-wide K-block:
+ *   y[m,n] = bf16( sum_kb  fl(s_x[m,kb] * s_w[n/128,kb]) * (x_q[m,kb,:] . w_q[n,kb,:]) ),
+ * fp32 accumulation, kb ascending, starting from 0 (fixed order, App. C).
+ * qarl_linear_fwd quantizes x first (as qarl_quantize_act) into `workspace`;
+ * qarl_linear_fwd_q takes activations that are already quantized.
+ * in : x_bf16 [M, K] dense;  w_codes [N, K], w_scales [N/128, K/128] from qarl_quantize_weight.
+ * out: y_bf16 [M, N];  y_f32 optional (may be NULL) fp32 copy of the accumulator [M, N].
+ * workspace: device scratch of at least qarl_linear_workspace_bytes(M, N, K) bytes, 256-byte
+ * aligned; its contents are undefined afterwards.  Calls that share a workspace must not
+ * overlap on the device. */
+size_t qarl_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int qarl_linear_fwd(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t K,
+                    const uint8_t* w_codes, const float* w_scales, int64_t N,
+                    void* y_bf16, float* y_f32, void* workspace, size_t workspace_bytes,
+                    void* stream);
+int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* x_codes, const float* x_scales,
+                      int64_t M, int64_t K, const uint8_t* w_codes, const float* w_scales,
+                      int64_t N, void* y_bf16, float* y_f32, void* stream);
+
+/* Optional dumps of the MoE layer's intermediates (every field may be NULL).  "Sorted
+ * order" is the order of token-expert pairs after grouping by expert: position q holds the
+ * flat pair sorted_pair[q] = t*k + j. */
+typedef struct {
+  int32_t* expert_offsets; /* [E+1]  first sorted position of each expert; [E] = M*k      */
+  int32_t* sorted_pair;    /* [M*k]  pairs stably sorted by expert id (ties by pair id)    */
+  void* gate_up_bf16;      /* [M*k, 2I] sorted order, bf16 of the gate_up accumulator      */
+  void* h_bf16;            /* [M*k, I]  sorted order, bf16( silu(gate) * up )              */
+  uint8_t* h_codes;        /* [M*k, I]  sorted order                                       */
+  float* h_scales;         /* [M*k, I/128] sorted order                                    */
+  float* down_f32;         /* [M*k, H]  sorted order, fp32 accumulator of the down GEMM    */
+} qarl_moe_debug;
+
+/* One routed-expert FFN layer on quantized weights (Sec. 3.1 items 1-2 applied to the MoE
+ * block; the paper notes MoE decode is memory-bound, App. D.1).  For every token t and slot j
+ * with expert e = topk_ids[t,j]:
+ *   x_q = quantize_act(x[t]);  gu = bf16(blockscaled(x_q, W13_e));  h = bf16(silu(gu[:I]) * gu[I:]);
+ *   h_q = quantize_act(h);     y = blockscaled(h_q, W2_e) (fp32);   c_j = bf16(topk_weights[t,j] * y);
+ *   out[t] = bf16( sum of float(c_j) over the token's slots in ASCENDING EXPERT ID, from 0 ).
+ * in : x_bf16 [M, H];  topk_ids i32 [M, k];  topk_weights f32 [M, k] (used as given);
+ *      w13_codes [E, 2I, H] (rows 0..I-1 gate, I..2I-1 up; scale blocks over the whole
+ *      [2I, H] matrix), w13_scales [E, 2I/128, H/128];  w2_codes [E, H, I], w2_scales [E, H/128, I/128].
+ * out: out_bf16 [M, H].
+ * Limits: 1 <= k <= 32, 1 <= E <= 1024, M*k < 2^31.
+ * workspace: at least qarl_moe_workspace_bytes(M, H, I, E, k) bytes, 256-byte aligned; the
+ * call clears what must start at zero; calls sharing a workspace must not overlap. */
+size_t qarl_moe_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k);
+int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
+                 const float* topk_weights, int64_t M, int64_t H, int64_t I, int64_t E,
+                 int64_t k, const uint8_t* w13_codes, const float* w13_scales,
+                 const uint8_t* w2_codes, const float* w2_scales, void* out_bf16,
+                 void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
+                 void* stream);
+
+/* Number of this library's kernels the context has launched since it was created. */
+int64_t qarl_launch_count(qarl_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QARL_H_ */

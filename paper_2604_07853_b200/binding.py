@@ -1,0 +1,232 @@
+"""Thin Python binding of the C-ABI library ``libqarl.so`` (see ``include/qarl.h``).
+
+Argument marshalling only: every step of the quantized forward runs in the library's CUDA
+kernels.  torch is used for device memory and streams.  There is no CPU path: loading fails
+loudly if the library has not been built, and creating a context fails without an sm_100
+device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqarl.so")
+
+QARL_OK = 0
+STATUS_NAMES = {
+    0: "QARL_OK", -1: "QARL_ERR_INVALID_ARG", -2: "QARL_ERR_UNSUPPORTED_SHAPE",
+    -3: "QARL_ERR_MISALIGNED", -4: "QARL_ERR_WORKSPACE_TOO_SMALL",
+    -5: "QARL_ERR_UNSUPPORTED_DEVICE", -6: "QARL_ERR_CUDA", -7: "QARL_ERR_DEVICE_TIMEOUT",
+    -8: "QARL_ERR_BAD_EXPERT_ID",
+}
+
+# every symbol include/qarl.h declares
+EXPORTS = [
+    "qarl_create", "qarl_destroy", "qarl_status_string", "qarl_poll_device_status",
+    "qarl_last_cuda_error", "qarl_quantize_weight", "qarl_quantize_act",
+    "qarl_linear_workspace_bytes", "qarl_linear_fwd", "qarl_linear_fwd_q",
+    "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
+]
+
+
+class QarlError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        name = STATUS_NAMES.get(status, str(status))
+        super().__init__(f"{name}{': ' + detail if detail else ''}")
+
+
+class MoeDebug(C.Structure):
+    _fields_ = [("expert_offsets", C.c_void_p), ("sorted_pair", C.c_void_p),
+                ("gate_up_bf16", C.c_void_p), ("h_bf16", C.c_void_p), ("h_codes", C.c_void_p),
+                ("h_scales", C.c_void_p), ("down_f32", C.c_void_p)]
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load libqarl.so and declare its signatures.  Raises if the library is not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2604_07853_b200.build` "
+            "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    i64, p, sz = C.c_int64, C.c_void_p, C.c_size_t
+    L.qarl_create.restype = C.c_int
+    L.qarl_create.argtypes = [C.POINTER(p), C.c_int]
+    L.qarl_destroy.restype = None
+    L.qarl_destroy.argtypes = [p]
+    L.qarl_status_string.restype = C.c_char_p
+    L.qarl_status_string.argtypes = [C.c_int]
+    L.qarl_poll_device_status.restype = C.c_int
+    L.qarl_poll_device_status.argtypes = [p, p]
+    L.qarl_last_cuda_error.restype = C.c_char_p
+    L.qarl_last_cuda_error.argtypes = [p]
+    L.qarl_quantize_weight.restype = C.c_int
+    L.qarl_quantize_weight.argtypes = [p, p, i64, i64, i64, p, p, p]
+    L.qarl_quantize_act.restype = C.c_int
+    L.qarl_quantize_act.argtypes = [p, p, i64, i64, i64, p, p, p]
+    L.qarl_linear_workspace_bytes.restype = sz
+    L.qarl_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.qarl_linear_fwd.restype = C.c_int
+    L.qarl_linear_fwd.argtypes = [p, p, i64, i64, p, p, i64, p, p, p, sz, p]
+    L.qarl_linear_fwd_q.restype = C.c_int
+    L.qarl_linear_fwd_q.argtypes = [p, p, p, i64, i64, p, p, i64, p, p, p]
+    L.qarl_moe_workspace_bytes.restype = sz
+    L.qarl_moe_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
+    L.qarl_moe_fwd.restype = C.c_int
+    L.qarl_moe_fwd.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, sz,
+                               C.POINTER(MoeDebug), p]
+    L.qarl_launch_count.restype = i64
+    L.qarl_launch_count.argtypes = [p]
+    _lib = L
+    return L
+
+
+def _ptr(t: torch.Tensor | None):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Context:
+    """One qarl_ctx on one CUDA device.  Methods take and return torch CUDA tensors; bf16
+    tensors are torch.bfloat16, codes torch.uint8, scales torch.float32."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load()
+        if not torch.cuda.is_available():
+            raise QarlError(-5, "no CUDA device (the library has no CPU fallback)")
+        self.device = torch.device("cuda", device)
+        h = C.c_void_p()
+        rc = self.lib.qarl_create(C.byref(h), device)
+        if rc != QARL_OK:
+            raise QarlError(rc)
+        self.h = h
+        self._ws: torch.Tensor | None = None
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.qarl_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ helpers
+    def _check(self, rc: int):
+        if rc != QARL_OK:
+            detail = self.lib.qarl_last_cuda_error(self.h).decode() if rc == -6 else ""
+            raise QarlError(rc, detail)
+
+    def workspace(self, nbytes: int) -> torch.Tensor:
+        """A cached device scratch buffer of at least nbytes (256-byte aligned)."""
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def poll(self) -> int:
+        """Synchronize the current stream; return and clear the device status word."""
+        return int(self.lib.qarl_poll_device_status(self.h, _stream()))
+
+    def check_device_status(self):
+        rc = self.poll()
+        if rc != QARL_OK:
+            raise QarlError(rc)
+
+    def launch_count(self) -> int:
+        return int(self.lib.qarl_launch_count(self.h))
+
+    # ------------------------------------------------------------------ calls
+    def quantize_weight(self, w: torch.Tensor, codes=None, scales=None):
+        """w bf16 [E, N, K] or [N, K] -> (codes u8 same shape, scales f32 [.., N/128, K/128])."""
+        assert w.dtype == torch.bfloat16 and w.is_cuda and w.is_contiguous()
+        shape = w.shape
+        E, N, K = (1, *shape) if w.dim() == 2 else shape
+        if codes is None:
+            codes = torch.empty(shape, dtype=torch.uint8, device=w.device)
+        if scales is None:
+            scales = torch.empty((*shape[:-2], N // 128, K // 128), dtype=torch.float32, device=w.device)
+        self._check(self.lib.qarl_quantize_weight(self.h, _ptr(w), E, N, K, _ptr(codes), _ptr(scales), _stream()))
+        return codes, scales
+
+    def quantize_act(self, x: torch.Tensor, codes=None, scales=None):
+        """x bf16 [M, K] (rows may be strided) -> (codes u8 [M, K], scales f32 [M, K/128])."""
+        assert x.dtype == torch.bfloat16 and x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+        M, K = x.shape
+        ldx = x.stride(0) if M > 1 else K
+        if codes is None:
+            codes = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+        if scales is None:
+            scales = torch.empty((M, K // 128), dtype=torch.float32, device=x.device)
+        self._check(self.lib.qarl_quantize_act(self.h, _ptr(x), M, K, ldx, _ptr(codes), _ptr(scales), _stream()))
+        return codes, scales
+
+    def linear_fwd(self, x, w_codes, w_scales, out=None, want_f32: bool = False):
+        """y = blockscaled(quantize_act(x), W) -> y bf16 [M, N] (and the fp32 accumulator)."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        M, K = x.shape
+        N = w_codes.shape[0]
+        y = out if out is not None else torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        y32 = torch.empty((M, N), dtype=torch.float32, device=x.device) if want_f32 else None
+        nbytes = int(self.lib.qarl_linear_workspace_bytes(M, N, K))
+        ws = self.workspace(nbytes)
+        self._check(self.lib.qarl_linear_fwd(self.h, _ptr(x), M, K, _ptr(w_codes), _ptr(w_scales), N,
+                                             _ptr(y), _ptr(y32), _ptr(ws), ws.numel(), _stream()))
+        return (y, y32) if want_f32 else y
+
+    def linear_fwd_q(self, x_codes, x_scales, w_codes, w_scales, out=None, want_f32: bool = False):
+        M, K = x_codes.shape
+        N = w_codes.shape[0]
+        y = out if out is not None else torch.empty((M, N), dtype=torch.bfloat16, device=x_codes.device)
+        y32 = torch.empty((M, N), dtype=torch.float32, device=x_codes.device) if want_f32 else None
+        self._check(self.lib.qarl_linear_fwd_q(self.h, _ptr(x_codes), _ptr(x_scales), M, K, _ptr(w_codes),
+                                               _ptr(w_scales), N, _ptr(y), _ptr(y32), _stream()))
+        return (y, y32) if want_f32 else y
+
+    def moe_workspace_bytes(self, M, H, I, E, k) -> int:
+        return int(self.lib.qarl_moe_workspace_bytes(M, H, I, E, k))
+
+    def moe_fwd(self, x, topk_ids, topk_weights, w13_codes, w13_scales, w2_codes, w2_scales,
+                out=None, debug: bool = False, workspace: torch.Tensor | None = None):
+        """One routed-expert FFN layer -> out bf16 [M, H] (and a dict of dumps if debug)."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        assert topk_ids.dtype == torch.int32 and topk_weights.dtype == torch.float32
+        M, H = x.shape
+        k = topk_ids.shape[1]
+        E, I2, _ = w13_codes.shape
+        I = I2 // 2
+        P = M * k
+        y = out if out is not None else torch.empty((M, H), dtype=torch.bfloat16, device=x.device)
+        nbytes = self.moe_workspace_bytes(M, H, I, E, k)
+        ws = workspace if workspace is not None else self.workspace(nbytes)
+        d, dbg = None, None
+        if debug:
+            dev = x.device
+            d = dict(expert_offsets=torch.zeros(E + 1, dtype=torch.int32, device=dev),
+                     sorted_pair=torch.zeros(P, dtype=torch.int32, device=dev),
+                     gate_up=torch.zeros((P, 2 * I), dtype=torch.bfloat16, device=dev),
+                     h=torch.zeros((P, I), dtype=torch.bfloat16, device=dev),
+                     h_codes=torch.zeros((P, I), dtype=torch.uint8, device=dev),
+                     h_scales=torch.zeros((P, I // 128), dtype=torch.float32, device=dev),
+                     down_f32=torch.zeros((P, H), dtype=torch.float32, device=dev))
+            dbg = MoeDebug(d["expert_offsets"].data_ptr(), d["sorted_pair"].data_ptr(),
+                           d["gate_up"].data_ptr(), d["h"].data_ptr(), d["h_codes"].data_ptr(),
+                           d["h_scales"].data_ptr(), d["down_f32"].data_ptr())
+        self._check(self.lib.qarl_moe_fwd(self.h, _ptr(x), _ptr(topk_ids), _ptr(topk_weights), M, H, I, E, k,
+                                          _ptr(w13_codes), _ptr(w13_scales), _ptr(w2_codes), _ptr(w2_scales),
+                                          _ptr(y), _ptr(ws), ws.numel(),
+                                          C.byref(dbg) if dbg is not None else None, _stream()))
+        return (y, d) if debug else y

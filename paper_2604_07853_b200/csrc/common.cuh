@@ -1,0 +1,108 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/qarl.h"
+
+namespace qarl {
+
+constexpr int kBlock = 128;               // 128x128 weight blocks, 1x128 activation groups
+constexpr float kAlpha = 448.0f;          // max finite e4m3 (Sec. 2.2)
+constexpr float kAmaxFloor = 0x1p-40f;    // all-zero block: amax_c = max(amax, 2^-40)
+
+// Scale of one block and the multiplier used to form the codes (Sec. 2.2, Quant):
+// s = fl(amax_c / 448), code = e4m3(fl(x * fl(448 / amax_c))).  IEEE division, no fast math.
+__device__ __forceinline__ float block_scale(float amax, float* inv) {
+  const float amax_c = fmaxf(amax, kAmaxFloor);
+  *inv = __fdiv_rn(kAlpha, amax_c);
+  return __fdiv_rn(amax_c, kAlpha);
+}
+
+// Two fp32 -> two e4m3 codes (round to nearest even, saturate to +-448); lo in bits [0,8).
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint32_t cvt_e4m3x4(float a, float b, float c, float d) {
+  return cvt_e4m3x2(a, b) | (cvt_e4m3x2(c, d) << 16);
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+// fp32 -> bf16 bits, round to nearest even.
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(f)));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+}
+
+// Device status word protocol: first error wins.
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+// ---- launchers (host), one per kernel family; every launcher returns a cudaError_t -------
+struct Launch {
+  cudaStream_t stream;
+  int device;
+  int sm_count;
+  int* d_status;
+  int64_t* launches;  // host counter
+};
+
+cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
+                                   uint8_t* codes, float* scales);
+// dst_rows == nullptr: row m of the output is m.  Otherwise each input row t is written to
+// the `fanout` output rows dst_rows[t*fanout + j] (quantize once, scatter k times).
+cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
+                                uint8_t* codes, float* scales, const int32_t* dst_rows, int fanout);
+
+struct PermuteBuffers {
+  int32_t* chunk_hist;   // [nchunks, E]
+  int32_t* offsets;      // [E+1]
+  int32_t* sorted_pair;  // [P]
+  int32_t* pos_of_pair;  // [P]
+};
+int64_t permute_num_chunks(int64_t P);
+cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
+                           const PermuteBuffers& b);
+
+cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
+                           int64_t H, int64_t E, uint16_t* out);
+
+enum GemmMode { kModeLinear = 0, kModeGateUp = 1, kModeDown = 2 };
+
+struct GemmArgs {
+  GemmMode mode;
+  // A: codes [rows_total, K] (rows = tokens for linear, sorted pairs for MoE) and scales [rows_total, K/128]
+  const uint8_t* a_codes;
+  const float* a_scales;
+  int64_t rows_total;
+  int64_t K;
+  // B: codes [E, N, K] and scales [E, N/128, K/128]
+  const uint8_t* b_codes;
+  const float* b_scales;
+  int64_t N;
+  int64_t E;
+  // row groups: expert e owns rows offsets[e] .. offsets[e+1]-1 (device array).  nullptr:
+  // one group of rows_total rows (dense).
+  const int32_t* offsets;
+  // outputs
+  uint16_t* out_bf16;        // linear: y [M, N]; gate_up (debug): gate_up [P, 2I]; down: contrib [P, H] by pair id
+  float* out_f32;            // optional fp32 accumulator dump (linear: [M,N]; down: [P,H] sorted order)
+  uint8_t* h_codes;          // gate_up: [P, I]
+  float* h_scales;           // gate_up: [P, I/128]
+  uint16_t* h_bf16;          // gate_up (debug): [P, I]
+  const int32_t* sorted_pair;   // down: [P]
+  const float* pair_weights;    // down: [M*k] by flat pair id
+};
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// Returns cudaSuccess, or an error; *cu_err receives a driver error from tensor-map encoding.
+cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
+
+}  // namespace qarl

@@ -1,0 +1,274 @@
+// Token-expert grouping: a stable counting sort of the M*k flat pairs p = t*k + j by expert
+// id, built from warp-level match/ballot prefix sums.  Output (exactly one correct answer):
+//   offsets[e]     first sorted position of expert e, offsets[E] = P
+//   sorted_pair[q] the pair at sorted position q (ties by ascending pair id)
+//   pos_of_pair[p] the inverse permutation
+// Integer work only.  Ids outside [0, E) are reported through the status word and skipped
+// (nothing is written for them), so the kernels stay memory-safe on bad input.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace qarl {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kPairsPerWarp = 256;
+constexpr int kChunk = kWarps * kPairsPerWarp;  // 2048 pairs per CTA
+
+// Per-warp histogram of the warp's contiguous 256-pair slice into hist_w[0..E).  Lanes with
+// equal ids are found with match_any; the lowest such lane adds the group's size, so no
+// atomics are needed (one warp owns hist_w).
+__device__ __forceinline__ void warp_histogram(const int32_t* __restrict__ ids, int64_t p0, int64_t P, int E,
+                                               int32_t* hist_w, int* status) {
+  const int lane = threadIdx.x & 31;
+  for (int r = 0; r < kPairsPerWarp / 32; ++r) {
+    const int64_t p = p0 + r * 32 + lane;
+    int e = -1;
+    if (p < P) {
+      e = ids[p];
+      if (e < 0 || e >= E) {
+        set_status(status, QARL_ERR_BAD_EXPERT_ID);
+        e = -1;
+      }
+    }
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
+    __syncwarp();
+  }
+}
+
+// Walk the warp's slice again in order; cursor_w[e] holds the next free sorted position for
+// expert e within this warp's slice.  rank among equal-id lanes = popc(peers below me).
+__device__ __forceinline__ void warp_scatter(const int32_t* __restrict__ ids, int64_t p0, int64_t P, int E,
+                                             int32_t* cursor_w, int32_t* __restrict__ sorted_pair,
+                                             int32_t* __restrict__ pos_of_pair) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t lt = (1u << lane) - 1u;
+  for (int r = 0; r < kPairsPerWarp / 32; ++r) {
+    const int64_t p = p0 + r * 32 + lane;
+    int e = -1;
+    if (p < P) {
+      e = ids[p];
+      if (e < 0 || e >= E) e = -1;
+    }
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    int pos = -1;
+    if (e >= 0) pos = cursor_w[e] + __popc(peers & lt);
+    __syncwarp();
+    if (e >= 0 && (__ffs(peers) - 1) == lane) cursor_w[e] += __popc(peers);
+    __syncwarp();
+    if (e >= 0) {
+      sorted_pair[pos] = static_cast<int32_t>(p);
+      pos_of_pair[p] = pos;
+    }
+  }
+}
+
+// Exclusive scan of a[0..n) in shared memory by the whole CTA (n <= 1024); returns the total.
+// scratch: 33 ints of shared memory.
+__device__ int block_exclusive_scan(int32_t* a, int n, int32_t* scratch) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int items = (n + nt - 1) / nt;
+  const int i0 = tid * items;
+  int sum = 0;
+  for (int i = 0; i < items; ++i)
+    if (i0 + i < n) sum += a[i0 + i];
+  // inclusive warp scan of the per-thread sums
+  int inc = sum;
+  const int lane = tid & 31, wid = tid >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) scratch[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    const int nw = nt >> 5;
+    int v = lane < nw ? scratch[lane] : 0;
+    int vi = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xFFFFFFFFu, vi, o);
+      if (lane >= o) vi += u;
+    }
+    if (lane < nw) scratch[lane] = vi - v;  // exclusive warp bases
+    if (lane == 31) scratch[32] = vi;       // total
+  }
+  __syncthreads();
+  int run = scratch[wid] + inc - sum;
+  for (int i = 0; i < items; ++i)
+    if (i0 + i < n) {
+      const int v = a[i0 + i];
+      a[i0 + i] = run;
+      run += v;
+    }
+  __syncthreads();
+  return scratch[32];
+}
+
+// ---- small problems (P <= 2048): one CTA does histogram, scan and scatter ----------------
+__global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int32_t* __restrict__ ids, int64_t P,
+                                                                      int E, int32_t* __restrict__ offsets,
+                                                                      int32_t* __restrict__ sorted_pair,
+                                                                      int32_t* __restrict__ pos_of_pair,
+                                                                      int* status) {
+  extern __shared__ int32_t sm[];
+  int32_t* whist = sm;                 // [kWarps][E]
+  int32_t* total = sm + kWarps * E;    // [E]
+  int32_t* scratch = total + E;        // [33]
+  const int tid = threadIdx.x, wid = tid >> 5;
+  for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
+  __syncthreads();
+  warp_histogram(ids, static_cast<int64_t>(wid) * kPairsPerWarp, P, E, whist + wid * E, status);
+  __syncthreads();
+  for (int e = tid; e < E; e += kThreads) {
+    int s = 0;
+    for (int w = 0; w < kWarps; ++w) s += whist[w * E + e];
+    total[e] = s;
+  }
+  __syncthreads();
+  const int all = block_exclusive_scan(total, E, scratch);
+  for (int e = tid; e < E; e += kThreads) {
+    int run = total[e];
+    offsets[e] = run;
+    for (int w = 0; w < kWarps; ++w) {
+      const int c = whist[w * E + e];
+      whist[w * E + e] = run;
+      run += c;
+    }
+  }
+  if (tid == 0) offsets[E] = all;
+  __syncthreads();
+  warp_scatter(ids, static_cast<int64_t>(wid) * kPairsPerWarp, P, E, whist + wid * E, sorted_pair, pos_of_pair);
+}
+
+// ---- large problems: per-chunk histogram, one-CTA scan, per-chunk scatter ----------------
+__global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ ids, int64_t P, int E,
+                                                                int32_t* __restrict__ chunk_hist, int* status) {
+  extern __shared__ int32_t sm[];
+  int32_t* whist = sm;
+  const int tid = threadIdx.x, wid = tid >> 5;
+  for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
+  __syncthreads();
+  const int64_t p0 = static_cast<int64_t>(blockIdx.x) * kChunk + static_cast<int64_t>(wid) * kPairsPerWarp;
+  warp_histogram(ids, p0, P, E, whist + wid * E, status);
+  __syncthreads();
+  for (int e = tid; e < E; e += kThreads) {
+    int s = 0;
+    for (int w = 0; w < kWarps; ++w) s += whist[w * E + e];
+    chunk_hist[static_cast<int64_t>(blockIdx.x) * E + e] = s;
+  }
+}
+
+// One CTA of 1024 threads.  Turns chunk_hist[c][e] into the exclusive running count of expert
+// e over chunks 0..c-1 and writes the expert offsets.  Threads are laid out (g, e): group g
+// handles a contiguous range of chunks for expert e so the chunk walk is G-way parallel.
+__global__ void __launch_bounds__(1024) permute_scan_kernel(int32_t* __restrict__ chunk_hist, int nchunks, int E,
+                                                            int32_t* __restrict__ offsets) {
+  extern __shared__ int32_t sm[];
+  const int G = max(1, min(static_cast<int>(blockDim.x) / E, nchunks));
+  int32_t* part = sm;            // [G][E]
+  int32_t* total = sm + G * E;   // [E]
+  int32_t* scratch = total + E;  // [33]
+  const int tid = threadIdx.x;
+  const int cpg = (nchunks + G - 1) / G;
+  const int g = tid / E, e = tid % E;
+  const bool active = g < G;
+  const int c0 = g * cpg, c1 = min(c0 + cpg, nchunks);
+  if (active) {
+    int s = 0;
+    for (int c = c0; c < c1; ++c) s += chunk_hist[static_cast<int64_t>(c) * E + e];
+    part[g * E + e] = s;
+  }
+  __syncthreads();
+  if (tid < E) {
+    int run = 0;
+    for (int gg = 0; gg < G; ++gg) {
+      const int v = part[gg * E + tid];
+      part[gg * E + tid] = run;
+      run += v;
+    }
+    total[tid] = run;
+  }
+  __syncthreads();
+  const int all = block_exclusive_scan(total, E, scratch);
+  if (tid < E) offsets[tid] = total[tid];
+  if (tid == 0) offsets[E] = all;
+  if (active) {
+    int run = part[g * E + e];
+    for (int c = c0; c < c1; ++c) {
+      const int64_t i = static_cast<int64_t>(c) * E + e;
+      const int v = chunk_hist[i];
+      chunk_hist[i] = run;
+      run += v;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) permute_scatter_kernel(const int32_t* __restrict__ ids, int64_t P, int E,
+                                                                   const int32_t* __restrict__ chunk_hist,
+                                                                   const int32_t* __restrict__ offsets,
+                                                                   int32_t* __restrict__ sorted_pair,
+                                                                   int32_t* __restrict__ pos_of_pair, int* status) {
+  extern __shared__ int32_t sm[];
+  int32_t* whist = sm;
+  const int tid = threadIdx.x, wid = tid >> 5;
+  for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
+  __syncthreads();
+  const int64_t p0 = static_cast<int64_t>(blockIdx.x) * kChunk + static_cast<int64_t>(wid) * kPairsPerWarp;
+  warp_histogram(ids, p0, P, E, whist + wid * E, status);
+  __syncthreads();
+  for (int e = tid; e < E; e += kThreads) {
+    int run = offsets[e] + chunk_hist[static_cast<int64_t>(blockIdx.x) * E + e];
+    for (int w = 0; w < kWarps; ++w) {
+      const int c = whist[w * E + e];
+      whist[w * E + e] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  warp_scatter(ids, p0, P, E, whist + wid * E, sorted_pair, pos_of_pair);
+}
+
+}  // namespace
+
+int64_t permute_num_chunks(int64_t P) { return (P + kChunk - 1) / kChunk; }
+
+cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
+                           const PermuteBuffers& b) {
+  const int64_t P = M * k;
+  const int e = static_cast<int>(E);
+  const int64_t nchunks = permute_num_chunks(P);
+  cudaError_t err;
+  if (nchunks <= 1) {
+    const size_t smem = (static_cast<size_t>(kWarps) * e + e + 33) * sizeof(int32_t);
+    if (smem > 48 * 1024) {
+      err = cudaFuncSetAttribute(permute_single_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem));
+      if (err != cudaSuccess) return err;
+    }
+    permute_single_cta_kernel<<<1, kThreads, smem, L.stream>>>(ids, P, e, b.offsets, b.sorted_pair, b.pos_of_pair,
+                                                               L.d_status);
+    ++*L.launches;
+    return cudaGetLastError();
+  }
+  const size_t smem_h = static_cast<size_t>(kWarps) * e * sizeof(int32_t);
+  const int G = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(1024 / e, nchunks)));
+  const size_t smem_s = (static_cast<size_t>(G) * e + e + 33) * sizeof(int32_t);
+  permute_hist_kernel<<<static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream>>>(ids, P, e, b.chunk_hist,
+                                                                                     L.d_status);
+  ++*L.launches;
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  permute_scan_kernel<<<1, 1024, smem_s, L.stream>>>(b.chunk_hist, static_cast<int>(nchunks), e, b.offsets);
+  ++*L.launches;
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  permute_scatter_kernel<<<static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream>>>(
+      ids, P, e, b.chunk_hist, b.offsets, b.sorted_pair, b.pos_of_pair, L.d_status);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+}  // namespace qarl
