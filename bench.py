@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 block-scaled MoE forward on B200 (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path over one synthetic batch of the training-forward
+MoE shape (M = 32768 tokens of hidden 2048, 128 experts, top-8, Zipf(1.1) popularity):
+on-the-fly weight quantization of the layer's bf16 masters (w13, w2), then the routed MoE FFN
+(quantize activations, group by expert, gate_up grouped GEMM + SwiGLU + re-quantization, down
+grouped GEMM + weighting, fixed-order combine).  The decode shape (M = 256, weights already
+quantized, as in the rollout engine) is measured in the same run and reported under "decode".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched by torch.distributed.run, one rank per GPU: data-parallel replicas over
+independent token batches, weights replicated, no collective on the data path (weak scaling).
+--impl reference times the CPU oracle (test infrastructure) on the host cores on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+H, I, E, TOPK = 2048, 768, 128, 8
+M_TRAIN, M_DECODE = 32768, 256
+FLOP_PER_TOKEN = TOPK * 2 * (H * 2 * I + I * H)          # 75.5 MFLOP
+METRIC = "FP8 MoE-layer tokens/s"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def peaks():
+    """Measured roofline denominators (generated file), else the documented fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(source="measured", hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])))
+    return dict(source="fallback", hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0)
+
+
+# --------------------------------------------------------------------------- inputs (device)
+def make_inputs(m: int, seed: int, device, zipf: bool):
+    """Synthetic layer of Qwen3-30B-A3B FFN shape, generated on the device: W ~ N(0, 0.02^2),
+    X ~ N(0, 1) with 1% of entries x50, router logits ~ N(0, 1) (+ ln Zipf(1.1) popularity for
+    the training shape), top-8 with softmax weights over the selected logits."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    w13 = (torch.randn((E, 2 * I, H), generator=g, device=device) * 0.02).to(torch.bfloat16)
+    w2 = (torch.randn((E, H, I), generator=g, device=device) * 0.02).to(torch.bfloat16)
+    x = torch.randn((m, H), generator=g, device=device)
+    x = torch.where(torch.rand((m, H), generator=g, device=device) < 0.01, x * 50.0, x).to(torch.bfloat16)
+    logits = torch.randn((m, E), generator=g, device=device, dtype=torch.float64)
+    if zipf:
+        rank = torch.randperm(E, generator=g, device=device).to(torch.float64) + 1.0
+        p = rank ** -1.1
+        logits = logits + torch.log(p / p.sum())[None, :]
+    sel, ids = torch.topk(logits, TOPK, dim=1)
+    wts = torch.softmax(sel, dim=1).to(torch.float32)
+    return w13, w2, x, ids.to(torch.int32).contiguous(), wts.contiguous()
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self, gpu_index: int) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        self.p.wait()
+        self.f.flush()
+        sm, smax, reasons, power = [], [], set(), []
+        for line in open(self.f.name):
+            c = [t.strip() for t in line.split(",")]
+            if len(c) < 9 or not c[0].isdigit() or int(c[0]) != gpu_index:
+                continue
+            try:
+                sm.append(float(c[1])); smax.append(float(c[2])); power.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, v in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.f.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s, w in zip(sm, power) if w > 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def cpu_reference_step(state, n_tokens, n_experts_q):
+    """One bounded oracle step; returns the estimated seconds of a full step (scaled linearly
+    in experts for the quantization part and in tokens for the layer part)."""
+    import oracle
+    t0 = time.perf_counter()
+    oracle.quantize_weight(state["w13"][:n_experts_q])
+    oracle.quantize_weight(state["w2"][:n_experts_q])
+    t_q = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.moe(state["x"][:n_tokens], state["ids"][:n_tokens], state["wts"][:n_tokens],
+               state["w13c"], state["w13s"], state["w2c"], state["w2s"])
+    t_m = time.perf_counter() - t0
+    return t_q * (E / n_experts_q) + t_m * (M_TRAIN / n_tokens), t_q + t_m
+
+
+def cpu_state(seed: int, n_tokens: int):
+    """Host copies of a synthetic layer for the oracle (same recipe, host RNG), with the
+    weights quantized by the oracle (untimed set-up)."""
+    import oracle
+    from paper_2604_07853_b200 import inputs
+    rng = np.random.default_rng(seed)
+    w13 = inputs.weight_bf16(rng, E, 2 * I, H)
+    w2 = inputs.weight_bf16(rng, E, H, I)
+    x = inputs.act_bf16(rng, n_tokens, H)
+    ids, wts = inputs.routing(rng, n_tokens, E, TOPK, inputs.zipf_log_popularity(rng, E, 1.1))
+    w13c, w13s = oracle.quantize_weight(w13)
+    w2c, w2s = oracle.quantize_weight(w2)
+    return dict(w13=w13, w2=w2, x=x, ids=ids, wts=wts, w13c=w13c, w13s=w13s, w2c=w2c, w2s=w2s)
+
+
+def run_reference(args, rank: int):
+    """--impl reference: the CPU oracle as it stands, on the host cores, bounded sample."""
+    if rank != 0:
+        return
+    import oracle
+    n_tokens, n_exp = 16, 1
+    st = cpu_state(4, n_tokens)
+    for _ in range(args.warmup):
+        cpu_reference_step(st, n_tokens, n_exp)
+    est, raw = [], []
+    for _ in range(args.steps):
+        e, r = cpu_reference_step(st, n_tokens, n_exp)
+        est.append(e); raw.append(r)
+    full_step_s = sum(est) / len(est)
+    value = M_TRAIN / full_step_s
+    cores = oracle.num_threads()
+    sample = (f"per step: oracle quantize_weight on {n_exp} of {E} experts (scaled x{E // n_exp}) + "
+              f"oracle MoE layer on {n_tokens} of {M_TRAIN} tokens (scaled x{M_TRAIN // n_tokens})")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": full_step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
+        "data": "synthetic", "config": config_dict(args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "measured_s_per_sample_step": sum(raw) / len(raw),
+    }))
+
+
+def config_dict(n_gpus: int) -> dict:
+    return {"workload": "moe_ffn_train_fwd_M32768_zipf1.1 (+ on-the-fly weight quantization)",
+            "tokens_per_gpu": M_TRAIN, "hidden": H, "intermediate": I, "experts": E, "top_k": TOPK,
+            "format": "fp8 e4m3, 128x128 weight blocks, 1x128 activation groups, fp32 scales",
+            "l2": "inputs larger than L2 (1.2 GB bf16 masters + 0.6 GB codes + 0.13 GB activations per step)",
+            "parallelism": f"dp{n_gpus} replicas, no collective"}
+
+
+# --------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch.distributed as dist
+    from paper_2604_07853_b200 import binding, build
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if local_rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    ctx = binding.Context(local_rank)
+    pk = peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v: float) -> float:
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---------------- training-forward shape: the headline step
+    w13, w2, x, ids, wts = make_inputs(M_TRAIN, 1000 + rank, dev, zipf=True)
+    w13c = torch.empty(w13.shape, dtype=torch.uint8, device=dev)
+    w13s = torch.empty((E, 2 * I // 128, H // 128), dtype=torch.float32, device=dev)
+    w2c = torch.empty(w2.shape, dtype=torch.uint8, device=dev)
+    w2s = torch.empty((E, H // 128, I // 128), dtype=torch.float32, device=dev)
+    out = torch.empty((M_TRAIN, H), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(ctx.moe_workspace_bytes(M_TRAIN, H, I, E, TOPK), dtype=torch.uint8, device=dev)
+
+    def step(xd=x, idd=ids, wtd=wts):
+        ctx.quantize_weight(w13, w13c, w13s)
+        ctx.quantize_weight(w2, w2c, w2s)
+        ctx.moe_fwd(xd, idd, wtd, w13c, w13s, w2c, w2s, out=out, workspace=ws)
+
+    for _ in range(args.warmup):
+        step()
+    ctx.check_device_status()
+    sampler = ClockSampler()
+    barrier()
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    ctx.profile_begin(max_marks=args.steps * 16 + 8)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    stages = ctx.profile_end()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop(local_rank) if rank == 0 else None
+    ctx.check_device_status()
+    ms_step = ms_total / args.steps
+    value = world * M_TRAIN / (ms_step * 1e-3)
+
+    # ---------------- end to end: pinned host inputs in, result out, copies inside the timing
+    hx, hids, hwts = x.cpu().pin_memory(), ids.cpu().pin_memory(), wts.cpu().pin_memory()
+    hout = torch.empty((M_TRAIN, H), dtype=torch.bfloat16).pin_memory()
+    dx, dids, dwts = torch.empty_like(x), torch.empty_like(ids), torch.empty_like(wts)
+
+    def e2e_step():
+        dx.copy_(hx, non_blocking=True)
+        dids.copy_(hids, non_blocking=True)
+        dwts.copy_(hwts, non_blocking=True)
+        step(dx, dids, dwts)
+        hout.copy_(out, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
+    e2e = {"value": world * M_TRAIN / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": hx.numel() * 2 + hids.numel() * 4 + hwts.numel() * 4,
+           "d2h_bytes_per_step": hout.numel() * 2,
+           "note": "bf16 masters stay resident on the device; activations, routing in and output out per step"}
+
+    # ---------------- roofline of the dominant kernel (gate_up grouped GEMM, tensor-bound)
+    gu_ms, gu_n = stages["gate_up_gemm"]
+    gu_ms_avg = gu_ms / max(gu_n, 1)
+    gu_flops = M_TRAIN * TOPK * 2.0 * H * 2 * I                     # algorithmic flops per launch
+    achieved = gu_flops / (gu_ms_avg * 1e-3) / 1e12
+    peak = 2.0 * pk["bf16_sustained"]                               # fp8 = 2 x bf16 (nominal ratio)
+    roofline = {"kernel": "gemm_blockscaled_kernel<gate_up>", "bound": "tensor", "achieved": achieved,
+                "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": f"2 x bf16 sustained of {pk['source']}", "traffic": None,
+                "ms_per_launch": gu_ms_avg, "frac_of_nominal_4500": achieved / 4500.0}
+    stage_ms = {k: (v[0] / max(args.steps, 1)) for k, v in stages.items()}
+    layer_ms = sum(stage_ms[k] for k in ("permute", "quantize_act", "gate_up_gemm", "down_gemm", "combine"))
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic", "config": config_dict(world),
+        "tflops": value * FLOP_PER_TOKEN / 1e12, "stage_ms_per_step": stage_ms,
+        "moe_layer_only": {"ms": layer_ms, "tokens_per_s": M_TRAIN / (layer_ms * 1e-3),
+                           "tflops": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12,
+                           "frac_fp8_peak_measured": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12 / peak,
+                           "frac_fp8_peak_nominal_4500": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12 / 4500.0},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches * world, "clocks": clocks,
+    }
+
+    # ---------------- decode shape (rollout engine: weights already quantized)
+    if not args.no_decode:
+        del w13, w2
+        _, _, xd, idd, wtd = make_inputs(M_DECODE, 2000 + rank, dev, zipf=False)
+        outd = torch.empty((M_DECODE, H), dtype=torch.bfloat16, device=dev)
+        # rotate over two copies of the codes so consecutive steps never re-read a resident copy
+        sets = [(w13c, w13s, w2c, w2s), (w13c.clone(), w13s.clone(), w2c.clone(), w2s.clone())]
+        dsteps = max(args.steps, 20) * 5
+
+        def dstep(i):
+            a, b, c, d = sets[i & 1]
+            ctx.moe_fwd(xd, idd, wtd, a, b, c, d, out=outd, workspace=ws)
+
+        for i in range(10):
+            dstep(i)
+        barrier()
+        ev0.record()
+        for i in range(dsteps):
+            dstep(i)
+        ev1.record()
+        barrier()
+        d_ms = max_over_ranks(ev0.elapsed_time(ev1)) / dsteps
+        ctx.profile_begin(max_marks=dsteps * 8 + 8)
+        for i in range(dsteps):
+            dstep(i)
+        dst = ctx.profile_end()
+        ctx.check_device_status()
+        wbytes = w13c.numel() + w2c.numel() + (w13s.numel() + w2s.numel()) * 4 + 2 * M_DECODE * H * 2
+        kern_ms = sum(v[0] for v in dst.values()) / dsteps
+        gu_d = dst["gate_up_gemm"][0] / max(dst["gate_up_gemm"][1], 1)
+        dn_d = dst["down_gemm"][0] / max(dst["down_gemm"][1], 1)
+        result["decode"] = {
+            "workload": "moe_ffn_decode_M256 (weights pre-quantized, two weight copies alternated: 1.2 GB > L2)",
+            "ms_per_step": d_ms, "tokens_per_s": world * M_DECODE / (d_ms * 1e-3),
+            "algorithmic_bytes": wbytes, "gbs": wbytes / (d_ms * 1e-3) / 1e9,
+            "frac_hbm_measured": wbytes / (d_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+            "frac_hbm_nominal_8000": wbytes / (d_ms * 1e-3) / 1e9 / 8000.0,
+            "stage_ms": {k: v[0] / dsteps for k, v in dst.items() if v[1]},
+            "gate_up_gbs": (w13c.numel() + w13s.numel() * 4) / (gu_d * 1e-3) / 1e9,
+            "down_gbs": (w2c.numel() + w2s.numel() * 4) / (dn_d * 1e-3) / 1e9,
+            "sum_of_kernel_ms": kern_ms,
+        }
+
+    # ---------------- CPU oracle baseline (rank 0, N = 1 only), bounded sample
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_tokens, n_exp = 128, 2
+        st = cpu_state(4, n_tokens)
+        est, raw = cpu_reference_step(st, n_tokens, n_exp)
+        result["cpu_baseline"] = {
+            "value": M_TRAIN / est, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": (f"oracle quantize_weight on {n_exp} of {E} experts (x{E // n_exp}) + oracle MoE layer on "
+                       f"{n_tokens} of {M_TRAIN} tokens (x{M_TRAIN // n_tokens}); {raw:.1f} s of CPU work"),
+        }
+    elif rank == 0:
+        result["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

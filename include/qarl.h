@@ -17,7 +17,8 @@
  *     passed as void*; all work is enqueued on it and the call returns without synchronizing.
  *   - bf16 tensors are row-major arrays of 16-bit patterns; codes are e4m3 ("fn": no
  *     infinities, max 448) bytes; scales are fp32.
- *   - Pointers must be 16-byte aligned; N, K, H, I must be multiples of 128.  M >= 0 is
+ *   - Pointers to bf16, code and fp32-output tensors must be 16-byte aligned (scale and id
+ *     arrays: 4-byte); N, K, H, I must be multiples of 128.  M >= 0 is
  *     arbitrary; M = 0 enqueues nothing and returns QARL_OK.
  *   - Errors the host can see (null pointer, bad shape, misalignment, small workspace) are
  *     returned before anything is launched.  Errors only the device can see (an expert id
@@ -129,6 +130,26 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
                  const uint8_t* w2_codes, const float* w2_scales, void* out_bf16,
                  void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
                  void* stream);
+
+/* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
+ * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
+ * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;
+ * at most max_marks events are used, later kernels go untimed).  qarl_profile_end
+ * synchronizes the device, adds the elapsed milliseconds and the number of timed launches of
+ * each stage into stage_ms[QARL_NUM_STAGES] / stage_launches[QARL_NUM_STAGES] (host arrays)
+ * and destroys the events. */
+enum {
+  QARL_STAGE_QUANT_WEIGHT = 0,
+  QARL_STAGE_QUANT_ACT = 1,
+  QARL_STAGE_LINEAR_GEMM = 2,
+  QARL_STAGE_PERMUTE = 3,
+  QARL_STAGE_GATE_UP_GEMM = 4,
+  QARL_STAGE_DOWN_GEMM = 5,
+  QARL_STAGE_COMBINE = 6,
+  QARL_NUM_STAGES = 7
+};
+int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
+int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);
 
 /* Number of this library's kernels the context has launched since it was created. */
 int64_t qarl_launch_count(qarl_ctx* ctx);

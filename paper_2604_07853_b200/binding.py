@@ -29,7 +29,10 @@ EXPORTS = [
     "qarl_last_cuda_error", "qarl_quantize_weight", "qarl_quantize_act",
     "qarl_linear_workspace_bytes", "qarl_linear_fwd", "qarl_linear_fwd_q",
     "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
+    "qarl_profile_begin", "qarl_profile_end",
 ]
+STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
+          "combine"]
 
 
 class QarlError(RuntimeError):
@@ -86,6 +89,10 @@ def load() -> C.CDLL:
                                C.POINTER(MoeDebug), p]
     L.qarl_launch_count.restype = i64
     L.qarl_launch_count.argtypes = [p]
+    L.qarl_profile_begin.restype = C.c_int
+    L.qarl_profile_begin.argtypes = [p, C.c_int]
+    L.qarl_profile_end.restype = C.c_int
+    L.qarl_profile_end.argtypes = [p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     _lib = L
     return L
 
@@ -148,6 +155,18 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.qarl_launch_count(self.h))
+
+    def profile_begin(self, max_marks: int = 4096):
+        """Start per-stage CUDA-event timing of this context's kernels."""
+        self._check(self.lib.qarl_profile_begin(self.h, max_marks))
+
+    def profile_end(self) -> dict:
+        """Stop stage timing; returns {stage: (total_ms, launches)}."""
+        n = len(STAGES)
+        ms = (C.c_double * n)()
+        cnt = (C.c_int64 * n)()
+        self._check(self.lib.qarl_profile_end(self.h, ms, cnt))
+        return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     # ------------------------------------------------------------------ calls
     def quantize_weight(self, w: torch.Tensor, codes=None, scales=None):

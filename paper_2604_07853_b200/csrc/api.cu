@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -14,6 +15,10 @@ struct qarl_ctx {
   int64_t launches;
   qarl::EncodeTiledFn encode;
   char err[256];
+  // stage timing: marks[i] closes stage mark_stage[i] (-1: an opening mark)
+  std::vector<cudaEvent_t> marks;
+  std::vector<int> mark_stage;
+  size_t marks_used = 0;
 };
 
 namespace {
@@ -36,6 +41,13 @@ Launch make_launch(qarl_ctx* ctx, void* stream) {
   L.d_status = ctx->d_status;
   L.launches = &ctx->launches;
   return L;
+}
+
+// Record a timing mark on the stream if stage timing is on and events are left.
+void mark(qarl_ctx* ctx, cudaStream_t st, int stage) {
+  if (ctx->marks_used >= ctx->marks.size()) return;
+  if (cudaEventRecord(ctx->marks[ctx->marks_used], st) != cudaSuccess) return;
+  ctx->mark_stage[ctx->marks_used++] = stage;
 }
 
 int run_gemm(qarl_ctx* ctx, const Launch& L, const GemmArgs& a) {
@@ -150,6 +162,43 @@ int qarl_poll_device_status(qarl_ctx* ctx, void* stream) {
 const char* qarl_last_cuda_error(qarl_ctx* ctx) { return ctx ? ctx->err : ""; }
 int64_t qarl_launch_count(qarl_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int qarl_profile_begin(qarl_ctx* ctx, int max_marks) {
+  if (!ctx || max_marks < 2) return QARL_ERR_INVALID_ARG;
+  if (!ctx->marks.empty()) return QARL_ERR_INVALID_ARG;  // already on
+  ctx->marks.resize(static_cast<size_t>(max_marks));
+  ctx->mark_stage.assign(static_cast<size_t>(max_marks), -1);
+  ctx->marks_used = 0;
+  for (size_t i = 0; i < ctx->marks.size(); ++i) {
+    cudaError_t e = cudaEventCreate(&ctx->marks[i]);
+    if (e != cudaSuccess) {
+      for (size_t j = 0; j < i; ++j) cudaEventDestroy(ctx->marks[j]);
+      ctx->marks.clear();
+      return cuda_fail(ctx, e, "cudaEventCreate");
+    }
+  }
+  return QARL_OK;
+}
+
+int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches) {
+  if (!ctx || !stage_ms || !stage_launches) return QARL_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  int rc = e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "profile_end");
+  for (size_t i = 1; rc == QARL_OK && i < ctx->marks_used; ++i) {
+    const int st = ctx->mark_stage[i];
+    if (st < 0 || st >= QARL_NUM_STAGES) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->marks[i - 1], ctx->marks[i]) == cudaSuccess) {
+      stage_ms[st] += ms;
+      stage_launches[st] += 1;
+    }
+  }
+  for (cudaEvent_t ev : ctx->marks) cudaEventDestroy(ev);
+  ctx->marks.clear();
+  ctx->mark_stage.clear();
+  ctx->marks_used = 0;
+  return rc;
+}
+
 int qarl_quantize_weight(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* codes,
                          float* scales, void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
@@ -158,8 +207,10 @@ int qarl_quantize_weight(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
   if (!w || !codes || !scales) return QARL_ERR_INVALID_ARG;
   if (!aligned16(w) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return QARL_ERR_MISALIGNED;
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
   cudaError_t e = launch_quantize_weight(make_launch(ctx, stream), static_cast<const uint16_t*>(w), E, N, K, codes,
                                          scales);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_WEIGHT);
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_weight");
 }
 
@@ -172,8 +223,10 @@ int qarl_quantize_act(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, int64_
   if (!x || !codes || !scales) return QARL_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(codes) || (ldx % 8) || (reinterpret_cast<uintptr_t>(scales) & 3u))
     return QARL_ERR_MISALIGNED;
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
   cudaError_t e = launch_quantize_act(make_launch(ctx, stream), static_cast<const uint16_t*>(x), M, K, ldx, codes,
                                       scales, nullptr, 1);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_ACT);
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_act");
 }
 
@@ -189,7 +242,8 @@ int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* xc, const float* xs, int64_t
   if (N % kBlock || K % kBlock || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
   if (!xc || !xs || !wc || !ws || !y) return QARL_ERR_INVALID_ARG;
-  if (!aligned16(xc) || !aligned16(wc) || !aligned16(y) || !aligned16(xs) || !aligned16(y_f32))
+  if (!aligned16(xc) || !aligned16(wc) || !aligned16(y) || !aligned16(y_f32) ||
+      (reinterpret_cast<uintptr_t>(xs) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 3u))
     return QARL_ERR_MISALIGNED;
   GemmArgs a{};
   a.mode = kModeLinear;
@@ -203,7 +257,10 @@ int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* xc, const float* xs, int64_t
   a.E = 1;
   a.out_bf16 = static_cast<uint16_t*>(y);
   a.out_f32 = y_f32;
-  return run_gemm(ctx, make_launch(ctx, stream), a);
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
+  const int rc = run_gemm(ctx, make_launch(ctx, stream), a);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_LINEAR_GEMM);
+  return rc;
 }
 
 int qarl_linear_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wc, const float* ws,
@@ -216,8 +273,10 @@ int qarl_linear_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const ui
   if (workspace_bytes < qarl_linear_workspace_bytes(M, N, K)) return QARL_ERR_WORKSPACE_TOO_SMALL;
   uint8_t* xc = static_cast<uint8_t*>(workspace);
   float* xs = reinterpret_cast<float*>(xc + align_up(static_cast<size_t>(M) * K, 256));
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
   cudaError_t e = launch_quantize_act(make_launch(ctx, stream), static_cast<const uint16_t*>(x), M, K, K, xc, xs,
                                       nullptr, 1);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_ACT);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "quantize_act");
   return qarl_linear_fwd_q(ctx, xc, xs, M, K, wc, ws, N, y, y_f32, stream);
 }
@@ -256,13 +315,16 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   if ((e = cudaMemsetAsync(pb.sorted_pair, 0, P * sizeof(int32_t), L.stream)) != cudaSuccess ||
       (e = cudaMemsetAsync(pb.pos_of_pair, 0, P * sizeof(int32_t), L.stream)) != cudaSuccess)
     return cuda_fail(ctx, e, "memset");
+  mark(ctx, L.stream, -1);
   if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
+  mark(ctx, L.stream, QARL_STAGE_PERMUTE);
 
   uint8_t* a_codes = ws + pl.a_codes;
   float* a_scales = reinterpret_cast<float*>(ws + pl.a_scales);
   if ((e = launch_quantize_act(L, static_cast<const uint16_t*>(x), M, H, H, a_codes, a_scales, pb.pos_of_pair,
                                static_cast<int>(k))) != cudaSuccess)
     return cuda_fail(ctx, e, "quantize_act");
+  mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
 
   uint8_t* h_codes = ws + pl.h_codes;
   float* h_scales = reinterpret_cast<float*>(ws + pl.h_scales);
@@ -283,6 +345,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   g.h_bf16 = dbg ? static_cast<uint16_t*>(dbg->h_bf16) : nullptr;
   int rc = run_gemm(ctx, L, g);
   if (rc != QARL_OK) return rc;
+  mark(ctx, L.stream, QARL_STAGE_GATE_UP_GEMM);
 
   uint16_t* contrib = reinterpret_cast<uint16_t*>(ws + pl.contrib);
   GemmArgs d{};
@@ -302,9 +365,11 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   d.pair_weights = wts;
   rc = run_gemm(ctx, L, d);
   if (rc != QARL_OK) return rc;
+  mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);
 
   if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out))) != cudaSuccess)
     return cuda_fail(ctx, e, "combine");
+  mark(ctx, L.stream, QARL_STAGE_COMBINE);
 
   if (dbg) {
     if (dbg->expert_offsets &&
