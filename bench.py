@@ -84,7 +84,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "20"], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
 
@@ -176,7 +176,7 @@ def run_reference(args, rank: int):
 
 
 def config_dict(n_gpus: int) -> dict:
-    return {"workload": "moe_ffn_train_fwd_M32768_zipf1.1 (+ on-the-fly weight quantization)",
+    return {"workload": f"moe_ffn_train_fwd_M{M_TRAIN}_zipf1.1 (+ on-the-fly weight quantization)",
             "tokens_per_gpu": M_TRAIN, "hidden": H, "intermediate": I, "experts": E, "top_k": TOPK,
             "format": "fp8 e4m3, 128x128 weight blocks, 1x128 activation groups, fp32 scales",
             "l2": "inputs larger than L2 (1.2 GB bf16 masters + 0.6 GB codes + 0.13 GB activations per step)",
@@ -185,16 +185,22 @@ def config_dict(n_gpus: int) -> dict:
 
 # --------------------------------------------------------------------------- GPU arm
 def main():
+    global M_TRAIN
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tokens", type=int, default=M_TRAIN,
+                    help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
+                         "only; the reported config names the size)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    M_TRAIN = args.tokens
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -278,8 +284,8 @@ def main():
         step(dx, dids, dwts)
         hout.copy_(out, non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
+    e2e_steps = 0 if args.no_e2e else max(3, min(args.steps, 10))
+    for _ in range(2 if e2e_steps else 0):
         e2e_step()
     barrier()
     ev0.record()
@@ -287,7 +293,7 @@ def main():
         e2e_step()
     ev1.record()
     barrier()
-    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / max(e2e_steps, 1) if e2e_steps else float("nan")
     e2e = {"value": world * M_TRAIN / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": hx.numel() * 2 + hids.numel() * 4 + hwts.numel() * 4,
            "d2h_bytes_per_step": hout.numel() * 2,
@@ -364,7 +370,7 @@ def main():
     # ---------------- CPU oracle baseline (rank 0, N = 1 only), bounded sample
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        n_tokens, n_exp = 128, 2
+        n_tokens, n_exp = min(8192, M_TRAIN), 32
         st = cpu_state(4, n_tokens)
         est, raw = cpu_reference_step(st, n_tokens, n_exp)
         result["cpu_baseline"] = {
