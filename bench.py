@@ -249,13 +249,13 @@ def main():
         ctx.quantize_weight(w2, w2c, w2s)
         ctx.moe_fwd(xd, idd, wtd, w13c, w13s, w2c, w2s, out=out, workspace=ws)
 
+    sampler = ClockSampler()
+    if rank == 0:
+        sampler.start()          # nvidia-smi needs a moment to start: begin before the warm-up
     for _ in range(args.warmup):
         step()
     ctx.check_device_status()
-    sampler = ClockSampler()
     barrier()
-    if rank == 0:
-        sampler.start()
     launches0 = ctx.launch_count()
     ctx.profile_begin(max_marks=args.steps * 16 + 8)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

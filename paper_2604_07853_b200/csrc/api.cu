@@ -63,7 +63,7 @@ int run_gemm(qarl_ctx* ctx, const Launch& L, const GemmArgs& a) {
 
 // Workspace carve-up of qarl_moe_fwd; every slice starts on a 256-byte boundary.
 struct MoePlan {
-  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, a_codes, a_scales, h_codes, h_scales, contrib, total;
+  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, a_codes, a_scales, h_codes, h_scales, contrib, total;
 };
 MoePlan plan_moe(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   const size_t P = static_cast<size_t>(M * k);
@@ -78,6 +78,7 @@ MoePlan plan_moe(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   p.offsets = take((E + 1) * sizeof(int32_t));
   p.sorted_pair = take(P * sizeof(int32_t));
   p.pos_of_pair = take(P * sizeof(int32_t));
+  p.sorted_w = take(P * sizeof(float));
   p.a_codes = take(P * H);
   p.a_scales = take(P * (H / kBlock) * sizeof(float));
   p.h_codes = take(P * I);
@@ -321,8 +322,10 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
 
   uint8_t* a_codes = ws + pl.a_codes;
   float* a_scales = reinterpret_cast<float*>(ws + pl.a_scales);
+  float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
+  if ((e = cudaMemsetAsync(sorted_w, 0, P * sizeof(float), L.stream)) != cudaSuccess) return cuda_fail(ctx, e, "memset");
   if ((e = launch_quantize_act(L, static_cast<const uint16_t*>(x), M, H, H, a_codes, a_scales, pb.pos_of_pair,
-                               static_cast<int>(k))) != cudaSuccess)
+                               static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
     return cuda_fail(ctx, e, "quantize_act");
   mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
 
@@ -362,7 +365,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   d.out_bf16 = contrib;
   d.out_f32 = dbg ? dbg->down_f32 : nullptr;
   d.sorted_pair = pb.sorted_pair;
-  d.pair_weights = wts;
+  d.pair_weights = sorted_w;
   rc = run_gemm(ctx, L, d);
   if (rc != QARL_OK) return rc;
   mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);

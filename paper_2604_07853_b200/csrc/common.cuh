@@ -57,8 +57,11 @@ cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E
                                    uint8_t* codes, float* scales);
 // dst_rows == nullptr: row m of the output is m.  Otherwise each input row t is written to
 // the `fanout` output rows dst_rows[t*fanout + j] (quantize once, scatter k times).
+// With dst_rows, pair_w [M*fanout] (the top-k weights by flat pair id) is scattered alongside
+// into sorted_w[dst] so that later kernels read a pair's weight by its sorted position.
 cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
-                                uint8_t* codes, float* scales, const int32_t* dst_rows, int fanout);
+                                uint8_t* codes, float* scales, const int32_t* dst_rows, int fanout,
+                                const float* pair_w = nullptr, float* sorted_w = nullptr);
 
 struct PermuteBuffers {
   int32_t* chunk_hist;   // [nchunks, E]
@@ -97,7 +100,7 @@ struct GemmArgs {
   float* h_scales;           // gate_up: [P, I/128]
   uint16_t* h_bf16;          // gate_up (debug): [P, I]
   const int32_t* sorted_pair;   // down: [P]
-  const float* pair_weights;    // down: [M*k] by flat pair id
+  const float* pair_weights;    // down: [M*k] by sorted position
 };
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

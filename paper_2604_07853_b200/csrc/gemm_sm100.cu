@@ -8,19 +8,25 @@
 // cta_group::1), four MMAs per K-block in ascending k, no split-K, no atomics.  A row's
 // result depends only on that row's codes and scales and on the weight tile.
 //
-// Structure of a CTA (576 threads, one CTA per SM, persistent over a static tile list):
-//   warp 16   TMA producer: per K-block one stage = A box 128x128 B + two B boxes 128x128 B
-//             (SWIZZLE_128B) into a 4-deep shared-memory ring;
-//   warp 17   MMA issuer: 4 x tcgen05.mma kind::f8f6f4 per K-block into one of two 256-column
-//             TMEM accumulators (overwrite on the first), then tcgen05.commit to free the
-//             smem stage and to publish the accumulator;
-//   warps 0-15 promotion + epilogue: warp w reads TMEM lanes 32*(w%4).. (its hardware
-//             quadrant) and two 32-column slices, one in each 128-column half of the tile,
-//             multiplies the block partial by the combined scale and adds it to fp32
-//             registers; MMA of block kb+1 overlaps promotion of block kb.
-// The two 128-column halves of a tile are rows [n_lo, n_lo+128) and [n_hi, n_hi+128) of the
-// weight: adjacent for linear/down, gate rows and the matching up rows for gate_up so that
-// SwiGLU and the 1x128 re-quantization of h happen in registers.
+// A tile is 128 rows x (128 + 128) columns: two half tiles, rows [n_lo, n_lo+128) and
+// [n_hi, n_hi+128) of the weight -- adjacent for linear/down, gate rows and the matching up
+// rows for gate_up so that SwiGLU and the 1x128 re-quantization of h need no second pass.
+//
+// Structure of a CTA (512 threads = 4 warpgroups, one CTA per SM, persistent, static tile list):
+//   warp 12     TMA producer: per K-block one stage = A box 128x128 B + two B boxes 128x128 B
+//               (SWIZZLE_128B) into a 3-deep shared-memory ring;
+//   warp 13     MMA issuer: 4 x tcgen05.mma kind::f8f6f4 per K-block into one of two
+//               256-column TMEM accumulators (overwrite on the first), then tcgen05.commit to
+//               free the smem stage and to publish the accumulator;
+//   warps 0-7   promotion (208 registers each via setmaxnreg): warp w reads TMEM lanes
+//               32*(w%4).. (its hardware quadrant) and the 64-column slice (w/4) of each half,
+//               in 16-column double-buffered chunks, releases the accumulator, and adds
+//               scale * partial into fp32 registers; MMA of block kb+1 overlaps promotion of kb.  At the
+//               end of a tile it rounds its 128 values to bf16 into a shared-memory staging
+//               tile and goes straight on to the next tile;
+//   warps 8-11  epilogue: read the staged bf16 tile (coalesced, several rows per pass) and
+//               finish it while the next tile's main loop runs: plain store (linear),
+//               scatter by pair id (down), or SwiGLU + 1x128 amax/scale/e4m3 codes (gate_up).
 //
 // Every wait on an mbarrier is bounded; on expiry the thread records
 // QARL_ERR_DEVICE_TIMEOUT, raises a CTA-wide abort flag that all other waits poll, and the
@@ -39,16 +45,24 @@ constexpr int BM = 128;           // rows per tile (UMMA M)
 constexpr int BNH = 128;          // columns per half tile
 constexpr int BN = 2 * BNH;       // UMMA N
 constexpr int BK = 128;           // one K-block = one 128-byte swizzle span of e4m3
-constexpr int kStages = 4;
-constexpr int kAccStages = 2;
-constexpr int kEpiWarps = 16;
-constexpr int kTmaWarp = 16;
-constexpr int kMmaWarp = 17;
-constexpr int kThreads = 18 * 32;
+constexpr int kStages = 3;
+constexpr int kAccBufs = 2;       // TMEM accumulators of 256 columns
+constexpr int kPromoWarps = 8;    // warps 0-7
+constexpr int kEpiWarps = 4;      // warps 8-11
+constexpr int kTmaWarp = 12;
+constexpr int kMmaWarp = 13;      // warps 14, 15 idle (setmaxnreg works on whole warpgroups)
+constexpr int kThreads = 16 * 32;
+// register re-allocation: 256 x 208 + 128 x 56 + 128 x 40 = 65536 = 512 x 128 (the launch allocation)
+constexpr int kPromoRegs = 208;
+constexpr int kEpiRegs = 56;
+constexpr int kAuxRegs = 40;
+constexpr int kSliceCols = 64;    // columns of each half owned by one promotion warp
 constexpr uint32_t kABytes = BM * BK;
 constexpr uint32_t kBBytes = BN * BK;
 constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 48 KB
 constexpr uint32_t kTmemCols = 512;
+constexpr int kOutPitch = BN * 2 + 16;  // bytes per row of the bf16 staging tile (padded: conflict-free)
+constexpr uint32_t kOutBytes = BM * kOutPitch;
 constexpr int kMaxExperts = 1024;
 
 struct GemmParams {
@@ -67,25 +81,27 @@ struct GemmParams {
   float* h_scales;
   uint16_t* h_bf16;
   const int32_t* sorted_pair;
-  const float* pair_weights;
+  const float* pair_weights;  // down: combine weight of each sorted position
   int* status;
   unsigned long long wait_limit_ns;
+  unsigned long long* trace;  // QARL_TRACE builds only: per-CTA wait-cycle counters [grid][8]
 };
 
 struct __align__(8) SmemTail {
   uint64_t full[kStages];
   uint64_t empty[kStages];
-  uint64_t tmem_full[kAccStages];
-  uint64_t tmem_empty[kAccStages];
-  uint64_t amax_bar[2];
+  uint64_t tmem_full[kAccBufs];
+  uint64_t tmem_empty[kAccBufs];
+  uint64_t out_full;
+  uint64_t out_empty;
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
   int32_t prefix[kMaxExperts + 1];
-  float amax[2][4][BM];
 };
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + sizeof(SmemTail);
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutBytes + sizeof(SmemTail);
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TileCoord {
   int e, n_tile, m0, m_end;
@@ -122,7 +138,35 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sm
   }
 }
 
-__device__ __forceinline__ float silu_mul(float g, float u) { return (g / (1.0f + __expf(-g))) * u; }
+// Wait-time tracing (development aid, compiled out unless QARL_TRACE is defined): cycles each
+// role spends blocked on each barrier, summed per CTA.
+#ifdef QARL_TRACE
+#define TRACE_T0() const long long _t0 = clock64()
+#define TRACE_ADD(slot) trace_acc[slot] += clock64() - _t0
+#else
+#define TRACE_T0()
+#define TRACE_ADD(slot)
+#endif
+
+// silu(g) * u in fp32 with the fast exp and reciprocal (relative error ~1e-6, far below the
+// half-ulp of the bf16 the result is rounded to).
+__device__ __forceinline__ float silu_mul(float g, float u) {
+  return __fdividef(g, 1.0f + __expf(-g)) * u;
+}
+
+// acc[j] = fmaf(sc, v[j], acc[j]) for 16 values (8 float2 accumulators).
+__device__ __forceinline__ void promote16(float2* acc, const uint32_t (&v)[16], float sc) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    acc[j].x = __fmaf_rn(sc, __uint_as_float(v[2 * j]), acc[j].x);
+    acc[j].y = __fmaf_rn(sc, __uint_as_float(v[2 * j + 1]), acc[j].y);
+  }
+}
+
+__device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
+  const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);  // .x = lo (low 16 bits), .y = hi
+  return *reinterpret_cast<const uint32_t*>(&b);
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -130,8 +174,13 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
                         const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  SmemTail* s = reinterpret_cast<SmemTail*>(smem + static_cast<size_t>(kStages) * kStageBytes);
+  uint8_t* out_tile = smem + static_cast<size_t>(kStages) * kStageBytes;
+  SmemTail* s = reinterpret_cast<SmemTail*>(out_tile + kOutBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef QARL_TRACE
+  long long trace_acc[12] = {0};
+  const long long trace_start = clock64();
+#endif
 
   // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
   if (threadIdx.x == 0) {
@@ -139,12 +188,12 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       mbar_init(&s->full[i], 1);
       mbar_init(&s->empty[i], 1);
     }
-    for (int i = 0; i < kAccStages; ++i) {
+    for (int i = 0; i < kAccBufs; ++i) {
       mbar_init(&s->tmem_full[i], 1);
-      mbar_init(&s->tmem_empty[i], kEpiWarps);
+      mbar_init(&s->tmem_empty[i], kPromoWarps);
     }
-    mbar_init(&s->amax_bar[0], kEpiWarps);
-    mbar_init(&s->amax_bar[1], kEpiWarps);
+    mbar_init(&s->out_full, kPromoWarps);
+    mbar_init(&s->out_empty, kEpiWarps);
     s->abort_flag = 0;
     fence_mbar_init();
   }
@@ -184,84 +233,200 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   const int KB = p.kblocks;
   const int NB = p.N / BNH;  // weight scale block-rows per expert
 
-  if (warp == kTmaWarp) {
-    // =============================== TMA producer =====================================
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      uint32_t armed = 0, armed_parity = 0;  // per-stage: has a load in flight / its parity
-      int cur_e = 0;
-      bool ok = true;
-      for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
-        const TileCoord c = decode_tile(s, T, cur_e);
-        int row_lo, row_hi;
-        if (MODE == kModeGateUp) {
-          row_lo = c.e * p.N + c.n_tile * BNH;
-          row_hi = row_lo + p.I;
-        } else {
-          row_lo = c.e * p.N + c.n_tile * BN;
-          row_hi = row_lo + BNH;
+  if (warp >= kPromoWarps + kEpiWarps) setmaxnreg_dec<kAuxRegs>();
+  else if (warp >= kPromoWarps) setmaxnreg_dec<kEpiRegs>();
+  else setmaxnreg_inc<kPromoRegs>();
+  if (warp >= kPromoWarps + kEpiWarps) {
+    if (warp == kTmaWarp) {
+      // =============================== TMA producer =====================================
+      if (lane == 0) {
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t armed = 0, armed_parity = 0;  // per-stage: has a load in flight / its parity
+        int cur_e = 0;
+        bool ok = true;
+        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
+          const TileCoord c = decode_tile(s, T, cur_e);
+          int row_lo, row_hi;
+          if (MODE == kModeGateUp) {
+            row_lo = c.e * p.N + c.n_tile * BNH;
+            row_hi = row_lo + p.I;
+          } else {
+            row_lo = c.e * p.N + c.n_tile * BN;
+            row_hi = row_lo + BNH;
+          }
+          for (int kb = 0; kb < KB; ++kb) {
+            {
+              TRACE_T0();
+              if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
+              TRACE_ADD(0);
+            }
+            uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
+            uint8_t* b_dst = a_dst + kABytes;
+            mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
+            tma_load_2d(a_dst, &tm_a, &s->full[stage], kb * BK, c.m0);
+            tma_load_2d(b_dst, &tm_b, &s->full[stage], kb * BK, row_lo);
+            tma_load_2d(b_dst + kBBytes / 2, &tm_b, &s->full[stage], kb * BK, row_hi);
+            armed |= 1u << stage;
+            armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+          }
         }
-        for (int kb = 0; kb < KB; ++kb) {
-          if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
-          uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
-          uint8_t* b_dst = a_dst + kABytes;
-          mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
-          tma_load_2d(a_dst, &tm_a, &s->full[stage], kb * BK, c.m0);
-          tma_load_2d(b_dst, &tm_b, &s->full[stage], kb * BK, row_lo);
-          tma_load_2d(b_dst + kBBytes / 2, &tm_b, &s->full[stage], kb * BK, row_hi);
-          armed |= 1u << stage;
-          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        if (!ok) {  // let copies in flight land before the CTA's shared memory is released
+          for (int i = 0; i < kStages; ++i)
+            if (armed & (1u << i)) mbar_wait_bounded(&s->full[i], (armed_parity >> i) & 1u, 20000000ull);
         }
       }
-      if (!ok) {  // let copies in flight land before the CTA's shared memory is released
-        for (int i = 0; i < kStages; ++i)
-          if (armed & (1u << i)) mbar_wait_bounded(&s->full[i], (armed_parity >> i) & 1u, 20000000ull);
+    } else if (warp == kMmaWarp) {
+      // =============================== MMA issuer =======================================
+      if (lane == 0) {
+        constexpr uint32_t idesc = umma_idesc_e4m3_f32(BM, BN);
+        int stage = 0, ks = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
+          for (int kb = 0; kb < KB; ++kb) {
+            {
+              TRACE_T0();
+              if (!wait_or_abort(&s->tmem_empty[ks], acc_phase ^ 1, s, p)) { ok = false; break; }
+              TRACE_ADD(2);
+            }
+            {
+              TRACE_T0();
+              if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
+              TRACE_ADD(1);
+            }
+            tc_fence_after_sync();
+            const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
+            const uint64_t a_desc = umma_desc_k_sw128(a_addr);
+            const uint64_t b_desc = umma_desc_k_sw128(a_addr + kABytes);
+            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ks) * BN;
+#pragma unroll
+            for (int k4 = 0; k4 < BK / 32; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
+              umma_f8(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
+            umma_commit(&s->empty[stage]);
+            umma_commit(&s->tmem_full[ks]);
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+            if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
+          }
+        }
       }
     }
-  } else if (warp == kMmaWarp) {
-    // =============================== MMA issuer =======================================
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_e4m3_f32(BM, BN);
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
-        for (int kb = 0; kb < KB; ++kb) {
-          if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) { ok = false; break; }
-          if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
-          tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
-          const uint64_t a_desc = umma_desc_k_sw128(a_addr);
-          const uint64_t b_desc = umma_desc_k_sw128(a_addr + kABytes);
-          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+  } else if (warp >= kPromoWarps) {
+    // =============================== epilogue warps ===================================
+    const int ew = warp - kPromoWarps;
+    int cur_e = 0;
+    uint32_t tile_iter = 0;
+    for (int T = blockIdx.x; T < total_tiles; T += gridDim.x, ++tile_iter) {
+      const TileCoord c = decode_tile(s, T, cur_e);
+      int my_pair = 0;  // down: destination (flat pair id) of the lane-th row this warp handles
+      if (MODE == kModeDown) {
+        const int row = c.m0 + ew + kEpiWarps * lane;
+        if (row < c.m_end) my_pair = __ldg(p.sorted_pair + row);
+      }
+      {
+        TRACE_T0();
+        if (!wait_or_abort(&s->out_full, tile_iter & 1u, s, p)) break;
+        TRACE_ADD(6);
+      }
+      if (MODE == kModeGateUp) {
+        // 8 lanes per row, 4 rows per pass.  Lane `sub` owns h columns [8 sub, 8 sub + 8) and
+        // [64 + 8 sub, 64 + 8 sub + 8) of the row's 128-wide quantization group, so that a
+        // quarter-warp reads 128 contiguous bytes of the staging tile (conflict-free).
+        const int sub = lane & 7, rsel = lane >> 3;
+        const int IB = p.I / BNH;
+#pragma unroll 2
+        for (int i = 0; i < BM / (kEpiWarps * 4); ++i) {
+          const int r0 = (i * kEpiWarps + ew) * 4;
+          if (c.m0 + r0 >= c.m_end) break;  // warp-uniform: rows ascend with i
+          const int rr = r0 + rsel;
+          const int row = c.m0 + rr;
+          const bool live = row < c.m_end;
+          const uint8_t* src = out_tile + rr * kOutPitch + sub * 16;
+          uint4 g[2], u[2];
+          g[0] = *reinterpret_cast<const uint4*>(src);
+          g[1] = *reinterpret_cast<const uint4*>(src + 128);
+          u[0] = *reinterpret_cast<const uint4*>(src + BNH * 2);
+          u[1] = *reinterpret_cast<const uint4*>(src + BNH * 2 + 128);
+          uint32_t hb[8];
+          uint32_t m = 0;
 #pragma unroll
-          for (int k4 = 0; k4 < BK / 32; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
-            umma_f8(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
-          umma_commit(&s->empty[stage]);
-          umma_commit(&s->tmem_full[acc]);
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
-          if (++acc == kAccStages) { acc = 0; acc_phase ^= 1; }
+          for (int t = 0; t < 2; ++t) {
+            const uint32_t gw[4] = {g[t].x, g[t].y, g[t].z, g[t].w};
+            const uint32_t uw[4] = {u[t].x, u[t].y, u[t].z, u[t].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float h0 = silu_mul(bf16_bits_to_f32(gw[j] & 0xFFFFu), bf16_bits_to_f32(uw[j] & 0xFFFFu));
+              const float h1 = silu_mul(__uint_as_float(gw[j] & 0xFFFF0000u), __uint_as_float(uw[j] & 0xFFFF0000u));
+              hb[4 * t + j] = bf16x2_bits(h0, h1);
+              m = __vmaxu2(m, hb[4 * t + j] & 0x7FFF7FFFu);  // |bf16| bit patterns: exact, order-free max
+            }
+          }
+          m = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+          for (int o = 4; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+          float inv;
+          const float sc = block_scale(bf16_bits_to_f32(m), &inv);
+          uint32_t cw[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t x0 = hb[2 * j], x1 = hb[2 * j + 1];
+            cw[j] = cvt_e4m3x4(__fmul_rn(bf16_bits_to_f32(x0 & 0xFFFFu), inv), __fmul_rn(__uint_as_float(x0 & 0xFFFF0000u), inv),
+                               __fmul_rn(bf16_bits_to_f32(x1 & 0xFFFFu), inv), __fmul_rn(__uint_as_float(x1 & 0xFFFF0000u), inv));
+          }
+          if (live) {
+            const int col = c.n_tile * BNH + 8 * sub;
+            uint8_t* hc = p.h_codes + static_cast<int64_t>(row) * p.I + col;
+            *reinterpret_cast<uint2*>(hc) = make_uint2(cw[0], cw[1]);
+            *reinterpret_cast<uint2*>(hc + 64) = make_uint2(cw[2], cw[3]);
+            if (sub == 0) p.h_scales[static_cast<int64_t>(row) * IB + c.n_tile] = sc;
+            if (p.h_bf16) {
+              uint16_t* hd = p.h_bf16 + static_cast<int64_t>(row) * p.I + col;
+              *reinterpret_cast<uint4*>(hd) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
+              *reinterpret_cast<uint4*>(hd + 64) = make_uint4(hb[4], hb[5], hb[6], hb[7]);
+            }
+            if (p.out_bf16) {  // debug dump of the bf16 gate_up row
+              uint16_t* gd = p.out_bf16 + static_cast<int64_t>(row) * p.N + col;
+              *reinterpret_cast<uint4*>(gd) = g[0];
+              *reinterpret_cast<uint4*>(gd + 64) = g[1];
+              *reinterpret_cast<uint4*>(gd + p.I) = u[0];
+              *reinterpret_cast<uint4*>(gd + p.I + 64) = u[1];
+            }
+          }
+        }
+      } else {
+        // the tile's 256 columns are contiguous in the output row: 512 bytes per row, 16 per lane
+        const int col = c.n_tile * BN + 8 * lane;
+        const bool col_ok = col < p.N;
+#pragma unroll 4
+        for (int i = 0; i < BM / kEpiWarps; ++i) {
+          const int rr = ew + kEpiWarps * i;
+          const int row = c.m0 + rr;
+          if (row >= c.m_end) break;
+          const uint4 v = *reinterpret_cast<const uint4*>(out_tile + rr * kOutPitch + lane * 16);
+          int64_t out_row = row;
+          if (MODE == kModeDown) out_row = __shfl_sync(0xFFFFFFFFu, my_pair, i);  // lane i holds row i's pair id
+          if (col_ok) *reinterpret_cast<uint4*>(p.out_bf16 + out_row * p.N + col) = v;
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s->out_empty);
     }
   } else {
-    // =============================== promotion + epilogue =============================
+    // =============================== promotion warps ==================================
     const int q = warp & 3;          // TMEM lane quadrant this warp may read
-    const int cg = warp >> 2;        // 32-column slice within each half tile
+    const int hs = warp >> 2;        // which 64-column slice of each half tile
     const int r = q * 32 + lane;     // row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-    int acc = 0;
+    int ks = 0;
     uint32_t acc_phase = 0;
     int cur_e = 0;
-    uint32_t tile_iter = 0;      // tiles this CTA has finished (selects the amax exchange buffer)
-    bool ok = true;
-    for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
-      const TileCoord c = decode_tile(s, T, cur_e);
-      const int row = c.m0 + r;
-      const bool valid = row < c.m_end;
-      const int row_c = min(row, p.rows_total - 1);
+    uint32_t tile_iter = 0;
+
+    // scale pointers of a tile for this thread's row: s_x[row, :], s_w[lo block-row, :] and
+    // the offset from the lo to the hi block-row
+    auto scale_ptrs = [&](const TileCoord& c, const float*& sx, const float*& swl, int& hi_off) {
+      const int row_c = min(c.m0 + r, p.rows_total - 1);
       int nb_lo, nb_hi;
       if (MODE == kModeGateUp) {
         nb_lo = c.n_tile;
@@ -270,158 +435,147 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         nb_lo = 2 * c.n_tile;
         nb_hi = min(2 * c.n_tile + 1, NB - 1);
       }
-      const float* sx_ptr = p.a_scales + static_cast<int64_t>(row_c) * KB;
-      const float* sw_lo_ptr = p.b_scales + (static_cast<int64_t>(c.e) * NB + nb_lo) * KB;
-      const float* sw_hi_ptr = p.b_scales + (static_cast<int64_t>(c.e) * NB + nb_hi) * KB;
+      sx = p.a_scales + static_cast<int64_t>(row_c) * KB;
+      swl = p.b_scales + (static_cast<int64_t>(c.e) * NB + nb_lo) * KB;
+      hi_off = (nb_hi - nb_lo) * KB;
+    };
 
-      float acc_lo[32], acc_hi[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) acc_lo[j] = acc_hi[j] = 0.0f;
+    int T = blockIdx.x;
+    if (T < total_tiles) {
+      TileCoord c = decode_tile(s, T, cur_e);
+      const float *sx_ptr, *sw_lo_ptr;
+      int sw_hi_off;
+      scale_ptrs(c, sx_ptr, sw_lo_ptr, sw_hi_off);
+      float sx_next = __ldg(sx_ptr), swl_next = __ldg(sw_lo_ptr), swh_next = __ldg(sw_lo_ptr + sw_hi_off);
+      bool ok = true;
+      for (;;) {
+        const int row = c.m0 + r;
+        const bool valid = row < c.m_end;
+        const int Tn = T + gridDim.x;
+        const bool has_next = Tn < total_tiles;
+        TileCoord cn = c;
+        float w = 0.0f;  // down: the pair's combine weight (sorted order), used at the end of the tile
+        if (MODE == kModeDown && valid) w = __ldg(p.pair_weights + row);
 
-      float sx_next = __ldg(sx_ptr), swl_next = __ldg(sw_lo_ptr), swh_next = __ldg(sw_hi_ptr);
-      for (int kb = 0; kb < KB; ++kb) {
-        const float sc_lo = __fmul_rn(sx_next, swl_next);
-        const float sc_hi = __fmul_rn(sx_next, swh_next);
-        if (kb + 1 < KB) {
-          sx_next = __ldg(sx_ptr + kb + 1);
-          swl_next = __ldg(sw_lo_ptr + kb + 1);
-          swh_next = __ldg(sw_hi_ptr + kb + 1);
-        }
-        if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) { ok = false; break; }
-        tc_fence_after_sync();
-        const uint32_t t_lo = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN + cg * 32);
-        const uint32_t t_hi = t_lo + BNH;
-        uint32_t v0[16], v1[16];
-        tmem_ld_x16(t_lo, v0);
-        tmem_ld_wait();
-        tmem_ld_x16(t_lo + 16, v1);
+        float2 acc_lo[32], acc_hi[32];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc_lo[j] = __fmaf_rn(sc_lo, __uint_as_float(v0[j]), acc_lo[j]);
-        tmem_ld_wait();
-        tmem_ld_x16(t_hi, v0);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc_lo[16 + j] = __fmaf_rn(sc_lo, __uint_as_float(v1[j]), acc_lo[16 + j]);
-        tmem_ld_wait();
-        tmem_ld_x16(t_hi + 16, v1);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc_hi[j] = __fmaf_rn(sc_hi, __uint_as_float(v0[j]), acc_hi[j]);
-        tmem_ld_wait();
-        // all of this warp's reads of the accumulator are done: hand it back to the MMA warp
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc_hi[16 + j] = __fmaf_rn(sc_hi, __uint_as_float(v1[j]), acc_hi[16 + j]);
-        if (++acc == kAccStages) { acc = 0; acc_phase ^= 1; }
-      }
-      if (!ok) break;
+        for (int j = 0; j < 32; ++j) acc_lo[j] = acc_hi[j] = make_float2(0.0f, 0.0f);
 
-      // ---- tile epilogue ------------------------------------------------------------------
-      if (MODE == kModeLinear || MODE == kModeDown) {
-        const int col_lo = c.n_tile * BN + cg * 32;
-        const int col_hi = col_lo + BNH;
-        const bool hi_valid = col_hi < p.N;
-        if (valid) {
-          int64_t out_row = row;
-          float w = 1.0f;
-          if (MODE == kModeDown) {
-            const int pair = __ldg(p.sorted_pair + row);
-            out_row = pair;
-            w = __ldg(p.pair_weights + pair);
+        for (int kb = 0; kb < KB; ++kb) {
+          const float sc_lo = __fmul_rn(sx_next, swl_next);
+          const float sc_hi = __fmul_rn(sx_next, swh_next);
+          if (kb + 1 < KB) {
+            sx_next = __ldg(sx_ptr + kb + 1);
+            swl_next = __ldg(sw_lo_ptr + kb + 1);
+            swh_next = __ldg(sw_lo_ptr + sw_hi_off + kb + 1);
+          } else if (has_next) {  // first scales of the next tile: their latency hides behind this block
+            cn = decode_tile(s, Tn, cur_e);
+            scale_ptrs(cn, sx_ptr, sw_lo_ptr, sw_hi_off);
+            sx_next = __ldg(sx_ptr);
+            swl_next = __ldg(sw_lo_ptr);
+            swh_next = __ldg(sw_lo_ptr + sw_hi_off);
           }
-          if (p.out_f32) {
-            float4* d_lo = reinterpret_cast<float4*>(p.out_f32 + static_cast<int64_t>(row) * p.N + col_lo);
-            float4* d_hi = reinterpret_cast<float4*>(p.out_f32 + static_cast<int64_t>(row) * p.N + col_hi);
+          {
+            TRACE_T0();
+            if (!wait_or_abort(&s->tmem_full[ks], acc_phase, s, p)) { ok = false; break; }
+            TRACE_ADD(3);
+          }
+          tc_fence_after_sync();
+          const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(ks * BN + hs * kSliceCols);
+          // 16-column chunks, double-buffered: the load of chunk c+1 is in flight while chunk c
+          // is accumulated; small enough that nothing spills under the register budget.
+          uint32_t va[16], vb[16];
+          tmem_ld_x16(t0, va);
+          tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              d_lo[j] = make_float4(acc_lo[4 * j], acc_lo[4 * j + 1], acc_lo[4 * j + 2], acc_lo[4 * j + 3]);
-              if (hi_valid)
-                d_hi[j] = make_float4(acc_hi[4 * j], acc_hi[4 * j + 1], acc_hi[4 * j + 2], acc_hi[4 * j + 3]);
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t next = (c < 3) ? t0 + 16 * (c + 1) : t0 + BNH;
+            if (c & 1) { tmem_ld_x16(next, va); promote16(acc_lo + 8 * c, vb, sc_lo); }
+            else       { tmem_ld_x16(next, vb); promote16(acc_lo + 8 * c, va, sc_lo); }
+            tmem_ld_wait();
+          }
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (c < 3) {
+              if (c & 1) tmem_ld_x16(t0 + BNH + 16 * (c + 1), va);
+              else       tmem_ld_x16(t0 + BNH + 16 * (c + 1), vb);
+            }
+            if (c & 1) promote16(acc_hi + 8 * c, vb, sc_hi);
+            else       promote16(acc_hi + 8 * c, va, sc_hi);
+            if (c < 3) tmem_ld_wait();
+            if (c == 2) {
+              // (the last chunk is in registers after this wait): this warp's reads of the
+              // accumulator are done, hand it back to the MMA warp
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&s->tmem_empty[ks]);
             }
           }
-          uint4* o_lo = reinterpret_cast<uint4*>(p.out_bf16 + out_row * p.N + col_lo);
-          uint4* o_hi = reinterpret_cast<uint4*>(p.out_bf16 + out_row * p.N + col_hi);
+          if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
+        }
+        if (!ok) break;
+#ifdef QARL_TRACE
+        const long long _tend0 = clock64();
+#endif
+
+        // ---- hand the tile to the epilogue warps as bf16 -----------------------------------
+        if ((MODE == kModeLinear || MODE == kModeDown) && p.out_f32 && valid) {  // debug fp32 dump
+          const int col_lo = c.n_tile * BN + hs * kSliceCols;
+          const int col_hi = col_lo + BNH;
+          float2* d_lo = reinterpret_cast<float2*>(p.out_f32 + static_cast<int64_t>(row) * p.N + col_lo);
+          float2* d_hi = reinterpret_cast<float2*>(p.out_f32 + static_cast<int64_t>(row) * p.N + col_hi);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint4 a, b;
-            if (MODE == kModeDown) {
-              a.x = pack_bf16x2(__fmul_rn(w, acc_lo[8 * j + 0]), __fmul_rn(w, acc_lo[8 * j + 1]));
-              a.y = pack_bf16x2(__fmul_rn(w, acc_lo[8 * j + 2]), __fmul_rn(w, acc_lo[8 * j + 3]));
-              a.z = pack_bf16x2(__fmul_rn(w, acc_lo[8 * j + 4]), __fmul_rn(w, acc_lo[8 * j + 5]));
-              a.w = pack_bf16x2(__fmul_rn(w, acc_lo[8 * j + 6]), __fmul_rn(w, acc_lo[8 * j + 7]));
-              b.x = pack_bf16x2(__fmul_rn(w, acc_hi[8 * j + 0]), __fmul_rn(w, acc_hi[8 * j + 1]));
-              b.y = pack_bf16x2(__fmul_rn(w, acc_hi[8 * j + 2]), __fmul_rn(w, acc_hi[8 * j + 3]));
-              b.z = pack_bf16x2(__fmul_rn(w, acc_hi[8 * j + 4]), __fmul_rn(w, acc_hi[8 * j + 5]));
-              b.w = pack_bf16x2(__fmul_rn(w, acc_hi[8 * j + 6]), __fmul_rn(w, acc_hi[8 * j + 7]));
-            } else {
-              a.x = pack_bf16x2(acc_lo[8 * j + 0], acc_lo[8 * j + 1]);
-              a.y = pack_bf16x2(acc_lo[8 * j + 2], acc_lo[8 * j + 3]);
-              a.z = pack_bf16x2(acc_lo[8 * j + 4], acc_lo[8 * j + 5]);
-              a.w = pack_bf16x2(acc_lo[8 * j + 6], acc_lo[8 * j + 7]);
-              b.x = pack_bf16x2(acc_hi[8 * j + 0], acc_hi[8 * j + 1]);
-              b.y = pack_bf16x2(acc_hi[8 * j + 2], acc_hi[8 * j + 3]);
-              b.z = pack_bf16x2(acc_hi[8 * j + 4], acc_hi[8 * j + 5]);
-              b.w = pack_bf16x2(acc_hi[8 * j + 6], acc_hi[8 * j + 7]);
-            }
-            o_lo[j] = a;
-            if (hi_valid) o_hi[j] = b;
+          for (int j = 0; j < 32; ++j) {
+            d_lo[j] = acc_lo[j];
+            if (col_hi < p.N) d_hi[j] = acc_hi[j];
           }
         }
-      } else {
-        // gate_up: lo half = gate columns, hi half = the matching up columns.
-        const int col = c.n_tile * BNH + cg * 32;  // column of h (and of gate) in [0, I)
-        uint32_t hb[16];                           // 32 bf16 values of h, packed in pairs
-        float amax = 0.0f;
+        if (MODE == kModeDown) {  // contribution = bf16( fl(w * y) )
+          const float2 w2 = make_float2(w, w);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const uint32_t g2 = pack_bf16x2(acc_lo[2 * j], acc_lo[2 * j + 1]);
-          const uint32_t u2 = pack_bf16x2(acc_hi[2 * j], acc_hi[2 * j + 1]);
-          const float h0 = silu_mul(bf16_bits_to_f32(g2 & 0xFFFFu), bf16_bits_to_f32(u2 & 0xFFFFu));
-          const float h1 = silu_mul(bf16_bits_to_f32(g2 >> 16), bf16_bits_to_f32(u2 >> 16));
-          hb[j] = pack_bf16x2(h0, h1);
-          amax = fmaxf(amax, fmaxf(fabsf(bf16_bits_to_f32(hb[j] & 0xFFFFu)), fabsf(bf16_bits_to_f32(hb[j] >> 16))));
-          if (p.out_bf16 && valid) {  // debug dump of the bf16 gate_up row
-            p.out_bf16[static_cast<int64_t>(row) * p.N + col + 2 * j] = static_cast<uint16_t>(g2 & 0xFFFFu);
-            p.out_bf16[static_cast<int64_t>(row) * p.N + col + 2 * j + 1] = static_cast<uint16_t>(g2 >> 16);
-            p.out_bf16[static_cast<int64_t>(row) * p.N + p.I + col + 2 * j] = static_cast<uint16_t>(u2 & 0xFFFFu);
-            p.out_bf16[static_cast<int64_t>(row) * p.N + p.I + col + 2 * j + 1] = static_cast<uint16_t>(u2 >> 16);
+          for (int j = 0; j < 32; ++j) {
+            acc_lo[j] = __fmul2_rn(w2, acc_lo[j]);
+            acc_hi[j] = __fmul2_rn(w2, acc_hi[j]);
           }
         }
-        // the 128-wide quantization group of this row spans the 4 column slices (4 warps)
-        // (double-buffered by tile so that a fast warp cannot overwrite values still being read)
-        const uint32_t xb = tile_iter & 1u;
-        s->amax[xb][cg][r] = amax;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s->amax_bar[xb]);
-        if (!wait_or_abort(&s->amax_bar[xb], (tile_iter >> 1) & 1u, s, p)) break;
-        amax = fmaxf(fmaxf(s->amax[xb][0][r], s->amax[xb][1][r]), fmaxf(s->amax[xb][2][r], s->amax[xb][3][r]));
-        float inv;
-        const float sc = block_scale(amax, &inv);
-        if (valid) {
-          uint32_t cw[8];
+        {
+          TRACE_T0();
+          if (!wait_or_abort(&s->out_empty, (tile_iter & 1u) ^ 1u, s, p)) break;  // previous tile drained
+          TRACE_ADD(4);
+        }
+        {
+          uint4* d_lo = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + hs * (kSliceCols * 2));
+          uint4* d_hi = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + BNH * 2 + hs * (kSliceCols * 2));
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float f0 = __fmul_rn(bf16_bits_to_f32(hb[2 * j] & 0xFFFFu), inv);
-            const float f1 = __fmul_rn(bf16_bits_to_f32(hb[2 * j] >> 16), inv);
-            const float f2 = __fmul_rn(bf16_bits_to_f32(hb[2 * j + 1] & 0xFFFFu), inv);
-            const float f3 = __fmul_rn(bf16_bits_to_f32(hb[2 * j + 1] >> 16), inv);
-            cw[j] = cvt_e4m3x4(f0, f1, f2, f3);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(p.h_codes + static_cast<int64_t>(row) * p.I + col);
-          dst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-          dst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
-          if (cg == 0) p.h_scales[static_cast<int64_t>(row) * (p.I / BNH) + c.n_tile] = sc;
-          if (p.h_bf16) {
-            uint4* hd = reinterpret_cast<uint4*>(p.h_bf16 + static_cast<int64_t>(row) * p.I + col);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) hd[j] = make_uint4(hb[4 * j], hb[4 * j + 1], hb[4 * j + 2], hb[4 * j + 3]);
+            d_lo[j] = make_uint4(bf16x2_bits(acc_lo[4 * j].x, acc_lo[4 * j].y), bf16x2_bits(acc_lo[4 * j + 1].x, acc_lo[4 * j + 1].y),
+                                 bf16x2_bits(acc_lo[4 * j + 2].x, acc_lo[4 * j + 2].y), bf16x2_bits(acc_lo[4 * j + 3].x, acc_lo[4 * j + 3].y));
+            d_hi[j] = make_uint4(bf16x2_bits(acc_hi[4 * j].x, acc_hi[4 * j].y), bf16x2_bits(acc_hi[4 * j + 1].x, acc_hi[4 * j + 1].y),
+                                 bf16x2_bits(acc_hi[4 * j + 2].x, acc_hi[4 * j + 2].y), bf16x2_bits(acc_hi[4 * j + 3].x, acc_hi[4 * j + 3].y));
           }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s->out_full);
+#ifdef QARL_TRACE
+        trace_acc[8] += clock64() - _tend0;
+#endif
+        if (!has_next) break;
+        T = Tn;
+        c = cn;
         ++tile_iter;
       }
     }
   }
 
+#ifdef QARL_TRACE
+  if (p.trace && lane == 0 && (warp == kTmaWarp || warp == kMmaWarp || warp == 0 || warp == kPromoWarps)) {
+    unsigned long long* t = p.trace + static_cast<size_t>(blockIdx.x) * 16;
+    if (warp == kTmaWarp) t[0] = trace_acc[0];
+    if (warp == kMmaWarp) { t[1] = trace_acc[1]; t[2] = trace_acc[2]; }
+    if (warp == 0) { t[3] = trace_acc[3]; t[4] = trace_acc[4]; t[5] = clock64() - trace_start; t[8] = trace_acc[8]; t[9] = trace_acc[9]; t[10] = trace_acc[10]; }
+    if (warp == kPromoWarps) { t[6] = trace_acc[6]; t[7] = clock64() - trace_start; }
+  }
+#endif
   // ---- teardown ---------------------------------------------------------------------------
   tc_fence_before_sync();
   __syncthreads();
@@ -432,6 +586,12 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
 }
 
 }  // namespace
+
+#ifdef QARL_TRACE
+static unsigned long long* g_trace = nullptr;
+static unsigned g_trace_launch = 0;
+extern "C" void qarl_trace_set(unsigned long long* dev_ptr) { g_trace = dev_ptr; }
+#endif
 
 namespace {
 
@@ -494,6 +654,9 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
   p.pair_weights = a.pair_weights;
   p.status = L.d_status;
   p.wait_limit_ns = 2000000000ull;
+#ifdef QARL_TRACE
+  p.trace = g_trace ? g_trace + static_cast<size_t>(g_trace_launch++ & 1) * 148 * 16 : nullptr;
+#endif
   // upper bound on the tile count (group sizes live on the device): each expert adds at most
   // one partial row tile
   const int64_t m_tiles_max = a.rows_total / BM + a.E;

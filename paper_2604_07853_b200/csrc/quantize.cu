@@ -80,7 +80,9 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const uint16_t* __
 __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __restrict__ x, int64_t M, int64_t K,
                                                            int64_t ldx, uint8_t* __restrict__ codes,
                                                            float* __restrict__ scales,
-                                                           const int32_t* __restrict__ dst_rows, int fanout) {
+                                                           const int32_t* __restrict__ dst_rows, int fanout,
+                                                           const float* __restrict__ pair_w,
+                                                           float* __restrict__ sorted_w) {
   const int64_t kb = K / kBlock;
   const int64_t gid = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;
   const bool live = gid < M * kb;
@@ -110,6 +112,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
       const int64_t d = dst_rows[row * fanout + j];
       *reinterpret_cast<uint4*>(codes + d * K + b * kBlock + sub * 16) = out;
       if (sub == 0) scales[d * kb + b] = s;
+      if (sub == 0 && b == 0 && sorted_w != nullptr) sorted_w[d] = pair_w[row * fanout + j];
     }
   }
 }
@@ -126,12 +129,13 @@ cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E
 }
 
 cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
-                                uint8_t* codes, float* scales, const int32_t* dst_rows, int fanout) {
+                                uint8_t* codes, float* scales, const int32_t* dst_rows, int fanout,
+                                const float* pair_w, float* sorted_w) {
   const int64_t groups = M * (K / kBlock);
   if (groups == 0) return cudaSuccess;
   const int64_t blocks = (groups * 8 + 255) / 256;
   quantize_act_kernel<<<static_cast<unsigned>(blocks), 256, 0, L.stream>>>(x, M, K, ldx, codes, scales, dst_rows,
-                                                                           fanout);
+                                                                           fanout, pair_w, sorted_w);
   ++*L.launches;
   return cudaGetLastError();
 }
