@@ -210,7 +210,7 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2604_07853_b200 import binding, build
+    from paper_2604_07853_b200 import binding, build, sharding
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -229,11 +229,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(v, dev)
 
     # ---------------- training-forward shape: the headline step
     w13, w2, x, ids, wts = make_inputs(M_TRAIN, 1000 + rank, dev, zipf=True)
