@@ -1,0 +1,27 @@
+/*
+ * qarl_harness.h -- test-harness helpers that ship in the same library but are NOT part of the
+ * quantized-forward API.  The paper's pipeline has no counterpart for them: they exist so that
+ * the rollout-alignment stack test (consecutive MoE layers with RMSNorm + residual in between)
+ * can glue layers together with an operation whose result for a row does not depend on the
+ * batch it runs in.
+ */
+#ifndef QARL_HARNESS_H_
+#define QARL_HARNESS_H_
+
+#include "qarl.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* out[m,:] = bf16( x[m,:] * rsqrt(mean(x[m,:]^2) + eps) ), weight = 1.  x, out: device bf16
+ * [M, H], H a multiple of 8, 16-byte aligned, may alias.  The sum of squares of a row is
+ * accumulated in fp32 in a fixed per-row order (lane-strided partial sums, then a butterfly),
+ * so a row's output bytes are the same for every M.  Asynchronous on `stream`. */
+int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H, float eps,
+                         void* out_bf16, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QARL_HARNESS_H_ */

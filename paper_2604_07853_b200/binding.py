@@ -31,6 +31,7 @@ EXPORTS = [
     "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
     "qarl_profile_begin", "qarl_profile_end",
 ]
+HARNESS_EXPORTS = ["qarl_harness_rmsnorm"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine"]
 
@@ -93,6 +94,8 @@ def load() -> C.CDLL:
     L.qarl_profile_begin.argtypes = [p, C.c_int]
     L.qarl_profile_end.restype = C.c_int
     L.qarl_profile_end.argtypes = [p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.qarl_harness_rmsnorm.restype = C.c_int
+    L.qarl_harness_rmsnorm.argtypes = [p, p, i64, i64, C.c_float, p, p]
     _lib = L
     return L
 
@@ -167,6 +170,14 @@ class Context:
         cnt = (C.c_int64 * n)()
         self._check(self.lib.qarl_profile_end(self.h, ms, cnt))
         return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
+
+    def harness_rmsnorm(self, x: torch.Tensor, eps: float = 1e-6, out=None):
+        """Row-invariant RMSNorm (weight 1) used by the alignment-stack test; not part of the API."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        M, H = x.shape
+        y = out if out is not None else torch.empty_like(x)
+        self._check(self.lib.qarl_harness_rmsnorm(self.h, _ptr(x), M, H, eps, _ptr(y), _stream()))
+        return y
 
     # ------------------------------------------------------------------ calls
     def quantize_weight(self, w: torch.Tensor, codes=None, scales=None):

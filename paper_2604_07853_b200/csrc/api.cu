@@ -7,19 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
-
-struct qarl_ctx {
-  int device;
-  int sm_count;
-  int* d_status;
-  int64_t launches;
-  qarl::EncodeTiledFn encode;
-  char err[256];
-  // stage timing: marks[i] closes stage mark_stage[i] (-1: an opening mark)
-  std::vector<cudaEvent_t> marks;
-  std::vector<int> mark_stage;
-  size_t marks_used = 0;
-};
+#include "../../include/qarl_harness.h"
 
 namespace {
 
@@ -391,6 +379,17 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
       return cuda_fail(ctx, e, "copy h_scales");
   }
   return QARL_OK;
+}
+
+int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, float eps, void* out, void* stream) {
+  if (!ctx || M < 0 || H <= 0) return QARL_ERR_INVALID_ARG;
+  if (H % 8) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (M == 0) return QARL_OK;
+  if (!x || !out) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(out)) return QARL_ERR_MISALIGNED;
+  cudaError_t e = launch_rmsnorm(make_launch(ctx, stream), static_cast<const uint16_t*>(x), M, H, eps,
+                                 static_cast<uint16_t*>(out));
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "rmsnorm");
 }
 
 }  // extern "C"

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/qarl.h"
 
 namespace qarl {
@@ -76,6 +78,8 @@ cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64
 cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
                            int64_t H, int64_t E, uint16_t* out);
 
+cudaError_t launch_rmsnorm(const Launch& L, const uint16_t* x, int64_t M, int64_t H, float eps, uint16_t* out);
+
 enum GemmMode { kModeLinear = 0, kModeGateUp = 1, kModeDown = 2 };
 
 struct GemmArgs {
@@ -109,3 +113,17 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
 
 }  // namespace qarl
+
+// The opaque context of the C ABI (one per device).
+struct qarl_ctx {
+  int device;
+  int sm_count;
+  int* d_status;
+  int64_t launches;
+  qarl::EncodeTiledFn encode;
+  char err[256];
+  // stage timing: marks[i] closes stage mark_stage[i] (-1: an opening mark)
+  std::vector<cudaEvent_t> marks;
+  std::vector<int> mark_stage;
+  size_t marks_used = 0;
+};

@@ -21,7 +21,10 @@ def test_exports_match_header(lib):
     code = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     declared = set(re.findall(r"\b(qarl_[a-z_0-9]+)\s*\(", code))
     assert declared == set(binding.EXPORTS)
-    for name in declared:
+    hdr2 = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "qarl_harness.h")).read(), flags=re.S)
+    declared2 = set(re.findall(r"\b(qarl_[a-z_0-9]+)\s*\(", hdr2))
+    assert declared2 == set(binding.HARNESS_EXPORTS)
+    for name in declared | declared2:
         assert hasattr(lib, name), name
 
 
