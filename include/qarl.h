@@ -97,6 +97,36 @@ int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* x_codes, const float* x_scal
                       int64_t M, int64_t K, const uint8_t* w_codes, const float* w_scales,
                       int64_t N, void* y_bf16, float* y_f32, void* stream);
 
+/* Allocation-free variant of qarl_linear_fwd (the paper has no counterpart; this is a
+ * packaging choice of this library).
+ *
+ * Who needs it: code that is not allowed to obtain device memory when it makes the call -- a
+ * serving process that handed every free byte of the GPU to its KV-cache pool at start-up, a
+ * plugin running under a host application that owns the allocator, a latency-critical loop
+ * in which cudaMalloc's implicit device synchronization is unacceptable.  Such a caller
+ * cannot hand over the workspace qarl_linear_fwd asks for.  Here the scratch (the e4m3 copy of
+ * the activations and their scales) is a fixed array inside the library's device image instead:
+ * QARL_STATIC_LINEAR_MAX_ELEMS bytes of codes plus 1/32 of that for scales (about 4.1 MiB),
+ * resident on every GPU that loads the library, for the life of the process.
+ *
+ * Same arithmetic and same output bytes as qarl_linear_fwd.  The caller still passes the
+ * input and the output: x_bf16 [M, K] dense, w_codes [N, K], w_scales [N/128, K/128], y_bf16
+ * [M, N] (device pointers, alignment as for qarl_linear_fwd); there is no fp32 dump.
+ *   - M * K must not exceed QARL_STATIC_LINEAR_MAX_ELEMS, otherwise the call returns
+ *     QARL_ERR_UNSUPPORTED_SHAPE before launching anything (qarl_last_cuda_error has the text).
+ *   - The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - The first call on a device looks up the array's device address; the context's device
+ *     must be the current device for that call, and that first call should be made before
+ *     any stream capture begins.
+ *   - All calls on a device share the one array, which keeps whatever the last call left in
+ *     it.  Every byte a call reads it has first rewritten itself, so nothing needs clearing
+ *     between calls; but two calls that overlap on the GPU (different streams, or different
+ *     contexts on the same device) race on the array and corrupt each other's results. */
+#define QARL_STATIC_LINEAR_MAX_ELEMS (4 * 1024 * 1024)
+int qarl_linear_fwd_static(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t K,
+                           const uint8_t* w_codes, const float* w_scales, int64_t N,
+                           void* y_bf16, void* stream);
+
 /* Optional dumps of the MoE layer's intermediates (every field may be NULL).  "Sorted
  * order" is the order of token-expert pairs after grouping by expert: position q holds the
  * flat pair sorted_pair[q] = t*k + j. */

@@ -29,8 +29,9 @@ EXPORTS = [
     "qarl_last_cuda_error", "qarl_quantize_weight", "qarl_quantize_act",
     "qarl_linear_workspace_bytes", "qarl_linear_fwd", "qarl_linear_fwd_q",
     "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
-    "qarl_profile_begin", "qarl_profile_end",
+    "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
 ]
+STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine"]
@@ -94,6 +95,8 @@ def load() -> C.CDLL:
     L.qarl_profile_begin.argtypes = [p, C.c_int]
     L.qarl_profile_end.restype = C.c_int
     L.qarl_profile_end.argtypes = [p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.qarl_linear_fwd_static.restype = C.c_int
+    L.qarl_linear_fwd_static.argtypes = [p, p, i64, i64, p, p, i64, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
     L.qarl_harness_rmsnorm.argtypes = [p, p, i64, i64, C.c_float, p, p]
     _lib = L
@@ -216,6 +219,21 @@ class Context:
         self._check(self.lib.qarl_linear_fwd(self.h, _ptr(x), M, K, _ptr(w_codes), _ptr(w_scales), N,
                                              _ptr(y), _ptr(y32), _ptr(ws), ws.numel(), _stream()))
         return (y, y32) if want_f32 else y
+
+    def linear_fwd_static(self, x, w_codes, w_scales, out):
+        """qarl_linear_fwd_static: the dense projection for callers that cannot allocate device
+        memory.  The scratch is a fixed array inside the library (M*K <= STATIC_LINEAR_MAX_ELEMS);
+        the caller passes the input and a preallocated output, and this wrapper allocates
+        nothing either.  Calls that overlap on the GPU race on that array."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous() and out.dtype == torch.bfloat16
+        M, K = x.shape
+        N = w_codes.shape[0]
+        assert out.shape == (M, N) and out.is_contiguous()
+        rc = self.lib.qarl_linear_fwd_static(self.h, _ptr(x), M, K, _ptr(w_codes), _ptr(w_scales), N,
+                                             _ptr(out), _stream())
+        if rc != QARL_OK:
+            raise QarlError(rc, self.lib.qarl_last_cuda_error(self.h).decode())
+        return out
 
     def linear_fwd_q(self, x_codes, x_scales, w_codes, w_scales, out=None, want_f32: bool = False):
         M, K = x_codes.shape

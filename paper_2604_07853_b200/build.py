@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqarl.so")
-SOURCES = ["api.cu", "quantize.cu", "permute.cu", "combine.cu", "gemm_sm100.cu", "harness.cu"]
+SOURCES = ["api.cu", "quantize.cu", "permute.cu", "combine.cu", "gemm_sm100.cu", "harness.cu", "linear_static.cu"]
 HEADERS = ["common.cuh", "ptx_sm100.cuh", os.path.join("..", "..", "include", "qarl.h"),
            os.path.join("..", "..", "include", "qarl_harness.h")]
 
