@@ -299,11 +299,8 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   pb.offsets = reinterpret_cast<int32_t*>(ws + pl.offsets);
   pb.sorted_pair = reinterpret_cast<int32_t*>(ws + pl.sorted_pair);
   pb.pos_of_pair = reinterpret_cast<int32_t*>(ws + pl.pos_of_pair);
-  // Bad ids are skipped by the permutation, which would leave sorted positions unwritten:
-  // start from a valid (if meaningless) permutation so later kernels stay in bounds.
-  if ((e = cudaMemsetAsync(pb.sorted_pair, 0, P * sizeof(int32_t), L.stream)) != cudaSuccess ||
-      (e = cudaMemsetAsync(pb.pos_of_pair, 0, P * sizeof(int32_t), L.stream)) != cudaSuccess)
-    return cuda_fail(ctx, e, "memset");
+  // Bad ids are skipped by the permutation and leave their entries of these arrays stale; every
+  // consumer clamps the indices it reads from them, so no clearing pass is needed.
   mark(ctx, L.stream, -1);
   if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
   mark(ctx, L.stream, QARL_STAGE_PERMUTE);
@@ -311,7 +308,6 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   uint8_t* a_codes = ws + pl.a_codes;
   float* a_scales = reinterpret_cast<float*>(ws + pl.a_scales);
   float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
-  if ((e = cudaMemsetAsync(sorted_w, 0, P * sizeof(float), L.stream)) != cudaSuccess) return cuda_fail(ctx, e, "memset");
   if ((e = launch_quantize_act(L, static_cast<const uint16_t*>(x), M, H, H, a_codes, a_scales, pb.pos_of_pair,
                                static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
     return cuda_fail(ctx, e, "quantize_act");

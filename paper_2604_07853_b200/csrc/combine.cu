@@ -13,6 +13,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint16_t* __restrict
                                                       const int32_t* __restrict__ ids, int64_t M, int k, int64_t H,
                                                       uint16_t* __restrict__ out, int* status) {
   __shared__ int order[kMaxTopK];
+  pdl_trigger();
+  pdl_wait();
   const int64_t t = blockIdx.x;
   const int tid = threadIdx.x;
   if (tid < k) {
@@ -55,10 +57,9 @@ cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32
                            int64_t H, int64_t E, uint16_t* out) {
   (void)E;
   if (M == 0) return cudaSuccess;
-  combine_kernel<<<static_cast<unsigned>(M), 256, 0, L.stream>>>(contrib, ids, M, static_cast<int>(k), H, out,
-                                                                  L.d_status);
   ++*L.launches;
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, static_cast<unsigned>(M), 256, 0, L.stream, contrib, ids, M, static_cast<int>(k), H,
+                    out, L.d_status);
 }
 
 }  // namespace qarl

@@ -43,6 +43,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
 }
 
+// Programmatic dependent launch: every kernel of the library is launched so that it may begin
+// while its predecessor in the stream is still draining.  A kernel calls pdl_trigger() at once
+// (its successor may start launching) and pdl_wait() before its first access to global memory
+// (the predecessor, and transitively everything before it, has completed and is visible).
+// Only barrier set-up, TMEM allocation and other memory-free preamble runs ahead of the wait.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Device status word protocol: first error wins.
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
@@ -54,6 +62,23 @@ struct Launch {
   int* d_status;
   int64_t* launches;  // host counter
 };
+
+// Launch with the programmatic-stream-serialization attribute (see pdl_wait above).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                       Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
                                    uint8_t* codes, float* scales);

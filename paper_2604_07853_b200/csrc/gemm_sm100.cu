@@ -183,6 +183,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
 #endif
 
   // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
+  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&s->full[i], 1);
@@ -205,6 +206,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     tmem_alloc(&s->tmem_addr, kTmemCols);
     tmem_relinquish();
   }
+  pdl_wait();  // everything above touched no global memory; from here on the predecessor's results are needed
   for (int e = threadIdx.x; e <= p.E; e += kThreads)
     s->off[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.rows_total);
   __syncthreads();
@@ -245,9 +247,8 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         uint32_t armed = 0, armed_parity = 0;  // per-stage: has a load in flight / its parity
         int cur_e = 0;
         bool ok = true;
-        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
-          const TileCoord c = decode_tile(s, T, cur_e);
-          int row_lo, row_hi;
+        // weight rows of a tile's two halves
+        auto b_rows = [&](const TileCoord& c, int& row_lo, int& row_hi) {
           if (MODE == kModeGateUp) {
             row_lo = c.e * p.N + c.n_tile * BNH;
             row_hi = row_lo + p.I;
@@ -255,6 +256,11 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             row_lo = c.e * p.N + c.n_tile * BN;
             row_hi = row_lo + BNH;
           }
+        };
+        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
+          const TileCoord c = decode_tile(s, T, cur_e);
+          int row_lo, row_hi;
+          b_rows(c, row_lo, row_hi);
           for (int kb = 0; kb < KB; ++kb) {
             {
               TRACE_T0();
@@ -322,7 +328,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       int my_pair = 0;  // down: destination (flat pair id) of the lane-th row this warp handles
       if (MODE == kModeDown) {
         const int row = c.m0 + ew + kEpiWarps * lane;
-        if (row < c.m_end) my_pair = __ldg(p.sorted_pair + row);
+        if (row < c.m_end) my_pair = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
       }
       {
         TRACE_T0();
@@ -451,6 +457,9 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       for (;;) {
         const int row = c.m0 + r;
         const bool valid = row < c.m_end;
+        // a warp whose 32 rows all lie past the group's end (ragged tails, decode-sized groups)
+        // keeps the barrier protocol going but reads and accumulates nothing
+        const bool warp_live = c.m0 + q * 32 < c.m_end;
         const int Tn = T + gridDim.x;
         const bool has_next = Tn < total_tiles;
         TileCoord cn = c;
@@ -481,34 +490,39 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             TRACE_ADD(3);
           }
           tc_fence_after_sync();
-          const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(ks * BN + hs * kSliceCols);
-          // 16-column chunks, double-buffered: the load of chunk c+1 is in flight while chunk c
-          // is accumulated; small enough that nothing spills under the register budget.
-          uint32_t va[16], vb[16];
-          tmem_ld_x16(t0, va);
-          tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint32_t next = (c < 3) ? t0 + 16 * (c + 1) : t0 + BNH;
-            if (c & 1) { tmem_ld_x16(next, va); promote16(acc_lo + 8 * c, vb, sc_lo); }
-            else       { tmem_ld_x16(next, vb); promote16(acc_lo + 8 * c, va, sc_lo); }
+          if (!warp_live) {
+            tc_fence_before_sync();
+            if (lane == 0) mbar_arrive(&s->tmem_empty[ks]);
+          } else {
+            const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(ks * BN + hs * kSliceCols);
+            // 16-column chunks, double-buffered: the load of chunk c+1 is in flight while chunk c
+            // is accumulated; small enough that nothing spills under the register budget.
+            uint32_t va[16], vb[16];
+            tmem_ld_x16(t0, va);
             tmem_ld_wait();
-          }
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if (c < 3) {
-              if (c & 1) tmem_ld_x16(t0 + BNH + 16 * (c + 1), va);
-              else       tmem_ld_x16(t0 + BNH + 16 * (c + 1), vb);
+            for (int c = 0; c < 4; ++c) {
+              const uint32_t next = (c < 3) ? t0 + 16 * (c + 1) : t0 + BNH;
+              if (c & 1) { tmem_ld_x16(next, va); promote16(acc_lo + 8 * c, vb, sc_lo); }
+              else       { tmem_ld_x16(next, vb); promote16(acc_lo + 8 * c, va, sc_lo); }
+              tmem_ld_wait();
             }
-            if (c & 1) promote16(acc_hi + 8 * c, vb, sc_hi);
-            else       promote16(acc_hi + 8 * c, va, sc_hi);
-            if (c < 3) tmem_ld_wait();
-            if (c == 2) {
-              // (the last chunk is in registers after this wait): this warp's reads of the
-              // accumulator are done, hand it back to the MMA warp
-              tc_fence_before_sync();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&s->tmem_empty[ks]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (c < 3) {
+                if (c & 1) tmem_ld_x16(t0 + BNH + 16 * (c + 1), va);
+                else       tmem_ld_x16(t0 + BNH + 16 * (c + 1), vb);
+              }
+              if (c & 1) promote16(acc_hi + 8 * c, vb, sc_hi);
+              else       promote16(acc_hi + 8 * c, va, sc_hi);
+              if (c < 3) tmem_ld_wait();
+              if (c == 2) {
+                // (the last chunk is in registers after this wait): this warp's reads of the
+                // accumulator are done, hand it back to the MMA warp
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s->tmem_empty[ks]);
+              }
             }
           }
           if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
@@ -543,7 +557,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           if (!wait_or_abort(&s->out_empty, (tile_iter & 1u) ^ 1u, s, p)) break;  // previous tile drained
           TRACE_ADD(4);
         }
-        {
+        if (warp_live) {
           uint4* d_lo = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + hs * (kSliceCols * 2));
           uint4* d_hi = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + BNH * 2 + hs * (kSliceCols * 2));
 #pragma unroll
@@ -617,9 +631,8 @@ cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMa
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  gemm_blockscaled_kernel<MODE><<<grid, kThreads, kSmemBytes, L.stream>>>(ta, tb, p);
   ++*L.launches;
-  return cudaGetLastError();
+  return launch_pdl(gemm_blockscaled_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
 }
 
 }  // namespace

@@ -110,19 +110,45 @@ __device__ int block_exclusive_scan(int32_t* a, int n, int32_t* scratch) {
 }
 
 // ---- small problems (P <= 2048): one CTA does histogram, scan and scatter ----------------
+// Each lane keeps its 8 ids in registers for both passes, so global memory is read once and
+// the eight loads are in flight together (this kernel is pure latency at decode sizes).
 __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int32_t* __restrict__ ids, int64_t P,
                                                                       int E, int32_t* __restrict__ offsets,
                                                                       int32_t* __restrict__ sorted_pair,
                                                                       int32_t* __restrict__ pos_of_pair,
                                                                       int* status) {
   extern __shared__ int32_t sm[];
+  pdl_trigger();
+  pdl_wait();
   int32_t* whist = sm;                 // [kWarps][E]
   int32_t* total = sm + kWarps * E;    // [E]
   int32_t* scratch = total + E;        // [33]
-  const int tid = threadIdx.x, wid = tid >> 5;
+  const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+  constexpr int kRounds = kPairsPerWarp / 32;
+  const int64_t p0 = static_cast<int64_t>(wid) * kPairsPerWarp + lane;
+  int my[kRounds];
+  bool bad = false;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int64_t p = p0 + r * 32;
+    int e = -1;
+    if (p < P) {
+      e = __ldg(ids + p);
+      if (e < 0 || e >= E) { bad = true; e = -1; }
+    }
+    my[r] = e;
+  }
+  if (bad) set_status(status, QARL_ERR_BAD_EXPERT_ID);
   for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
   __syncthreads();
-  warp_histogram(ids, static_cast<int64_t>(wid) * kPairsPerWarp, P, E, whist + wid * E, status);
+  int32_t* hist_w = whist + wid * E;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int e = my[r];
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
+    __syncwarp();
+  }
   __syncthreads();
   for (int e = tid; e < E; e += kThreads) {
     int s = 0;
@@ -142,13 +168,30 @@ __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int3
   }
   if (tid == 0) offsets[E] = all;
   __syncthreads();
-  warp_scatter(ids, static_cast<int64_t>(wid) * kPairsPerWarp, P, E, whist + wid * E, sorted_pair, pos_of_pair);
+  const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int e = my[r];
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    int pos = -1;
+    if (e >= 0) pos = hist_w[e] + __popc(peers & lt);
+    __syncwarp();
+    if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
+    __syncwarp();
+    if (e >= 0) {
+      const int64_t p = p0 + r * 32;
+      sorted_pair[pos] = static_cast<int32_t>(p);
+      pos_of_pair[p] = pos;
+    }
+  }
 }
 
 // ---- large problems: per-chunk histogram, one-CTA scan, per-chunk scatter ----------------
 __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ ids, int64_t P, int E,
                                                                 int32_t* __restrict__ chunk_hist, int* status) {
   extern __shared__ int32_t sm[];
+  pdl_trigger();
+  pdl_wait();
   int32_t* whist = sm;
   const int tid = threadIdx.x, wid = tid >> 5;
   for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
@@ -169,6 +212,8 @@ __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* _
 __global__ void __launch_bounds__(1024) permute_scan_kernel(int32_t* __restrict__ chunk_hist, int nchunks, int E,
                                                             int32_t* __restrict__ offsets) {
   extern __shared__ int32_t sm[];
+  pdl_trigger();
+  pdl_wait();
   const int G = max(1, min(static_cast<int>(blockDim.x) / E, nchunks));
   int32_t* part = sm;            // [G][E]
   int32_t* total = sm + G * E;   // [E]
@@ -214,6 +259,8 @@ __global__ void __launch_bounds__(kThreads) permute_scatter_kernel(const int32_t
                                                                    int32_t* __restrict__ sorted_pair,
                                                                    int32_t* __restrict__ pos_of_pair, int* status) {
   extern __shared__ int32_t sm[];
+  pdl_trigger();
+  pdl_wait();
   int32_t* whist = sm;
   const int tid = threadIdx.x, wid = tid >> 5;
   for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
@@ -250,25 +297,22 @@ cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64
                                  static_cast<int>(smem));
       if (err != cudaSuccess) return err;
     }
-    permute_single_cta_kernel<<<1, kThreads, smem, L.stream>>>(ids, P, e, b.offsets, b.sorted_pair, b.pos_of_pair,
-                                                               L.d_status);
     ++*L.launches;
-    return cudaGetLastError();
+    return launch_pdl(permute_single_cta_kernel, 1, kThreads, smem, L.stream, ids, P, e, b.offsets, b.sorted_pair,
+                      b.pos_of_pair, L.d_status);
   }
   const size_t smem_h = static_cast<size_t>(kWarps) * e * sizeof(int32_t);
   const int G = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(1024 / e, nchunks)));
   const size_t smem_s = (static_cast<size_t>(G) * e + e + 33) * sizeof(int32_t);
-  permute_hist_kernel<<<static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream>>>(ids, P, e, b.chunk_hist,
-                                                                                     L.d_status);
-  ++*L.launches;
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  permute_scan_kernel<<<1, 1024, smem_s, L.stream>>>(b.chunk_hist, static_cast<int>(nchunks), e, b.offsets);
-  ++*L.launches;
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  permute_scatter_kernel<<<static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream>>>(
-      ids, P, e, b.chunk_hist, b.offsets, b.sorted_pair, b.pos_of_pair, L.d_status);
-  ++*L.launches;
-  return cudaGetLastError();
+  *L.launches += 3;
+  if ((err = launch_pdl(permute_hist_kernel, static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream, ids, P, e,
+                        b.chunk_hist, L.d_status)) != cudaSuccess)
+    return err;
+  if ((err = launch_pdl(permute_scan_kernel, 1, 1024, smem_s, L.stream, b.chunk_hist, static_cast<int>(nchunks), e,
+                        b.offsets)) != cudaSuccess)
+    return err;
+  return launch_pdl(permute_scatter_kernel, static_cast<unsigned>(nchunks), kThreads, smem_h, L.stream, ids, P, e,
+                    b.chunk_hist, b.offsets, b.sorted_pair, b.pos_of_pair, L.d_status);
 }
 
 }  // namespace qarl

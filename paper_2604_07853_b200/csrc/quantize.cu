@@ -33,6 +33,8 @@ __device__ __forceinline__ void encode8(const uint4& v, float inv, uint32_t& c0,
 __global__ void __launch_bounds__(256) quantize_weight_kernel(const uint16_t* __restrict__ w, int64_t N, int64_t K,
                                                               uint8_t* __restrict__ codes,
                                                               float* __restrict__ scales) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t kb = K / kBlock, nb = N / kBlock;
   const int64_t blk = blockIdx.x;
   const int64_t bk = blk % kb, bn = (blk / kb) % nb, e = blk / (kb * nb);
@@ -81,8 +83,11 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
                                                            int64_t ldx, uint8_t* __restrict__ codes,
                                                            float* __restrict__ scales,
                                                            const int32_t* __restrict__ dst_rows, int fanout,
+                                                           int64_t dst_rows_total,
                                                            const float* __restrict__ pair_w,
                                                            float* __restrict__ sorted_w) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t kb = K / kBlock;
   const int64_t gid = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;
   const bool live = gid < M * kb;
@@ -109,7 +114,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
     if (sub == 0) scales[row * kb + b] = s;
   } else {
     for (int j = 0; j < fanout; ++j) {
-      const int64_t d = dst_rows[row * fanout + j];
+      // clamped: a pair with a bad expert id has no sorted position and leaves this entry stale
+      const int64_t d = min(max(static_cast<int64_t>(dst_rows[row * fanout + j]), int64_t(0)), dst_rows_total - 1);
       *reinterpret_cast<uint4*>(codes + d * K + b * kBlock + sub * 16) = out;
       if (sub == 0) scales[d * kb + b] = s;
       if (sub == 0 && b == 0 && sorted_w != nullptr) sorted_w[d] = pair_w[row * fanout + j];
@@ -123,9 +129,8 @@ cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E
                                    uint8_t* codes, float* scales) {
   const int64_t blocks = E * (N / kBlock) * (K / kBlock);
   if (blocks == 0) return cudaSuccess;
-  quantize_weight_kernel<<<static_cast<unsigned>(blocks), 256, 0, L.stream>>>(w, N, K, codes, scales);
   ++*L.launches;
-  return cudaGetLastError();
+  return launch_pdl(quantize_weight_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, N, K, codes, scales);
 }
 
 cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
@@ -134,10 +139,9 @@ cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, i
   const int64_t groups = M * (K / kBlock);
   if (groups == 0) return cudaSuccess;
   const int64_t blocks = (groups * 8 + 255) / 256;
-  quantize_act_kernel<<<static_cast<unsigned>(blocks), 256, 0, L.stream>>>(x, M, K, ldx, codes, scales, dst_rows,
-                                                                           fanout, pair_w, sorted_w);
   ++*L.launches;
-  return cudaGetLastError();
+  return launch_pdl(quantize_act_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, x, M, K, ldx, codes, scales,
+                    dst_rows, fanout, M * fanout, pair_w, sorted_w);
 }
 
 }  // namespace qarl
