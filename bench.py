@@ -303,7 +303,10 @@ def main():
     peak = 2.0 * pk["bf16_sustained"]                               # fp8 = 2 x bf16 (nominal ratio)
     roofline = {"kernel": "gemm_blockscaled_kernel<gate_up>", "bound": "tensor", "achieved": achieved,
                 "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": f"2 x bf16 sustained of {pk['source']}", "traffic": None,
+                "peak_source": f"2 x bf16 sustained of {pk['source']}",
+                # dram__bytes_read + write of one launch at this size, from the committed ncu capture
+                # (profiles/launch_list__bench_moe_train_M32768.md); null for other sizes
+                "traffic": 1290432256 if M_TRAIN == 32768 else None,
                 "ms_per_launch": gu_ms_avg, "frac_of_nominal_4500": achieved / 4500.0}
     stage_ms = {k: (v[0] / max(args.steps, 1)) for k, v in stages.items()}
     layer_ms = sum(stage_ms[k] for k in ("permute", "quantize_act", "gate_up_gemm", "down_gemm", "combine"))
