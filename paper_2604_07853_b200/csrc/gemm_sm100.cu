@@ -75,6 +75,7 @@ struct GemmParams {
   int E;
   int n_tiles;             // column tiles per expert
   int I;                   // gate_up: intermediate size (N = 2I)
+  int early_prefetch;      // decode-sized calls: weight tiles to pull into L2 before the predecessor finishes
   uint16_t* out_bf16;
   float* out_f32;
   uint8_t* h_codes;
@@ -206,7 +207,31 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     tmem_alloc(&s->tmem_addr, kTmemCols);
     tmem_relinquish();
   }
-  pdl_wait();  // everything above touched no global memory; from here on the predecessor's results are needed
+  if (warp == kTmaWarp && lane == 0 && p.early_prefetch > 0) {
+    // Decode-sized calls are bound by streaming the weights from HBM, and the kernels before
+    // this one in the stream (permute, activation quantization) leave the memory system idle.
+    // The weights do not depend on them, so pull this CTA's first weight tiles into L2 now.
+    // Tile T is guessed as (expert T / n_tiles, column tile T % n_tiles), exact when every
+    // expert has one row tile; a wrong guess only costs an unused L2 fill.
+    for (int t = 0; t < p.early_prefetch; ++t) {
+      const int T = blockIdx.x + t * gridDim.x;
+      if (T >= p.E * p.n_tiles) break;
+      const int e = T / p.n_tiles, n_tile = T % p.n_tiles;
+      int row_lo, row_hi;
+      if (MODE == kModeGateUp) {
+        row_lo = e * p.N + n_tile * BNH;
+        row_hi = row_lo + p.I;
+      } else {
+        row_lo = e * p.N + n_tile * BN;
+        row_hi = row_lo + BNH;
+      }
+      for (int kb = 0; kb < p.kblocks; ++kb) {
+        tma_prefetch_2d(&tm_b, kb * BK, row_lo);
+        tma_prefetch_2d(&tm_b, kb * BK, row_hi);
+      }
+    }
+  }
+  pdl_wait();  // everything above read no data of the predecessor; from here on its results are needed
   for (int e = threadIdx.x; e <= p.E; e += kThreads)
     s->off[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.rows_total);
   __syncthreads();
@@ -667,6 +692,12 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
   p.pair_weights = a.pair_weights;
   p.status = L.d_status;
   p.wait_limit_ns = 2000000000ull;
+  // decode-sized call (at most one row tile per expert): see the early prefetch in the kernel
+  if (a.rows_total <= a.E * BM) {
+    const int64_t tile_bytes = static_cast<int64_t>(p.kblocks) * kBBytes;
+    const int64_t budget = 80ll << 20;  // stay well inside the 126 MB L2
+    p.early_prefetch = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(3, budget / (tile_bytes * L.sm_count))));
+  }
 #ifdef QARL_TRACE
   p.trace = g_trace ? g_trace + static_cast<size_t>(g_trace_launch++ & 1) * 148 * 16 : nullptr;
 #endif
