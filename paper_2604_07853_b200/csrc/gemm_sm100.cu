@@ -257,6 +257,16 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   tc_fence_after_sync();
   const uint32_t tmem_base = s->tmem_addr;
   const int total_tiles = s->prefix[p.E];
+  // Balance the static schedule: with W = ceil(tiles / CTAs) rounds, ceil(tiles / W) CTAs already
+  // finish in W rounds; using exactly that many keeps every round full (768 decode tiles: 128 CTAs
+  // x 6 instead of 148 CTAs of which 120 idle through the sixth round) and leaves the streaming
+  // bandwidth to the CTAs that still have work.  The CTAs beyond that count retire at once.
+  int num_ctas = gridDim.x;
+  if (total_tiles > 0) {
+    const int rounds = (total_tiles + num_ctas - 1) / num_ctas;
+    num_ctas = (total_tiles + rounds - 1) / rounds;
+  }
+  const int first_tile = static_cast<int>(blockIdx.x) < num_ctas ? static_cast<int>(blockIdx.x) : total_tiles;
   const int KB = p.kblocks;
   const int NB = p.N / BNH;  // weight scale block-rows per expert
 
@@ -282,7 +292,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             row_hi = row_lo + BNH;
           }
         };
-        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
+        for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
           const TileCoord c = decode_tile(s, T, cur_e);
           int row_lo, row_hi;
           b_rows(c, row_lo, row_hi);
@@ -315,7 +325,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         int stage = 0, ks = 0;
         uint32_t phase = 0, acc_phase = 0;
         bool ok = true;
-        for (int T = blockIdx.x; ok && T < total_tiles; T += gridDim.x) {
+        for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
           for (int kb = 0; kb < KB; ++kb) {
             {
               TRACE_T0();
@@ -348,7 +358,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     const int ew = warp - kPromoWarps;
     int cur_e = 0;
     uint32_t tile_iter = 0;
-    for (int T = blockIdx.x; T < total_tiles; T += gridDim.x, ++tile_iter) {
+    for (int T = first_tile; T < total_tiles; T += num_ctas, ++tile_iter) {
       const TileCoord c = decode_tile(s, T, cur_e);
       int my_pair = 0;  // down: destination (flat pair id) of the lane-th row this warp handles
       if (MODE == kModeDown) {
@@ -471,7 +481,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       hi_off = (nb_hi - nb_lo) * KB;
     };
 
-    int T = blockIdx.x;
+    int T = first_tile;
     if (T < total_tiles) {
       TileCoord c = decode_tile(s, T, cur_e);
       const float *sx_ptr, *sw_lo_ptr;
@@ -485,7 +495,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         // a warp whose 32 rows all lie past the group's end (ragged tails, decode-sized groups)
         // keeps the barrier protocol going but reads and accumulates nothing
         const bool warp_live = c.m0 + q * 32 < c.m_end;
-        const int Tn = T + gridDim.x;
+        const int Tn = T + num_ctas;
         const bool has_next = Tn < total_tiles;
         TileCoord cn = c;
         float w = 0.0f;  // down: the pair's combine weight (sorted order), used at the end of the tile
