@@ -21,6 +21,13 @@ extern "C" {
 int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H, float eps,
                          void* out_bf16, void* stream);
 
+/* Exercises the bounded-wait path every pipeline wait of the GEMM uses: one thread waits on an
+ * mbarrier that nothing ever arrives on, with a limit of `limit_ns` nanoseconds (clamped to
+ * [1 us, 100 ms]).  The wait gives up at the limit, records QARL_ERR_DEVICE_TIMEOUT in the
+ * context's status word and the kernel returns normally: the context stays usable and
+ * qarl_poll_device_status reports (and clears) the error.  Nothing traps, faults or hangs. */
+int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,7 +32,7 @@ EXPORTS = [
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
-HARNESS_EXPORTS = ["qarl_harness_rmsnorm"]
+HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine"]
 
@@ -99,6 +99,8 @@ def load() -> C.CDLL:
     L.qarl_linear_fwd_static.argtypes = [p, p, i64, i64, p, p, i64, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
     L.qarl_harness_rmsnorm.argtypes = [p, p, i64, i64, C.c_float, p, p]
+    L.qarl_harness_wait_selftest.restype = C.c_int
+    L.qarl_harness_wait_selftest.argtypes = [p, C.c_uint64, p]
     _lib = L
     return L
 
@@ -173,6 +175,10 @@ class Context:
         cnt = (C.c_int64 * n)()
         self._check(self.lib.qarl_profile_end(self.h, ms, cnt))
         return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
+
+    def harness_wait_selftest(self, limit_ns: int = 1_000_000):
+        """Launch the bounded-wait self test (a wait nothing satisfies); poll() then returns -7."""
+        self._check(self.lib.qarl_harness_wait_selftest(self.h, limit_ns, _stream()))
 
     def harness_rmsnorm(self, x: torch.Tensor, eps: float = 1e-6, out=None):
         """Row-invariant RMSNorm (weight 1) used by the alignment-stack test; not part of the API."""

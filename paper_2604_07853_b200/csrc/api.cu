@@ -388,4 +388,12 @@ int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, flo
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "rmsnorm");
 }
 
+int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx) return QARL_ERR_INVALID_ARG;
+  if (limit_ns < 1000) limit_ns = 1000;
+  if (limit_ns > 100000000ull) limit_ns = 100000000ull;
+  cudaError_t e = launch_wait_selftest(make_launch(ctx, stream), limit_ns);
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "wait_selftest");
+}
+
 }  // extern "C"

@@ -103,6 +103,7 @@ cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64
 cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
                            int64_t H, int64_t E, uint16_t* out);
 
+cudaError_t launch_wait_selftest(const Launch& L, unsigned long long limit_ns);
 cudaError_t launch_rmsnorm(const Launch& L, const uint16_t* x, int64_t M, int64_t H, float eps, uint16_t* out);
 
 enum GemmMode { kModeLinear = 0, kModeGateUp = 1, kModeDown = 2 };

@@ -2,6 +2,7 @@
 // between layers by the alignment-stack test.
 #include "common.cuh"
 #include "../../include/qarl_harness.h"
+#include "ptx_sm100.cuh"
 
 namespace qarl {
 namespace {
@@ -41,7 +42,23 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* __restrict
   }
 }
 
+// A wait that can never be satisfied, bounded like every wait in the GEMM pipeline.
+__global__ void wait_selftest_kernel(unsigned long long limit_ns, int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+    if (!ptx::mbar_wait_bounded(&bar, 0, limit_ns)) set_status(status, QARL_ERR_DEVICE_TIMEOUT);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_selftest(const Launch& L, unsigned long long limit_ns) {
+  wait_selftest_kernel<<<1, 32, 0, L.stream>>>(limit_ns, L.d_status);
+  ++*L.launches;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_rmsnorm(const Launch& L, const uint16_t* x, int64_t M, int64_t H, float eps, uint16_t* out) {
   if (M == 0) return cudaSuccess;
