@@ -151,7 +151,7 @@ def run_reference(args, rank: int):
     if rank != 0:
         return
     import oracle
-    n_tokens, n_exp = 16, 1
+    n_tokens, n_exp = 512, 8      # per step: about a second of oracle work on 8-16 cores
     st = cpu_state(4, n_tokens)
     for _ in range(args.warmup):
         cpu_reference_step(st, n_tokens, n_exp)
