@@ -49,6 +49,14 @@ def lib() -> C.CDLL:
         L.oracle_combine.argtypes = [p, p, p, i64, i64, i64, p]
         L.oracle_moe.restype = C.c_int
         L.oracle_moe.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p]
+        L.oracle_quantize_weight_w4.restype = C.c_int
+        L.oracle_quantize_weight_w4.argtypes = [p, i64, i64, i64, p, p, p]
+        L.oracle_dequant_w4.restype = None
+        L.oracle_dequant_w4.argtypes = [p, p, p, i64, i64, p]
+        L.oracle_linear_bf16.restype = None
+        L.oracle_linear_bf16.argtypes = [p, i64, i64, p, i64, p, p]
+        L.oracle_moe_w4a16.restype = C.c_int
+        L.oracle_moe_w4a16.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
     return _lib
@@ -201,6 +209,65 @@ def moe(x_bits, ids, wts, w13c, w13s, w2c, w2s, dumps: bool = False):
                           _ptr(w13c), _ptr(w13s), _ptr(w2c), _ptr(w2s), _ptr(out),
                           _ptr(d.get("gate_up")), _ptr(d.get("h")), _ptr(d.get("h_codes")),
                           _ptr(d.get("h_scales")), _ptr(d.get("y32")))
+    if rc:
+        raise OracleError(rc)
+    return (out, d) if dumps else out
+
+
+# ---------------------------------------------------------------------------- W4A16
+def quantize_weight_w4(w_bits: np.ndarray):
+    """w bf16 bits [E, N, K] or [N, K] -> (packed u8 [.., N, K/2], scales f32 [.., N, K/128],
+    zeros u8 [.., N, K/128]); unsigned 4-bit codes, one (s, z) per 128 K-elements of a row."""
+    w = _c(w_bits, np.uint16)
+    squeeze = w.ndim == 2
+    if squeeze:
+        w = w[None]
+    E, N, K = w.shape
+    packed = np.empty((E, N, K // 2), dtype=np.uint8)
+    scales = np.empty((E, N, K // 128), dtype=np.float32)
+    zeros = np.empty((E, N, K // 128), dtype=np.uint8)
+    rc = lib().oracle_quantize_weight_w4(_ptr(w), E, N, K, _ptr(packed), _ptr(scales), _ptr(zeros))
+    if rc:
+        raise OracleError(rc)
+    return (packed[0], scales[0], zeros[0]) if squeeze else (packed, scales, zeros)
+
+
+def dequant_w4(packed, scales, zeros) -> np.ndarray:
+    """-> w^ bf16 bits, same leading shape, last dim K."""
+    packed, scales, zeros = _c(packed, np.uint8), _c(scales, np.float32), _c(zeros, np.uint8)
+    K = packed.shape[-1] * 2
+    rows = int(np.prod(packed.shape[:-1]))
+    out = np.empty((*packed.shape[:-1], K), dtype=np.uint16)
+    lib().oracle_dequant_w4(_ptr(packed), _ptr(scales), _ptr(zeros), rows, K, _ptr(out))
+    return out
+
+
+def linear_bf16(x_bits, w_hat_bits):
+    """y = x . w^T on bf16 operands -> (y fp32 [M, N], y bf16 bits)."""
+    x, w = _c(x_bits, np.uint16), _c(w_hat_bits, np.uint16)
+    M, K = x.shape
+    N = w.shape[0]
+    y32 = np.empty((M, N), dtype=np.float32)
+    y16 = np.empty((M, N), dtype=np.uint16)
+    lib().oracle_linear_bf16(_ptr(x), M, K, _ptr(w), N, _ptr(y32), _ptr(y16))
+    return y32, y16
+
+
+def moe_w4a16(x_bits, ids, wts, w13_hat, w2_hat, dumps: bool = False):
+    x, ids, wts = _c(x_bits, np.uint16), _c(ids, np.int32), _c(wts, np.float32)
+    w13_hat, w2_hat = _c(w13_hat, np.uint16), _c(w2_hat, np.uint16)
+    M, H = x.shape
+    k = ids.shape[1]
+    E, I2, _ = w13_hat.shape
+    I = I2 // 2
+    P = M * k
+    out = np.empty((M, H), dtype=np.uint16)
+    d = {}
+    if dumps:
+        d = dict(gate_up=np.empty((P, 2 * I), np.uint16), h=np.empty((P, I), np.uint16),
+                 y32=np.empty((P, H), np.float32))
+    rc = lib().oracle_moe_w4a16(_ptr(x), _ptr(ids), _ptr(wts), M, H, I, E, k, _ptr(w13_hat), _ptr(w2_hat),
+                                _ptr(out), _ptr(d.get("gate_up")), _ptr(d.get("h")), _ptr(d.get("y32")))
     if rc:
         raise OracleError(rc)
     return (out, d) if dumps else out

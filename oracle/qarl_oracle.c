@@ -406,6 +406,123 @@ int oracle_moe(const uint16_t *x, const int32_t *ids, const float *wts,
     return 0;
 }
 
+/* =======================================================================================
+ * W4A16: 4-bit integer weight-only quantization (Sec. 2.2, "Integer quantization"), the format
+ * the paper's headline results use (Sec. 3.1 item 1: W4A16 for larger MoE models).
+ *   Quant:   W_q = clamp( round(W / s) + z, q_min, q_max ),   Dequant:  W^ = s (W_q - z)
+ * Readings where the paper is silent: unsigned 4-bit codes (q_min = 0, q_max = 15); one
+ * (s, z) per group of 128 consecutive K elements of one weight row; asymmetric min/max
+ * calibration with zero kept representable: lo = min(0, min W), hi = max(0, max W),
+ * s = fl(max(hi - lo, 2^-40) / 15), z = clamp(rint(-lo / s), 0, 15); round() is round to
+ * nearest, ties to even; W / s is an IEEE fp32 division.  The GEMM consumes the dequantized
+ * weight rounded to bf16, w^ = bf16( fl(s * (W_q - z)) ), with bf16 activations ("A16") and
+ * higher-precision (fp32) accumulation.
+ * Packed layout: byte j of a row holds code 2j in its low nibble and code 2j+1 in its high nibble.
+ * ===================================================================================== */
+int oracle_quantize_weight_w4(const uint16_t *w, int64_t E, int64_t N, int64_t K,
+                              uint8_t *packed, float *scales, uint8_t *zeros) {
+    if (K % QBLOCK) return -2;
+    int64_t kb = K / QBLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < E * N; ++r)
+        for (int64_t g = 0; g < kb; ++g) {
+            const uint16_t *base = w + r * K + g * QBLOCK;
+            float lo = 0.0f, hi = 0.0f;
+            for (int c = 0; c < QBLOCK; ++c) {
+                float v = bf16_to_f32(base[c]);
+                if (v < lo) lo = v;
+                if (v > hi) hi = v;
+            }
+            float range = hi - lo;
+            if (range < AMAX_FLOOR) range = AMAX_FLOOR;
+            float s = range / 15.0f;
+            float zf = nearbyintf(-lo / s);
+            if (zf < 0.0f) zf = 0.0f;
+            if (zf > 15.0f) zf = 15.0f;
+            scales[r * kb + g] = s;
+            zeros[r * kb + g] = (uint8_t)zf;
+            for (int c = 0; c < QBLOCK; c += 2) {
+                int q[2];
+                for (int t = 0; t < 2; ++t) {
+                    float v = nearbyintf(bf16_to_f32(base[c + t]) / s) + zf;
+                    if (v < 0.0f) v = 0.0f;
+                    if (v > 15.0f) v = 15.0f;
+                    q[t] = (int)v;
+                }
+                packed[r * (K / 2) + (g * QBLOCK + c) / 2] = (uint8_t)(q[0] | (q[1] << 4));
+            }
+        }
+    return 0;
+}
+
+/* w^ bf16 bits [rows, K] from packed codes, scales and zeros (rows = E*N). */
+void oracle_dequant_w4(const uint8_t *packed, const float *scales, const uint8_t *zeros,
+                       int64_t rows, int64_t K, uint16_t *w_hat) {
+    int64_t kb = K / QBLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t b = packed[r * (K / 2) + k / 2];
+            int q = (k & 1) ? (b >> 4) : (b & 15);
+            float s = scales[r * kb + k / QBLOCK];
+            int z = zeros[r * kb + k / QBLOCK];
+            w_hat[r * K + k] = oracle_bf16_rne(s * (float)(q - z));
+        }
+}
+
+/* y[m,n] = sum_k x[m,k] * w^[n,k]: bf16 operands, products and sum exact in double (each
+ * product has <= 16 significant bits), rounded once to fp32, then to bf16.  The paper asks
+ * only for "higher precision" accumulation; the GPU's tensor-core order is compared with this
+ * ideal within the stated tolerance. */
+void oracle_linear_bf16(const uint16_t *x, int64_t M, int64_t K, const uint16_t *w_hat, int64_t N,
+                        float *y32, uint16_t *y16) {
+    float *wf = (float *)malloc((size_t)N * K * sizeof(float));
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N * K; ++i) wf[i] = bf16_to_f32(w_hat[i]);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k)
+                acc += (double)bf16_to_f32(x[m * K + k]) * (double)wf[n * K + k];
+            float a = (float)acc;
+            if (y32) y32[m * N + n] = a;
+            if (y16) y16[m * N + n] = oracle_bf16_rne(a);
+        }
+    free(wf);
+}
+
+/* One routed MoE FFN layer with W4A16 weights: activations stay bf16 between the GEMMs.
+ *   gate_up[p] = bf16( x[t] . W13^_e ),  h[p] = swiglu(gate_up[p]),  y32[p] = h[p] . W2^_e (fp32),
+ *   out[t] = combine (same rule as the FP8 layer).  w13_hat [E, 2I, H], w2_hat [E, H, I] bf16. */
+int oracle_moe_w4a16(const uint16_t *x, const int32_t *ids, const float *wts,
+                     int64_t M, int64_t H, int64_t I, int64_t E, int64_t k,
+                     const uint16_t *w13_hat, const uint16_t *w2_hat, uint16_t *out,
+                     uint16_t *d_gate_up, uint16_t *d_h, float *d_y32) {
+    if (k > 64) return -2;
+    int64_t P = M * k;
+    for (int64_t p = 0; p < P; ++p)
+        if (ids[p] < 0 || ids[p] >= E) return -8;
+    size_t Pn = (size_t)(P > 0 ? P : 1);
+    uint16_t *gate_up = d_gate_up ? d_gate_up : (uint16_t *)malloc(Pn * 2 * I * sizeof(uint16_t));
+    uint16_t *h = d_h ? d_h : (uint16_t *)malloc(Pn * I * sizeof(uint16_t));
+    float *y32 = d_y32 ? d_y32 : (float *)malloc(Pn * H * sizeof(float));
+    for (int64_t p = 0; p < P; ++p) {
+        int64_t t = p / k, e = ids[p];
+        oracle_linear_bf16(x + t * H, 1, H, w13_hat + e * 2 * I * H, 2 * I, NULL, gate_up + p * 2 * I);
+    }
+    oracle_swiglu(gate_up, P, I, h);
+    for (int64_t p = 0; p < P; ++p) {
+        int64_t e = ids[p];
+        oracle_linear_bf16(h + p * I, 1, I, w2_hat + e * H * I, H, y32 + p * H, NULL);
+    }
+    oracle_combine(y32, ids, wts, M, k, H, out);
+    if (!d_gate_up) free(gate_up);
+    if (!d_h) free(h);
+    if (!d_y32) free(y32);
+    return 0;
+}
+
 /* Number of OpenMP threads the oracle will use (reported beside its timing). */
 #ifdef _OPENMP
 #include <omp.h>
