@@ -413,10 +413,13 @@ int oracle_moe(const uint16_t *x, const int32_t *ids, const float *wts,
  * Readings where the paper is silent: unsigned 4-bit codes (q_min = 0, q_max = 15); one
  * (s, z) per group of 128 consecutive K elements of one weight row; asymmetric min/max
  * calibration with zero kept representable: lo = min(0, min W), hi = max(0, max W),
- * s = fl(max(hi - lo, 2^-40) / 15), z = clamp(rint(-lo / s), 0, 15); round() is round to
- * nearest, ties to even; W / s is an IEEE fp32 division.  The GEMM consumes the dequantized
- * weight rounded to bf16, w^ = bf16( fl(s * (W_q - z)) ), with bf16 activations ("A16") and
- * higher-precision (fp32) accumulation.
+ * s = bf16( fl(max(hi - lo, 2^-40) / 15) ) -- the group scale is kept in the model's 16-bit type,
+ * as W4A16 checkpoints store it, and is returned here as the fp32 of that bf16 value --
+ * z = clamp(rint(-lo / s), 0, 15); round() is round to nearest, ties to even; W / s and -lo / s
+ * are IEEE fp32 divisions by that stored s.  The GEMM consumes the dequantized weight rounded
+ * to bf16, w^ = bf16( s * (W_q - z) ): s has 8 significant bits and |W_q - z| <= 15, so the
+ * product is exact before its one rounding.  Activations stay bf16 ("A16"), accumulation is
+ * higher precision (fp32).
  * Packed layout: byte j of a row holds code 2j in its low nibble and code 2j+1 in its high nibble.
  * ===================================================================================== */
 int oracle_quantize_weight_w4(const uint16_t *w, int64_t E, int64_t N, int64_t K,
@@ -435,7 +438,7 @@ int oracle_quantize_weight_w4(const uint16_t *w, int64_t E, int64_t N, int64_t K
             }
             float range = hi - lo;
             if (range < AMAX_FLOOR) range = AMAX_FLOOR;
-            float s = range / 15.0f;
+            float s = bf16_to_f32(oracle_bf16_rne(range / 15.0f));
             float zf = nearbyintf(-lo / s);
             if (zf < 0.0f) zf = 0.0f;
             if (zf > 15.0f) zf = 15.0f;

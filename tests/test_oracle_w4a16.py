@@ -12,6 +12,13 @@ def _unpack(packed):
     return np.stack([lo, hi], axis=-1).reshape(*packed.shape[:-1], packed.shape[-1] * 2)
 
 
+def _bf16_round(a):
+    """fp32 -> nearest bf16 (ties to even), by integer arithmetic on the bit pattern."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
 def test_hand_worked_group_follows_the_paper_formula():
     """Values k/4 for k = -8..7 repeated: lo = -2, hi = 1.75, s = 3.75/15 = 0.25, z = round(2/0.25) = 8,
     W_q = W/s + 8 = 0..15 exactly and s (W_q - z) reproduces W exactly."""
@@ -34,6 +41,7 @@ def test_codes_scales_zeros_vs_independent_numpy():
     lo = np.minimum(wf.min(axis=3), 0).astype(np.float32)
     hi = np.maximum(wf.max(axis=3), 0).astype(np.float32)
     s_ref = (np.maximum(hi - lo, np.float32(2.0 ** -40)) / np.float32(15)).astype(np.float32)
+    s_ref = _bf16_round(s_ref)                                     # the scale is stored as bf16
     z_ref = np.clip(np.rint((-lo / s_ref).astype(np.float32)), 0, 15)
     assert np.array_equal(s, s_ref) and np.array_equal(z, z_ref.astype(np.uint8))
     q_ref = np.clip(np.rint((wf / s_ref[..., None]).astype(np.float32)) + z_ref[..., None], 0, 15)
@@ -53,10 +61,16 @@ def test_round_trip_bound_and_exact_zero():
     wf = inputs.bf16_bits_to_f32(w).astype(np.float64)
     what = inputs.bf16_bits_to_f32(oracle.dequant_w4(p, s, z)).astype(np.float64)
     se = np.repeat(s, 128, axis=1).astype(np.float64)
+    q = _unpack(p).astype(np.int64)
+    inner = (q > 0) & (q < 15)                                     # codes that were not clamped
     # half a step from rounding, plus the bf16 rounding of the dequantized value
-    assert (np.abs(wf - what) <= 0.5 * se * (1 + 1e-5) + np.abs(what) * 2.0 ** -8).all()
+    bound = 0.5 * se * (1 + 1e-5) + np.abs(what) * 2.0 ** -8
+    assert (np.abs(wf - what)[inner] <= bound[inner]).all()
+    # clamped codes: the rounded zero point and the bf16-rounded scale add at most one more step
+    assert (np.abs(wf - what) <= bound + se * (0.5 + 16 * 2.0 ** -8)).all()
     assert (what[wf == 0] == 0).all()                              # zero is representable (code z)
-    assert np.isfinite(s).all() and s[5, 0] == np.float32(2.0 ** -40) / np.float32(15)
+    assert np.array_equal(s, _bf16_round(s))                       # scales are bf16 values
+    assert np.isfinite(s).all() and s[5, 0] == _bf16_round(np.float32(2.0 ** -40) / np.float32(15))
 
 
 def test_dequant_is_bf16_of_one_fp32_product():
