@@ -161,6 +161,58 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
                  void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
                  void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * W4A16: 4-bit integer weight-only quantization with bf16 activations (Sec. 2.2, integer
+ * quantization: W_q = clamp(round(W/s) + z, q_min, q_max), W^ = s (W_q - z); Sec. 3.1 item 1
+ * names W4A16 as the format of the larger MoE models).  Choices the paper leaves open, fixed
+ * here: unsigned codes 0..15; one (s, z) per 128 consecutive K elements of one weight row;
+ * lo = min(0, min W), hi = max(0, max W); s = bf16(max(hi - lo, 2^-40) / 15);
+ * z = clamp(rint(-lo / s), 0, 15); round = nearest, ties to even; the GEMM multiplies bf16
+ * activations by w^ = bf16(s * (W_q - z)) and accumulates in fp32 in ascending k.
+ *
+ * Storage (all device pointers):
+ *   packed  u8  [E, N, K/2]   every aligned 32-bit word holds eight consecutive codes e0..e7
+ *                             of a row, nibble by nibble from the low end in the order
+ *                             e0 e2 e4 e6 e1 e3 e5 e7 (so bits [4j, 4j+4) and [16+4j, 20+4j)
+ *                             hold the adjacent pair e_2j, e_2j+1);
+ *   scales  bf16 [E, K/128, N]  group-major: the scales of one K-group for all rows of an
+ *                             expert are contiguous;
+ *   zeros   u8  [E, K/128, N]  same layout.
+ * ------------------------------------------------------------------------------------- */
+
+/* in : w_bf16 [E, N, K], 16-byte aligned, K % 128 == 0.  out: packed (16-byte aligned),
+ * scales (2-byte aligned), zeros, as above; caller-owned.  One kernel, every input byte read once. */
+int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
+                            uint8_t* packed, void* scales_bf16, uint8_t* zeros, void* stream);
+
+/* y[m, n] = bf16( sum_k x[m,k] * w^[n,k] ), fp32 accumulation (Sec. 2.2 Dequant applied inside
+ * the GEMM).  in: x_bf16 [M, K] 16-byte aligned; weights as produced by qarl_quantize_weight_w4
+ * with E = 1;  N % 128 == 0, K % 128 == 0.  out: y_bf16 [M, N]; y_f32 [M, N] optional (NULL:
+ * skipped) dump of the fp32 accumulator.  Needs no workspace.  Row m of y depends only on row m
+ * of x and on the weights (App. C): bitwise the same for any M. */
+int qarl_linear_fwd_w4a16(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t K,
+                          const uint8_t* w_packed, const void* w_scales_bf16,
+                          const uint8_t* w_zeros, int64_t N, void* y_bf16, float* y_f32,
+                          void* stream);
+
+/* The routed-expert FFN layer of qarl_moe_fwd on W4A16 weights; activations stay bf16:
+ *   gu = bf16(x[t] . W13^_e);  h = bf16(silu(gu[:I]) * gu[I:]);  y = h . W2^_e (fp32);
+ *   c_j = bf16(topk_weights[t,j] * y);  out[t] = bf16(sum of float(c_j) in ascending expert id).
+ * w13: [E, 2I, H] quantized along H (rows 0..I-1 gate, I..2I-1 up); w2: [E, H, I] quantized
+ * along I.  Limits: H % 256 == 0, I % 128 == 0, 1 <= k <= 32, 1 <= E <= 1024, M*k < 2^31.
+ * dbg: expert_offsets, sorted_pair, gate_up_bf16, h_bf16 and down_f32 are filled when non-NULL;
+ * h_codes and h_scales are not used.  workspace: at least
+ * qarl_moe_w4a16_workspace_bytes(M, H, I, E, k) bytes, 256-byte aligned; calls sharing a
+ * workspace must not overlap.  Errors as qarl_moe_fwd. */
+size_t qarl_moe_w4a16_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k);
+int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
+                       const float* topk_weights, int64_t M, int64_t H, int64_t I, int64_t E,
+                       int64_t k, const uint8_t* w13_packed, const void* w13_scales_bf16,
+                       const uint8_t* w13_zeros, const uint8_t* w2_packed,
+                       const void* w2_scales_bf16, const uint8_t* w2_zeros, void* out_bf16,
+                       void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
+                       void* stream);
+
 /* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
  * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
  * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;
@@ -170,7 +222,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
  * and destroys the events. */
 enum {
   QARL_STAGE_QUANT_WEIGHT = 0,
-  QARL_STAGE_QUANT_ACT = 1,
+  QARL_STAGE_QUANT_ACT = 1,   /* W4A16 MoE: the copy of the bf16 rows into expert-sorted order */
   QARL_STAGE_LINEAR_GEMM = 2,
   QARL_STAGE_PERMUTE = 3,
   QARL_STAGE_GATE_UP_GEMM = 4,

@@ -9,34 +9,11 @@
 #include "common.cuh"
 #include "../../include/qarl_harness.h"
 
+#include "api_util.cuh"
+
 namespace {
 
 using namespace qarl;
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
-int cuda_fail(qarl_ctx* ctx, cudaError_t e, const char* where) {
-  snprintf(ctx->err, sizeof(ctx->err), "%s: %s", where, cudaGetErrorString(e));
-  return QARL_ERR_CUDA;
-}
-
-Launch make_launch(qarl_ctx* ctx, void* stream) {
-  Launch L;
-  L.stream = static_cast<cudaStream_t>(stream);
-  L.device = ctx->device;
-  L.sm_count = ctx->sm_count;
-  L.d_status = ctx->d_status;
-  L.launches = &ctx->launches;
-  return L;
-}
-
-// Record a timing mark on the stream if stage timing is on and events are left.
-void mark(qarl_ctx* ctx, cudaStream_t st, int stage) {
-  if (ctx->marks_used >= ctx->marks.size()) return;
-  if (cudaEventRecord(ctx->marks[ctx->marks_used], st) != cudaSuccess) return;
-  ctx->mark_stage[ctx->marks_used++] = stage;
-}
 
 int run_gemm(qarl_ctx* ctx, const Launch& L, const GemmArgs& a) {
   CUresult cu = CUDA_SUCCESS;

@@ -1,0 +1,191 @@
+// C ABI entry points of the W4A16 path (4-bit group-quantized weights, bf16 activations):
+// argument checks, workspace planning, kernel sequencing.  No device memory is allocated here.
+#include "api_util.cuh"
+
+namespace {
+
+using namespace qarl;
+
+int run_gemm_w4(qarl_ctx* ctx, const Launch& L, const GemmW4Args& a) {
+  CUresult cu = CUDA_SUCCESS;
+  cudaError_t e = launch_gemm_w4a16(L, ctx->encode, a, &cu);
+  if (cu != CUDA_SUCCESS) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+    return QARL_ERR_CUDA;
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "w4a16 gemm launch");
+  return QARL_OK;
+}
+
+// Workspace carve-up of qarl_moe_fwd_w4a16; every slice starts on a 256-byte boundary.
+struct MoeW4Plan {
+  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, x_sorted, h, contrib, total;
+};
+MoeW4Plan plan_moe_w4(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
+  const size_t P = static_cast<size_t>(M * k);
+  MoeW4Plan p{};
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = o;
+    o = align_up(o + bytes, 256);
+    return at;
+  };
+  p.chunk_hist = take(static_cast<size_t>(permute_num_chunks(M * k)) * E * sizeof(int32_t));
+  p.offsets = take((E + 1) * sizeof(int32_t));
+  p.sorted_pair = take(P * sizeof(int32_t));
+  p.pos_of_pair = take(P * sizeof(int32_t));
+  p.sorted_w = take(P * sizeof(float));
+  p.x_sorted = take(P * H * sizeof(uint16_t));
+  p.h = take(P * I * sizeof(uint16_t));
+  p.contrib = take(P * H * sizeof(uint16_t));
+  p.total = o;
+  return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                            void* scales, uint8_t* zeros, void* stream) {
+  if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
+  if (K % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (E * N * (K / kBlock) > (0x7FFFFFFFll << 5)) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (E == 0 || N == 0 || K == 0) return QARL_OK;
+  if (!w || !packed || !scales || !zeros) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(w) || !aligned16(packed) || (reinterpret_cast<uintptr_t>(scales) & 1u)) return QARL_ERR_MISALIGNED;
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
+  cudaError_t e = launch_quantize_weight_w4(make_launch(ctx, stream), static_cast<const uint16_t*>(w), E, N, K, packed,
+                                            static_cast<uint16_t*>(scales), zeros);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_WEIGHT);
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_weight_w4");
+}
+
+int qarl_linear_fwd_w4a16(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wp, const void* ws,
+                          const uint8_t* wz, int64_t N, void* y, float* y_f32, void* stream) {
+  if (!ctx || M < 0 || K <= 0 || N <= 0) return QARL_ERR_INVALID_ARG;
+  if (N % kBlock || K % kBlock || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (M == 0) return QARL_OK;
+  if (!x || !wp || !ws || !wz || !y) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(wp) || !aligned16(y) || !aligned16(y_f32) ||
+      (reinterpret_cast<uintptr_t>(ws) & 1u))
+    return QARL_ERR_MISALIGNED;
+  GemmW4Args a{};
+  a.mode = kModeLinear;
+  a.a_bf16 = static_cast<const uint16_t*>(x);
+  a.rows_total = M;
+  a.K = K;
+  a.b_packed = wp;
+  a.b_scales = static_cast<const uint16_t*>(ws);
+  a.b_zeros = wz;
+  a.N = N;
+  a.E = 1;
+  a.out_bf16 = static_cast<uint16_t*>(y);
+  a.out_f32 = y_f32;
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
+  const int rc = run_gemm_w4(ctx, make_launch(ctx, stream), a);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_LINEAR_GEMM);
+  return rc;
+}
+
+size_t qarl_moe_w4a16_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
+  if (M <= 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0) return 0;
+  return plan_moe_w4(M, H, I, E, k).total;
+}
+
+int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
+                       int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w13z,
+                       const uint8_t* w2p, const void* w2s, const uint8_t* w2z, void* out, void* workspace,
+                       size_t workspace_bytes, const qarl_moe_debug* dbg, void* stream) {
+  if (!ctx || M < 0 || H <= 0 || I <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
+  // the down tile spans 256 adjacent weight rows of one expert
+  if (H % 256 || I % kBlock || E > 1024 || M * k >= 0x7FFFFF00ll || E * 2 * I > 0x7FFFFF00ll)
+    return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (M == 0) return QARL_OK;
+  if (!x || !ids || !wts || !w13p || !w13s || !w13z || !w2p || !w2s || !w2z || !out || !workspace)
+    return QARL_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(w13p) || !aligned16(w2p) || !aligned16(out) ||
+      (reinterpret_cast<uintptr_t>(w13s) & 1u) || (reinterpret_cast<uintptr_t>(w2s) & 1u) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return QARL_ERR_MISALIGNED;
+  const MoeW4Plan pl = plan_moe_w4(M, H, I, E, k);
+  if (workspace_bytes < pl.total) return QARL_ERR_WORKSPACE_TOO_SMALL;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const int64_t P = M * k;
+  Launch L = make_launch(ctx, stream);
+  cudaError_t e;
+
+  PermuteBuffers pb;
+  pb.chunk_hist = reinterpret_cast<int32_t*>(ws + pl.chunk_hist);
+  pb.offsets = reinterpret_cast<int32_t*>(ws + pl.offsets);
+  pb.sorted_pair = reinterpret_cast<int32_t*>(ws + pl.sorted_pair);
+  pb.pos_of_pair = reinterpret_cast<int32_t*>(ws + pl.pos_of_pair);
+  mark(ctx, L.stream, -1);
+  if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
+  mark(ctx, L.stream, QARL_STAGE_PERMUTE);
+
+  uint16_t* x_sorted = reinterpret_cast<uint16_t*>(ws + pl.x_sorted);
+  float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
+  if ((e = launch_scatter_rows(L, static_cast<const uint16_t*>(x), M, H, x_sorted, pb.pos_of_pair,
+                               static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
+    return cuda_fail(ctx, e, "scatter_rows");
+  mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
+
+  uint16_t* h = reinterpret_cast<uint16_t*>(ws + pl.h);
+  GemmW4Args g{};
+  g.mode = kModeGateUp;
+  g.a_bf16 = x_sorted;
+  g.rows_total = P;
+  g.K = H;
+  g.b_packed = w13p;
+  g.b_scales = static_cast<const uint16_t*>(w13s);
+  g.b_zeros = w13z;
+  g.N = 2 * I;
+  g.E = E;
+  g.offsets = pb.offsets;
+  g.out_bf16 = dbg ? static_cast<uint16_t*>(dbg->gate_up_bf16) : nullptr;
+  g.h_bf16 = h;
+  int rc = run_gemm_w4(ctx, L, g);
+  if (rc != QARL_OK) return rc;
+  mark(ctx, L.stream, QARL_STAGE_GATE_UP_GEMM);
+
+  uint16_t* contrib = reinterpret_cast<uint16_t*>(ws + pl.contrib);
+  GemmW4Args d{};
+  d.mode = kModeDown;
+  d.a_bf16 = h;
+  d.rows_total = P;
+  d.K = I;
+  d.b_packed = w2p;
+  d.b_scales = static_cast<const uint16_t*>(w2s);
+  d.b_zeros = w2z;
+  d.N = H;
+  d.E = E;
+  d.offsets = pb.offsets;
+  d.out_bf16 = contrib;
+  d.out_f32 = dbg ? dbg->down_f32 : nullptr;
+  d.sorted_pair = pb.sorted_pair;
+  d.pair_weights = sorted_w;
+  rc = run_gemm_w4(ctx, L, d);
+  if (rc != QARL_OK) return rc;
+  mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);
+
+  if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out))) != cudaSuccess)
+    return cuda_fail(ctx, e, "combine");
+  mark(ctx, L.stream, QARL_STAGE_COMBINE);
+
+  if (dbg) {
+    if (dbg->expert_offsets &&
+        (e = cudaMemcpyAsync(dbg->expert_offsets, pb.offsets, (E + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice,
+                             L.stream)) != cudaSuccess)
+      return cuda_fail(ctx, e, "copy offsets");
+    if (dbg->sorted_pair && (e = cudaMemcpyAsync(dbg->sorted_pair, pb.sorted_pair, P * sizeof(int32_t),
+                                                 cudaMemcpyDeviceToDevice, L.stream)) != cudaSuccess)
+      return cuda_fail(ctx, e, "copy sorted_pair");
+    if (dbg->h_bf16 && (e = cudaMemcpyAsync(dbg->h_bf16, h, static_cast<size_t>(P) * I * sizeof(uint16_t),
+                                            cudaMemcpyDeviceToDevice, L.stream)) != cudaSuccess)
+      return cuda_fail(ctx, e, "copy h");
+  }
+  return QARL_OK;
+}
+
+}  // extern "C"

@@ -138,6 +138,32 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // Returns cudaSuccess, or an error; *cu_err receives a driver error from tensor-map encoding.
 cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
 
+// ---- W4A16 (4-bit group-quantized weights, bf16 activations) --------------------------------
+cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
+                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros);
+// bf16 row t of x [M, H] -> rows dst_rows[t*fanout + j] of out; pair weights scattered alongside.
+cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,
+                                const int32_t* dst_rows, int fanout, const float* pair_w, float* sorted_w);
+
+struct GemmW4Args {
+  GemmMode mode;
+  const uint16_t* a_bf16;   // [rows_total, K]
+  int64_t rows_total;
+  int64_t K;
+  const uint8_t* b_packed;  // [E, N, K/2]
+  const uint16_t* b_scales; // bf16 bits [E, K/128, N]
+  const uint8_t* b_zeros;   // [E, K/128, N]
+  int64_t N;
+  int64_t E;
+  const int32_t* offsets;   // row groups per expert, or nullptr (dense)
+  uint16_t* out_bf16;       // linear: y [M, N]; gate_up (debug): gate_up [P, 2I]; down: contrib [P, H] by pair id
+  float* out_f32;           // optional fp32 accumulator dump (linear: [M, N]; down: [P, H] sorted order)
+  uint16_t* h_bf16;         // gate_up: h [P, I]
+  const int32_t* sorted_pair;
+  const float* pair_weights;
+};
+cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err);
+
 }  // namespace qarl
 
 // The opaque context of the C ABI (one per device).

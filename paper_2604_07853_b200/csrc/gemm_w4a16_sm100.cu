@@ -1,0 +1,502 @@
+// Persistent W4A16 GEMM for sm_100a (dense projection, MoE gate_up, MoE down): bf16 activations
+// times 4-bit group-quantized weights (Sec. 2.2, integer quantization; the format of the
+// paper's larger MoE models, Sec. 3.1).
+//
+//   y[m,n] = sum_k x[m,k] * w^[n,k],   w^ = bf16( s * (W_q - z) )   (Dequant of Sec. 2.2)
+//
+// with one (s, z) per 128 K-elements of a weight row, s a bf16 value.  The weights cross HBM
+// and L2 as 4-bit codes only; they are expanded to bf16 in shared memory, next to the tensor
+// core, and the whole K reduction of a tile accumulates in TMEM (fp32) in ascending k, one MMA
+// shape, no split-K: a row's result depends on that row and the weight tile only, never on the
+// batch around it (App. C).
+//
+// A tile is 128 rows x (128 + 128) columns, as in the FP8 kernel: the two halves are adjacent
+// weight rows for linear/down, gate rows and the matching up rows for gate_up (SwiGLU in the
+// epilogue).  One K-step is 64 elements = one 128-byte swizzle span of bf16.
+//
+// Structure of a CTA (512 threads, one CTA per SM, persistent, static tile list):
+//   warp 12     TMA producer: per K-step the A box (128 rows x 64 bf16, SWIZZLE_128B) and two
+//               boxes of packed codes (128 weight rows x 32 bytes) into a ring of load stages;
+//   warps 4-11  dequantization: thread n owns weight row n of the tile; it reads its 32 bytes
+//               of codes, forms pairs (w >> 4j) & 0x000F000F | 0x43004300 = bf16x2 (128 + q),
+//               subtracts 128 + z (exact), multiplies by s (one rounding: the bf16 of the exact
+//               product), and writes the 128-byte row of the bf16 B tile in the 128-byte swizzle
+//               the tensor core expects; a proxy fence, then the warp arrives on the stage;
+//   warp 13     MMA issuer: 4 x tcgen05.mma kind::f16 (128 x 256 x 16) per K-step into one of
+//               two 256-column TMEM accumulators; tcgen05.commit frees the stages, and after
+//               the last K-step publishes the accumulator;
+//   warps 0-3   epilogue: TMEM -> registers -> bf16 output (linear), SwiGLU -> h (gate_up),
+//               weight * y -> contribution by pair id (down), while the next tile's main loop
+//               runs on the other accumulator.
+//
+// Every wait on an mbarrier is bounded; on expiry the thread records QARL_ERR_DEVICE_TIMEOUT,
+// raises a CTA-wide abort flag that all other waits poll, and the CTA drains and frees its TMEM.
+#include <algorithm>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+#include "sched.cuh"
+
+namespace qarl {
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;            // rows per tile (UMMA M)
+constexpr int BNH = 128;           // columns per half tile
+constexpr int BN = 2 * BNH;        // UMMA N
+constexpr int BK = 64;             // bf16 elements per K-step (128 bytes)
+constexpr int kLoadStages = 4;     // A + packed codes
+constexpr int kDqStages = 3;       // dequantized B tiles
+constexpr int kAccBufs = 2;
+constexpr int kEpiWarps = 4;       // warps 0-3 (TMEM quadrant = warp index)
+constexpr int kDqWarps = 8;        // warps 4-11
+constexpr int kTmaWarp = 12;
+constexpr int kMmaWarp = 13;
+constexpr int kThreads = 16 * 32;
+constexpr uint32_t kABytes = BM * BK * 2;        // 16 KB
+constexpr uint32_t kQHalfBytes = BNH * BK / 2;   // 4 KB: 128 rows x 32 bytes of codes
+constexpr uint32_t kQBytes = 2 * kQHalfBytes;    // 8 KB
+constexpr uint32_t kLoadBytes = kABytes + kQBytes;
+constexpr uint32_t kDqBytes = BN * BK * 2;       // 32 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxExperts = 1024;
+
+struct W4Params {
+  const uint16_t* b_scales;  // bf16 bits [E][K/128][N]
+  const uint8_t* b_zeros;    // [E][K/128][N]
+  const int32_t* offsets;
+  int rows_total;
+  int ksteps;                // K / 64
+  int N;
+  int E;
+  int n_tiles;
+  int I;
+  uint16_t* out_bf16;
+  float* out_f32;
+  uint16_t* h_bf16;
+  const int32_t* sorted_pair;
+  const float* pair_weights;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+struct __align__(8) SmemTail {
+  uint64_t ld_full[kLoadStages];
+  uint64_t ld_empty[kLoadStages];
+  uint64_t dq_full[kDqStages];
+  uint64_t dq_empty[kDqStages];
+  uint64_t tmem_full[kAccBufs];
+  uint64_t tmem_empty[kAccBufs];
+  uint32_t tmem_addr;
+  int abort_flag;
+  int32_t off[kMaxExperts + 1];
+  int32_t prefix[kMaxExperts + 1];
+};
+
+constexpr size_t kSmemBytes =
+    1024 + static_cast<size_t>(kLoadStages) * kLoadBytes + static_cast<size_t>(kDqStages) * kDqBytes + sizeof(SmemTail);
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const W4Params& p) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*reinterpret_cast<volatile int*>(&s->abort_flag)) return false;
+    if (globaltimer_ns() - t0 > p.wait_limit_ns) {
+      set_status(p.status, QARL_ERR_DEVICE_TIMEOUT);
+      *reinterpret_cast<volatile int*>(&s->abort_flag) = 1;
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+__device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
+  const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&b);
+}
+
+// Two codes in bits [0,4) and [16,20) of `pair` -> bf16x2 of s * (q - z): 128 + q is exact in
+// bf16 (0x4300 | q), the subtraction of 128 + z is exact, the product is rounded once.
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t pair, uint32_t zc2, uint32_t s2) {
+  uint32_t t, d, v;
+  asm("lop3.b32 %0, %1, 0x000F000F, 0x43004300, 0xEA;" : "=r"(t) : "r"(pair));  // (a & b) | c
+  asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(t), "r"(zc2));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(d), "r"(s2));
+  return v;
+}
+
+// Eight codes of one 32-bit word -> 16 bytes (eight bf16 in K order).
+__device__ __forceinline__ uint4 dequant_word(uint32_t w, uint32_t zc2, uint32_t s2) {
+  return make_uint4(dequant_pair(w, zc2, s2), dequant_pair(w >> 4, zc2, s2), dequant_pair(w >> 8, zc2, s2),
+                    dequant_pair(w >> 12, zc2, s2));
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_q,
+                  const W4Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* dq_base = smem + static_cast<size_t>(kLoadStages) * kLoadBytes;
+  SmemTail* s = reinterpret_cast<SmemTail*>(dq_base + static_cast<size_t>(kDqStages) * kDqBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
+  pdl_trigger();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kLoadStages; ++i) {
+      mbar_init(&s->ld_full[i], 1);
+      mbar_init(&s->ld_empty[i], kDqWarps + 1);  // the dequant warps (codes read) + the MMA commit (A read)
+    }
+    for (int i = 0; i < kDqStages; ++i) {
+      mbar_init(&s->dq_full[i], kDqWarps);
+      mbar_init(&s->dq_empty[i], 1);
+    }
+    for (int i = 0; i < kAccBufs; ++i) {
+      mbar_init(&s->tmem_full[i], 1);
+      mbar_init(&s->tmem_empty[i], kEpiWarps);
+    }
+    s->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == kTmaWarp && lane == 0) {
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_q);
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(&s->tmem_addr, kTmemCols);
+    tmem_relinquish();
+  }
+  pdl_wait();  // nothing above read the predecessor's results
+  build_tile_list(s->off, s->prefix, p.offsets, p.rows_total, p.E, BM, p.n_tiles);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = s->tmem_addr;
+  const int total_tiles = s->prefix[p.E];
+  const int num_ctas = balanced_cta_count(total_tiles, gridDim.x);
+  const int first_tile = static_cast<int>(blockIdx.x) < num_ctas ? static_cast<int>(blockIdx.x) : total_tiles;
+  const int KS = p.ksteps;
+
+  // weight rows (within the [E*N] row space) of a tile's two halves
+  auto b_rows = [&](const TileCoord& c, int& n_lo, int& n_hi) {
+    if (MODE == kModeGateUp) {
+      n_lo = c.n_tile * BNH;
+      n_hi = n_lo + p.I;
+    } else {
+      n_lo = c.n_tile * BN;
+      n_hi = n_lo + BNH;
+    }
+  };
+
+  if (warp == kTmaWarp) {
+    // =============================== TMA producer =====================================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0, armed_parity = 0;
+      int cur_e = 0;
+      bool ok = true;
+      for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
+        const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+        int n_lo, n_hi;
+        b_rows(c, n_lo, n_hi);
+        const int row_lo = c.e * p.N + n_lo, row_hi = c.e * p.N + n_hi;
+        for (int ks = 0; ks < KS; ++ks) {
+          if (!wait_or_abort(&s->ld_empty[stage], phase ^ 1, s, p)) { ok = false; break; }
+          uint8_t* a_dst = smem + static_cast<size_t>(stage) * kLoadBytes;
+          uint8_t* q_dst = a_dst + kABytes;
+          mbar_arrive_expect_tx(&s->ld_full[stage], kLoadBytes);
+          tma_load_2d(a_dst, &tm_a, &s->ld_full[stage], ks * BK, c.m0);
+          tma_load_2d(q_dst, &tm_q, &s->ld_full[stage], ks * (BK / 2), row_lo);
+          tma_load_2d(q_dst + kQHalfBytes, &tm_q, &s->ld_full[stage], ks * (BK / 2), row_hi);
+          armed |= 1u << stage;
+          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == kLoadStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {  // let copies in flight land before the CTA's shared memory is released
+        for (int i = 0; i < kLoadStages; ++i)
+          if (armed & (1u << i)) mbar_wait_bounded(&s->ld_full[i], (armed_parity >> i) & 1u, 20000000ull);
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // =============================== MMA issuer =======================================
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+      int ls = 0, ds = 0, acc = 0;
+      uint32_t ld_phase = 0, dq_phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
+        if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+        for (int ks = 0; ks < KS; ++ks) {
+          if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
+          if (!wait_or_abort(&s->dq_full[ds], dq_phase, s, p)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint64_t a_desc = umma_desc_k_sw128(smem_u32(smem + static_cast<size_t>(ls) * kLoadBytes));
+          const uint64_t b_desc = umma_desc_k_sw128(smem_u32(dq_base + static_cast<size_t>(ds) * kDqBytes));
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 16; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
+            umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (ks > 0 || k4 > 0) ? 1u : 0u);
+          umma_commit(&s->ld_empty[ls]);
+          umma_commit(&s->dq_empty[ds]);
+          if (ks == KS - 1) umma_commit(&s->tmem_full[acc]);
+          if (++ls == kLoadStages) { ls = 0; ld_phase ^= 1; }
+          if (++ds == kDqStages) { ds = 0; dq_phase ^= 1; }
+        }
+        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else if (warp >= kEpiWarps && warp < kEpiWarps + kDqWarps) {
+    // =============================== dequantization warps =============================
+    const int n = (warp - kEpiWarps) * 32 + lane;  // weight row of the tile, 0..255
+    const int half = n >> 7, nr = n & 127;
+    const int KG = KS / 2;                         // 128-element groups along K
+    int ls = 0, ds = 0;
+    uint32_t ld_phase = 0, dq_phase = 0;
+    int cur_e = 0;
+    bool ok = true;
+    // (s, z) of group g of this thread's row in tile c; rows past N (dense, ragged N) clamp
+    auto sz_index = [&](const TileCoord& c, int g) -> int64_t {
+      int n_lo, n_hi;
+      b_rows(c, n_lo, n_hi);
+      const int row = min((half ? n_hi : n_lo) + nr, p.N - 1);
+      return (static_cast<int64_t>(c.e) * KG + g) * p.N + row;
+    };
+    int T = first_tile;
+    if (T < total_tiles) {
+      TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+      int64_t idx = sz_index(c, 0);
+      uint32_t s_next = __ldg(p.b_scales + idx), z_next = __ldg(p.b_zeros + idx);
+      for (;;) {
+        const int Tn = T + num_ctas;
+        const bool has_next = Tn < total_tiles;
+        TileCoord cn = c;
+        uint32_t s2 = 0, zc2 = 0;
+        for (int ks = 0; ks < KS; ++ks) {
+          if ((ks & 1) == 0) {
+            s2 = s_next | (s_next << 16);
+            zc2 = (0x4300u | z_next) * 0x00010001u;  // bf16x2 of 128 + z
+            const int g = ks >> 1;
+            if (g + 1 < KG) {
+              idx = sz_index(c, g + 1);
+            } else if (has_next) {
+              cn = decode_tile(s->off, s->prefix, BM, Tn, cur_e);
+              idx = sz_index(cn, 0);
+            }
+            s_next = __ldg(p.b_scales + idx);
+            z_next = __ldg(p.b_zeros + idx);
+          }
+          if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
+          const uint4* q_src = reinterpret_cast<const uint4*>(smem + static_cast<size_t>(ls) * kLoadBytes + kABytes +
+                                                              half * kQHalfBytes + nr * (BK / 2));
+          const uint4 q0 = q_src[0], q1 = q_src[1];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s->ld_empty[ls]);  // the codes are in registers
+          if (!wait_or_abort(&s->dq_empty[ds], dq_phase ^ 1, s, p)) { ok = false; break; }
+          uint8_t* row_dst = dq_base + static_cast<size_t>(ds) * kDqBytes + n * 128;
+          const uint32_t words[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+          for (int i = 0; i < 8; ++i)  // 16-byte chunk i of the row lands at chunk i ^ (row % 8): SWIZZLE_128B
+            *reinterpret_cast<uint4*>(row_dst + ((i ^ (n & 7)) << 4)) = dequant_word(words[i], zc2, s2);
+          fence_proxy_async_smem();  // generic-proxy stores -> visible to the tensor core's async proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s->dq_full[ds]);
+          if (++ls == kLoadStages) { ls = 0; ld_phase ^= 1; }
+          if (++ds == kDqStages) { ds = 0; dq_phase ^= 1; }
+        }
+        if (!ok || !has_next) break;
+        T = Tn;
+        c = cn;
+      }
+    }
+  } else if (warp < kEpiWarps) {
+    // =============================== epilogue warps ===================================
+    const int q = warp;              // TMEM lane quadrant
+    const int r = q * 32 + lane;     // row within the tile
+    const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    int cur_e = 0;
+    for (int T = first_tile; T < total_tiles; T += num_ctas) {
+      const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+      const int row = c.m0 + r;
+      const bool valid = row < c.m_end;
+      const bool warp_live = c.m0 + q * 32 < c.m_end;
+      float w = 0.0f;
+      int64_t out_row = row;
+      if (MODE == kModeDown && valid) {
+        w = __ldg(p.pair_weights + row);
+        out_row = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
+      }
+      if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
+      tc_fence_after_sync();
+      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN);
+      if (warp_live) {
+        if (MODE == kModeGateUp) {
+#pragma unroll 1
+          for (int ch = 0; ch < BNH / 16; ++ch) {
+            uint32_t vg[16], vu[16];
+            tmem_ld_x16(t0 + 16 * ch, vg);
+            tmem_ld_x16(t0 + BNH + 16 * ch, vu);
+            tmem_ld_wait();
+            uint32_t gb[8], ub[8], hb[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              gb[j] = bf16x2_bits(__uint_as_float(vg[2 * j]), __uint_as_float(vg[2 * j + 1]));
+              ub[j] = bf16x2_bits(__uint_as_float(vu[2 * j]), __uint_as_float(vu[2 * j + 1]));
+              const float h0 = silu_mul(bf16_bits_to_f32(gb[j] & 0xFFFFu), bf16_bits_to_f32(ub[j] & 0xFFFFu));
+              const float h1 = silu_mul(__uint_as_float(gb[j] & 0xFFFF0000u), __uint_as_float(ub[j] & 0xFFFF0000u));
+              hb[j] = bf16x2_bits(h0, h1);
+            }
+            if (valid) {
+              const int col = c.n_tile * BNH + 16 * ch;
+              uint4* hd = reinterpret_cast<uint4*>(p.h_bf16 + static_cast<int64_t>(row) * p.I + col);
+              hd[0] = make_uint4(hb[0], hb[1], hb[2], hb[3]);
+              hd[1] = make_uint4(hb[4], hb[5], hb[6], hb[7]);
+              if (p.out_bf16) {  // debug dump of the bf16 gate_up row
+                uint4* gd = reinterpret_cast<uint4*>(p.out_bf16 + static_cast<int64_t>(row) * p.N + col);
+                gd[0] = make_uint4(gb[0], gb[1], gb[2], gb[3]);
+                gd[1] = make_uint4(gb[4], gb[5], gb[6], gb[7]);
+                uint4* ud = reinterpret_cast<uint4*>(p.out_bf16 + static_cast<int64_t>(row) * p.N + p.I + col);
+                ud[0] = make_uint4(ub[0], ub[1], ub[2], ub[3]);
+                ud[1] = make_uint4(ub[4], ub[5], ub[6], ub[7]);
+              }
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (int ch = 0; ch < BN / 16; ++ch) {
+            uint32_t v[16];
+            tmem_ld_x16(t0 + 16 * ch, v);
+            tmem_ld_wait();
+            const int col = c.n_tile * BN + 16 * ch;
+            if (valid && col < p.N) {
+              if (p.out_f32) {  // fp32 accumulator dump (down: in sorted order)
+                float4* fd = reinterpret_cast<float4*>(p.out_f32 + static_cast<int64_t>(row) * p.N + col);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  fd[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                      __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+              }
+              uint32_t ob[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float a = __uint_as_float(v[2 * j]), b = __uint_as_float(v[2 * j + 1]);
+                if (MODE == kModeDown) {  // contribution = bf16( fl(w * y) )
+                  a = __fmul_rn(w, a);
+                  b = __fmul_rn(w, b);
+                }
+                ob[j] = bf16x2_bits(a, b);
+              }
+              if (p.out_bf16) {
+                uint4* od = reinterpret_cast<uint4*>(p.out_bf16 + out_row * p.N + col);
+                od[0] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+                od[1] = make_uint4(ob[4], ob[5], ob[6], ob[7]);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
+      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // ---- teardown ---------------------------------------------------------------------------
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+CUresult make_tmap_a(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint64_t rows, uint64_t K) {
+  // bf16 tensor [rows, K] row-major; box = 64 elements (128 bytes) x 128 rows, 128-byte swizzle.
+  const cuuint64_t dims[2] = {K, rows};
+  const cuuint64_t strides[1] = {K * 2};
+  const cuuint32_t box[2] = {BK, BM};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+CUresult make_tmap_q(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint64_t rows, uint64_t bytes_per_row) {
+  // u8 tensor [rows, K/2] row-major; box = 32 bytes x 128 rows, dense (no swizzle) in shared memory.
+  const cuuint64_t dims[2] = {bytes_per_row, rows};
+  const cuuint64_t strides[1] = {bytes_per_row};
+  const cuuint32_t box[2] = {BK / 2, BNH};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+template <int MODE>
+cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tq, const W4Params& p, int grid) {
+  static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
+  bool& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemBytes));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  ++*L.launches;
+  return launch_pdl(gemm_w4a16_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tq, p);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err) {
+  *cu_err = CUDA_SUCCESS;
+  if (a.rows_total == 0) return cudaSuccess;
+  CUtensorMap ta, tq;
+  CUresult r = make_tmap_a(encode, &ta, a.a_bf16, static_cast<uint64_t>(a.rows_total), static_cast<uint64_t>(a.K));
+  if (r == CUDA_SUCCESS)
+    r = make_tmap_q(encode, &tq, a.b_packed, static_cast<uint64_t>(a.E * a.N), static_cast<uint64_t>(a.K / 2));
+  if (r != CUDA_SUCCESS) {
+    *cu_err = r;
+    return cudaErrorUnknown;
+  }
+  W4Params p{};
+  p.b_scales = a.b_scales;
+  p.b_zeros = a.b_zeros;
+  p.offsets = a.offsets;
+  p.rows_total = static_cast<int>(a.rows_total);
+  p.ksteps = static_cast<int>(a.K / BK);
+  p.N = static_cast<int>(a.N);
+  p.E = static_cast<int>(a.E);
+  p.I = static_cast<int>(a.N / 2);
+  p.n_tiles = a.mode == kModeGateUp ? static_cast<int>(a.N / 2 / BNH) : static_cast<int>((a.N + BN - 1) / BN);
+  p.out_bf16 = a.out_bf16;
+  p.out_f32 = a.out_f32;
+  p.h_bf16 = a.h_bf16;
+  p.sorted_pair = a.sorted_pair;
+  p.pair_weights = a.pair_weights;
+  p.status = L.d_status;
+  p.wait_limit_ns = 2000000000ull;
+  const int64_t m_tiles_max = a.rows_total / BM + a.E;
+  const int grid = static_cast<int>(std::min<int64_t>(L.sm_count, m_tiles_max * p.n_tiles));
+  switch (a.mode) {
+    case kModeLinear: return launch_mode<kModeLinear>(L, ta, tq, p, grid);
+    case kModeGateUp: return launch_mode<kModeGateUp>(L, ta, tq, p, grid);
+    case kModeDown: return launch_mode<kModeDown>(L, ta, tq, p, grid);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace qarl

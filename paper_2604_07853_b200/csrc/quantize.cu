@@ -123,6 +123,101 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
   }
 }
 
+
+// ---- W4A16 weights (Sec. 2.2, integer quantization): W_q = clamp(round(W/s) + z, 0, 15) ------
+// One (s, z) per 128 consecutive K elements of a weight row: lo = min(0, min W), hi = max(0, max W),
+// s = bf16(max(hi - lo, 2^-40) / 15), z = clamp(rint(-lo / s), 0, 15).  8 threads per group, 16
+// elements (two 32-bit words of codes) each.  Inside a word the eight codes e0..e7 sit in the
+// nibble order e0 e2 e4 e6 e1 e3 e5 e7 (low nibble first), so that (word >> 4j) & 0x000F000F
+// yields the adjacent pair (e_2j, e_2j+1) in the two halves of a register.  Scales (bf16 bits)
+// and zero points are stored group-major, [E][K/128][N], contiguous along the weight rows.
+__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float zf) {
+  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+  uint32_t word = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float q0 = fminf(fmaxf(rintf(__fdiv_rn(bf16_bits_to_f32(in[j] & 0xFFFFu), s)) + zf, 0.0f), 15.0f);
+    const float q1 = fminf(fmaxf(rintf(__fdiv_rn(__uint_as_float(in[j] & 0xFFFF0000u), s)) + zf, 0.0f), 15.0f);
+    word |= static_cast<uint32_t>(q0) << (4 * j);
+    word |= static_cast<uint32_t>(q1) << (4 * j + 16);
+  }
+  return word;
+}
+
+__device__ __forceinline__ void minmax_u4(const uint4& v, float& lo, float& hi) {
+  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float a = bf16_bits_to_f32(in[j] & 0xFFFFu), b = __uint_as_float(in[j] & 0xFFFF0000u);
+    lo = fminf(lo, fminf(a, b));
+    hi = fmaxf(hi, fmaxf(a, b));
+  }
+}
+
+__global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t* __restrict__ w, int64_t rows,
+                                                                 int64_t N, int64_t K,
+                                                                 uint8_t* __restrict__ packed,
+                                                                 uint16_t* __restrict__ scales,
+                                                                 uint8_t* __restrict__ zeros) {
+  pdl_trigger();
+  pdl_wait();
+  const int64_t kb = K / kBlock;
+  const int64_t gid = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;
+  const bool live = gid < rows * kb;
+  const int64_t gg = live ? gid : 0;
+  const int64_t row = gg / kb, g = gg % kb;
+  const int sub = threadIdx.x & 7;
+  const uint4* src = reinterpret_cast<const uint4*>(w + row * K + g * kBlock + sub * 16);
+  uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+  if (live) {
+    v0 = __ldg(src);
+    v1 = __ldg(src + 1);
+  }
+  float lo = 0.0f, hi = 0.0f;
+  minmax_u4(v0, lo, hi);
+  minmax_u4(v1, lo, hi);
+#pragma unroll
+  for (int o = 4; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+  }
+  const float range = fmaxf(__fsub_rn(hi, lo), kAmaxFloor);
+  const uint32_t s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
+  const float s = bf16_bits_to_f32(s_bits);
+  const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
+  const uint2 out = make_uint2(w4_word(v0, s, zf), w4_word(v1, s, zf));
+  if (!live) return;
+  *reinterpret_cast<uint2*>(packed + row * (K / 2) + g * (kBlock / 2) + sub * 8) = out;
+  if (sub == 0) {
+    const int64_t e = row / N, n = row % N;
+    const int64_t idx = (e * kb + g) * N + n;
+    scales[idx] = static_cast<uint16_t>(s_bits);
+    zeros[idx] = static_cast<uint8_t>(zf);
+  }
+}
+
+// Copies bf16 row t of x to the `fanout` rows dst_rows[t*fanout + j] of out (expert-sorted
+// order) and scatters the pair weights alongside; 16 bytes per thread.
+__global__ void __launch_bounds__(256) scatter_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int64_t H,
+                                                           uint16_t* __restrict__ out,
+                                                           const int32_t* __restrict__ dst_rows, int fanout,
+                                                           int64_t dst_rows_total,
+                                                           const float* __restrict__ pair_w,
+                                                           float* __restrict__ sorted_w) {
+  pdl_trigger();
+  pdl_wait();
+  const int64_t per_row = H / 8;
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= M * per_row) return;
+  const int64_t row = idx / per_row, c = idx % per_row;
+  const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + row * H) + c);
+  for (int j = 0; j < fanout; ++j) {
+    const int64_t d = min(max(static_cast<int64_t>(dst_rows[row * fanout + j]), int64_t(0)), dst_rows_total - 1);
+    reinterpret_cast<uint4*>(out + d * H)[c] = v;
+    if (c == 0 && sorted_w != nullptr) sorted_w[d] = pair_w[row * fanout + j];
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
@@ -141,6 +236,25 @@ cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, i
   const int64_t blocks = (groups * 8 + 255) / 256;
   ++*L.launches;
   return launch_pdl(quantize_act_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, x, M, K, ldx, codes, scales,
+                    dst_rows, fanout, M * fanout, pair_w, sorted_w);
+}
+
+cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
+                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros) {
+  const int64_t groups = E * N * (K / kBlock);
+  if (groups == 0) return cudaSuccess;
+  const int64_t blocks = (groups * 8 + 255) / 256;
+  ++*L.launches;
+  return launch_pdl(quantize_weight_w4_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, E * N, N, K, packed,
+                    scales, zeros);
+}
+
+cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,
+                                const int32_t* dst_rows, int fanout, const float* pair_w, float* sorted_w) {
+  const int64_t threads = M * (H / 8);
+  if (threads == 0) return cudaSuccess;
+  ++*L.launches;
+  return launch_pdl(scatter_rows_kernel, static_cast<unsigned>((threads + 255) / 256), 256, 0, L.stream, x, M, H, out,
                     dst_rows, fanout, M * fanout, pair_w, sorted_w);
 }
 

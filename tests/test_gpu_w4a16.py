@@ -1,0 +1,253 @@
+"""GPU parity of the W4A16 path (Sec. 2.2, integer quantization; weight-only 4-bit with bf16
+activations): quantizer bit-exact against the oracle, the GEMM and the MoE layer teacher-forced
+against the oracle on the GPU's own codes, and the bitwise row invariance across batch shapes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_07853_b200 import binding, build, inputs
+from util import bf16_ulp_dist, bits_to_torch, to_dev, torch_to_bits
+
+pytestmark = pytest.mark.gpu
+
+# element held by nibble p of a 32-bit word in the library's storage order
+_NIBBLE_ELEM = np.array([0, 2, 4, 6, 1, 3, 5, 7])
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    build.build()
+    c = binding.Context(0)
+    yield c
+    assert c.poll() == 0
+    c.close()
+
+
+def unpack_lib(packed: np.ndarray) -> np.ndarray:
+    """library storage [.., K/2] u8 -> codes [.., K] (pure re-ordering of nibbles)."""
+    words = np.ascontiguousarray(packed).view("<u4")
+    nib = np.stack([(words >> (4 * p)) & 15 for p in range(8)], axis=-1).astype(np.uint8)
+    codes = np.empty_like(nib)
+    codes[..., _NIBBLE_ELEM] = nib
+    return codes.reshape(*packed.shape[:-1], packed.shape[-1] * 2)
+
+
+def unpack_linear(packed: np.ndarray) -> np.ndarray:
+    """oracle storage (code 2j low nibble, 2j+1 high nibble of byte j) -> codes [.., K]."""
+    return np.stack([packed & 15, packed >> 4], axis=-1).reshape(*packed.shape[:-1], packed.shape[-1] * 2)
+
+
+def pack_linear(codes: np.ndarray) -> np.ndarray:
+    c = codes.reshape(*codes.shape[:-1], codes.shape[-1] // 2, 2)
+    return (c[..., 0] | (c[..., 1] << 4)).astype(np.uint8)
+
+
+def host_weights(q):
+    """GPU (packed, scales, zeros) -> oracle-layout (packed, scales f32 [.., N, K/128], zeros)."""
+    packed, scales, zeros = q
+    p = pack_linear(unpack_lib(packed.cpu().numpy()))
+    s = inputs.bf16_bits_to_f32(torch_to_bits(scales))
+    return p, np.ascontiguousarray(np.swapaxes(s, -1, -2)), np.ascontiguousarray(np.swapaxes(zeros.cpu().numpy(), -1, -2))
+
+
+def w_hat_of(q):
+    return oracle.dequant_w4(*host_weights(q))
+
+
+# ------------------------------------------------------------------------------ quantizer
+@pytest.mark.parametrize("e,n,k", [(1, 128, 128), (3, 96, 384), (2, 1536, 2048), (4, 7, 256)])
+def test_quantizer_bit_exact(ctx, e, n, k):
+    rng = np.random.default_rng(10 + n)
+    w = inputs.weight_bf16(rng, e, n, k)
+    w[0, 0, :128] = 0                      # an all-zero group
+    w[-1, -1, ::3] = 0
+    op, os_, oz = oracle.quantize_weight_w4(w)
+    gp, gs, gz = host_weights(ctx.quantize_weight_w4(bits_to_torch(w)))
+    assert np.array_equal(unpack_linear(gp), unpack_linear(op))
+    assert np.array_equal(gs.view(np.uint32), os_.view(np.uint32))
+    assert np.array_equal(gz, oz)
+
+
+def test_quantizer_all_positive_and_all_negative_groups(ctx):
+    rng = np.random.default_rng(3)
+    w = inputs.bf16_bits_to_f32(inputs.weight_bf16(rng, 1, 64, 256))
+    w[:, :32, :128] = np.abs(w[:, :32, :128]) + 0.01     # lo clamps to 0: z = 0
+    w[:, 32:, 128:] = -np.abs(w[:, 32:, 128:]) - 0.01    # hi clamps to 0: z = 15
+    wb = inputs.f32_to_bf16_bits(w)
+    op, os_, oz = oracle.quantize_weight_w4(wb)
+    gp, gs, gz = host_weights(ctx.quantize_weight_w4(bits_to_torch(wb)))
+    assert (oz[0, :32, 0] == 0).all() and (oz[0, 32:, 1] == 15).all()
+    assert np.array_equal(unpack_linear(gp), unpack_linear(op))
+    assert np.array_equal(gs, os_) and np.array_equal(gz, oz)
+
+
+# ------------------------------------------------------------------------------ dense GEMM
+def check_linear(ctx, seed, m, n, k):
+    """fp32: |gpu - oracle| <= 1e-3 * ||x_row|| * ||w^_col|| (the oracle sums exactly; the tensor
+    core adds K exact products in fp32).  bf16: the rounding of the GPU's own fp32, bit for bit,
+    and within 1 ulp of the oracle's except where cancellation makes an ulp smaller than the
+    fp32 bound (rare)."""
+    case = inputs.linear_case(seed, m, n, k)
+    q = ctx.quantize_weight_w4(bits_to_torch(case.w))
+    xt = bits_to_torch(case.x)
+    y, y32 = ctx.linear_fwd_w4a16(xt, *q, want_f32=True)
+    assert ctx.poll() == 0
+    w_hat = w_hat_of(q)
+    o32, o16 = oracle.linear_bf16(case.x, w_hat)
+    g32, g16 = y32.cpu().numpy(), torch_to_bits(y)
+    nx = np.linalg.norm(inputs.bf16_bits_to_f32(case.x).astype(np.float64), axis=1)
+    nw = np.linalg.norm(inputs.bf16_bits_to_f32(w_hat).astype(np.float64), axis=1)
+    tol = 1e-3 * nx[:, None] * nw[None, :]
+    err = np.abs(g32.astype(np.float64) - o32.astype(np.float64))
+    assert (err <= tol).all(), f"max err/tol = {(err / tol).max()}"
+    assert np.array_equal(g16, oracle.bf16_rne(g32))
+    far = bf16_ulp_dist(g16, o16) > 1
+    assert far.mean() < 1e-3, f"{far.sum()} elements beyond 1 ulp"
+    return float((err / tol).max())
+
+
+@pytest.mark.parametrize("m,n,k", [(1, 128, 128), (127, 256, 256), (128, 384, 512), (129, 640, 2048),
+                                   (300, 1280, 768), (5, 256, 4096), (70, 4096, 2048)])
+def test_linear_shapes_and_ragged_tails(ctx, m, n, k):
+    check_linear(ctx, 200 + m, m, n, k)
+
+
+def test_linear_exact_on_integer_data(ctx):
+    """Small integers: every product and partial sum is exact in fp32, so the GPU must match the
+    exact result bit for bit (a wrong nibble, scale, zero point or swizzle cannot hide)."""
+    rng = np.random.default_rng(4)
+    m, n, k = 37, 256, 384
+    x = inputs.f32_to_bf16_bits(rng.integers(-4, 5, size=(m, k)).astype(np.float32))
+    # rows spanning exactly -8..7 quantize to s = 1, z = 8 and reproduce the integers exactly
+    wf = rng.integers(-8, 8, size=(n, k)).astype(np.float32)
+    wf[:, ::128] = -8
+    wf[:, 1::128] = 7
+    w = inputs.f32_to_bf16_bits(wf)
+    q = ctx.quantize_weight_w4(bits_to_torch(w))
+    assert np.array_equal(inputs.bf16_bits_to_f32(w_hat_of(q)), wf)
+    _, y32 = ctx.linear_fwd_w4a16(bits_to_torch(x), *q, want_f32=True)
+    assert np.array_equal(y32.cpu().numpy(), inputs.bf16_bits_to_f32(x) @ wf.T)
+
+
+def test_linear_rows_do_not_depend_on_the_batch(ctx):
+    case = inputs.linear_case(9, 300, 512, 1024)
+    q = ctx.quantize_weight_w4(bits_to_torch(case.w))
+    xt = bits_to_torch(case.x)
+    full = ctx.linear_fwd_w4a16(xt, *q)
+    for rows in ([0], [299], list(range(120, 140)), list(range(0, 300, 7))):
+        part = ctx.linear_fwd_w4a16(xt[rows].contiguous(), *q)
+        assert torch.equal(part, full[rows])
+
+
+# ------------------------------------------------------------------------------ MoE layer
+class DeviceCase:
+    def __init__(self, ctx, case):
+        self.case = case
+        self.x = bits_to_torch(case.x)
+        self.ids = to_dev(case.ids)
+        self.wts = to_dev(case.weights)
+        self.w13 = ctx.quantize_weight_w4(bits_to_torch(case.w13))
+        self.w2 = ctx.quantize_weight_w4(bits_to_torch(case.w2))
+
+    def run(self, ctx, debug=False, rows=None):
+        x, ids, wts = self.x, self.ids, self.wts
+        if rows is not None:
+            x, ids, wts = x[rows].contiguous(), ids[rows].contiguous(), wts[rows].contiguous()
+        return ctx.moe_fwd_w4a16(x, ids, wts, self.w13, self.w2, debug=debug)
+
+
+def _norm_tol(a_bits, w_hat_bits):
+    na = np.linalg.norm(inputs.bf16_bits_to_f32(a_bits).astype(np.float64), axis=1)
+    nw = np.linalg.norm(inputs.bf16_bits_to_f32(w_hat_bits).astype(np.float64), axis=1)
+    return 1e-3 * na[:, None] * nw[None, :]
+
+
+def check_moe(ctx, case, end_to_end=True):
+    dc = DeviceCase(ctx, case)
+    out, d = dc.run(ctx, debug=True)
+    assert ctx.poll() == 0
+    c = case
+    w13h, w2h = w_hat_of(dc.w13), w_hat_of(dc.w2)
+
+    # 1. permutation: bit-exact
+    off, srt, _ = oracle.permute(c.ids, c.E)
+    assert np.array_equal(d["expert_offsets"].cpu().numpy(), off)
+    assert np.array_equal(d["sorted_pair"].cpu().numpy(), srt)
+
+    # 2. gate_up (sorted order): <= 1 bf16 ulp of the oracle, beyond that only inside the fp32 bound
+    tok = srt // c.k
+    gu_gpu = torch_to_bits(d["gate_up"])
+    n_far = 0
+    for e in range(c.E):
+        a, b = off[e], off[e + 1]
+        if a == b:
+            continue
+        o32, o16 = oracle.linear_bf16(c.x[tok[a:b]], w13h[e])
+        far = bf16_ulp_dist(gu_gpu[a:b], o16) > 1
+        if far.any():
+            tol = _norm_tol(c.x[tok[a:b]], w13h[e])
+            g = inputs.bf16_bits_to_f32(gu_gpu[a:b]).astype(np.float64)
+            assert (np.abs(g - o32)[far] <= tol[far] + np.abs(g[far]) * 2.0 ** -8).all()
+        n_far += int(far.sum())
+    assert n_far <= 1e-3 * gu_gpu.size
+
+    # 3. SwiGLU on the GPU's own gate_up: <= 1 bf16 ulp
+    h_gpu = torch_to_bits(d["h"])
+    h_or = oracle.swiglu(gu_gpu)
+    assert bf16_ulp_dist(h_gpu, h_or).max() <= 1
+    assert (h_gpu == h_or).mean() > 0.99
+
+    # 4. down projection (fp32, sorted order) on the GPU's own h
+    dn = d["down_f32"].cpu().numpy()
+    for e in range(c.E):
+        a, b = off[e], off[e + 1]
+        if a == b:
+            continue
+        o32, _ = oracle.linear_bf16(h_gpu[a:b], w2h[e])
+        tol = _norm_tol(h_gpu[a:b], w2h[e])
+        err = np.abs(dn[a:b].astype(np.float64) - o32)
+        assert (err <= tol).all(), f"expert {e}: max err/tol {(err / tol).max()}"
+
+    # 5. combine: exact arithmetic on the GPU's fp32 rows -> bit-exact
+    by_pair = np.empty_like(dn)
+    by_pair[srt] = dn
+    assert np.array_equal(torch_to_bits(out), oracle.combine(by_pair, c.ids, c.weights))
+
+    # 6. end to end against the independent oracle
+    stats = {}
+    if end_to_end:
+        ref = oracle.moe_w4a16(c.x, c.ids, c.weights, w13h, w2h)
+        g = inputs.bf16_bits_to_f32(torch_to_bits(out)).astype(np.float64)
+        r = inputs.bf16_bits_to_f32(ref).astype(np.float64)
+        rel = np.linalg.norm(g - r) / np.linalg.norm(r)
+        dist = bf16_ulp_dist(torch_to_bits(out), ref)
+        stats.update(rel=float(rel), exact=float((dist == 0).mean()), within1=float((dist <= 1).mean()))
+        assert rel < 5e-3, stats
+    return stats
+
+
+def test_moe_small_layer(ctx):
+    check_moe(ctx, inputs.moe_case(5, 24, h=256, i=128, e=8, k=2))
+
+
+def test_moe_ragged_groups_and_empty_experts(ctx):
+    check_moe(ctx, inputs.moe_case(6, 3, h=256, i=256, e=16, k=4))
+    check_moe(ctx, inputs.moe_case(7, 333, h=512, i=256, e=4, k=2))
+
+
+def test_moe_skewed_popularity(ctx):
+    check_moe(ctx, inputs.moe_case(8, 1200, h=256, i=128, e=32, k=8, zipf_s=1.1), end_to_end=False)
+
+
+def test_moe_decode_layer_shape(ctx):
+    stats = check_moe(ctx, inputs.config3())
+    assert stats["within1"] > 0.98
+
+
+def test_moe_rows_do_not_depend_on_the_batch(ctx):
+    case = inputs.moe_case(11, 256, h=512, i=256, e=16, k=4, zipf_s=1.1)
+    dc = DeviceCase(ctx, case)
+    full = dc.run(ctx)
+    for rows in ([0], [255], list(range(100, 164)), list(range(0, 256, 5))):
+        assert torch.equal(dc.run(ctx, rows=rows), full[rows])
