@@ -171,8 +171,12 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
  * activations by w^ = bf16(s * (W_q - z)) and accumulates in fp32 in ascending k.
  *
  * Storage (all device pointers):
- *   packed  u8  [E, N, K/2]   every aligned 32-bit word holds eight consecutive codes e0..e7
- *                             of a row, nibble by nibble from the low end in the order
+ *   packed  u8, E*N*K/2 bytes, tile-major: the codes of weight rows [128b, 128b+128) x K
+ *                             elements [64c, 64c+64) of expert e form the contiguous 4096-byte
+ *                             chunk number (e*(N/128) + b)*(K/64) + c.  Inside a chunk the
+ *                             32-bit word w (0..7, eight consecutive codes e0..e7 each) of row
+ *                             r sits at byte (w/4)*2048 + r*16 + (w%4)*4; inside a word the
+ *                             codes lie nibble by nibble from the low end in the order
  *                             e0 e2 e4 e6 e1 e3 e5 e7 (so bits [4j, 4j+4) and [16+4j, 20+4j)
  *                             hold the adjacent pair e_2j, e_2j+1);
  *   scales  bf16 [E, K/128, N]  group-major: the scales of one K-group for all rows of an
@@ -180,7 +184,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
  *   zeros   u8  [E, K/128, N]  same layout.
  * ------------------------------------------------------------------------------------- */
 
-/* in : w_bf16 [E, N, K], 16-byte aligned, K % 128 == 0.  out: packed (16-byte aligned),
+/* in : w_bf16 [E, N, K], 16-byte aligned, N % 128 == 0, K % 128 == 0.  out: packed (16-byte aligned),
  * scales (2-byte aligned), zeros, as above; caller-owned.  One kernel, every input byte read once. */
 int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
                             uint8_t* packed, void* scales_bf16, uint8_t* zeros, void* stream);

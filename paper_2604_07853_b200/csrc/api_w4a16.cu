@@ -49,7 +49,7 @@ extern "C" {
 int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
                             void* scales, uint8_t* zeros, void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
-  if (K % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (K % kBlock || N % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E * N * (K / kBlock) > (0x7FFFFFFFll << 5)) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
   if (!w || !packed || !scales || !zeros) return QARL_ERR_INVALID_ARG;

@@ -16,7 +16,8 @@
 //
 // Structure of a CTA (512 threads, one CTA per SM, persistent, static tile list):
 //   warp 12     TMA producer: per K-step the A box (128 rows x 64 bf16, SWIZZLE_128B) and two
-//               boxes of packed codes (128 weight rows x 32 bytes) into a ring of load stages;
+//               4 KB chunks of packed codes (128 weight rows x 64 K-elements each, contiguous
+//               in the tile-major weight storage: one bulk copy per half) into a ring of load stages;
 //   warps 4-11  dequantization: thread n owns weight row n of the tile; it reads its 32 bytes
 //               of codes, forms pairs (w >> 4j) & 0x000F000F | 0x43004300 = bf16x2 (128 + q),
 //               subtracts 128 + z (exact), multiplies by s (one rounding: the bf16 of the exact
@@ -63,6 +64,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxExperts = 1024;
 
 struct W4Params {
+  const uint8_t* b_packed;   // tile-major 4 KB chunks [E][N/128][K/64]
   const uint16_t* b_scales;  // bf16 bits [E][K/128][N]
   const uint8_t* b_zeros;    // [E][K/128][N]
   const int32_t* offsets;
@@ -141,8 +143,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.p
 
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_q,
-                  const W4Params p) {
+gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* dq_base = smem + static_cast<size_t>(kLoadStages) * kLoadBytes;
@@ -169,7 +170,6 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   }
   if (warp == kTmaWarp && lane == 0) {
     prefetch_tensormap(&tm_a);
-    prefetch_tensormap(&tm_q);
   }
   if (warp == kMmaWarp) {
     tmem_alloc(&s->tmem_addr, kTmemCols);
@@ -209,15 +209,17 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
         int n_lo, n_hi;
         b_rows(c, n_lo, n_hi);
-        const int row_lo = c.e * p.N + n_lo, row_hi = c.e * p.N + n_hi;
+        const int NB = p.N / BNH;  // 128-row blocks per expert; a half tile past N re-reads the last one
+        const uint8_t* q_lo = p.b_packed + (static_cast<int64_t>(c.e) * NB + n_lo / BNH) * KS * kQHalfBytes;
+        const uint8_t* q_hi = p.b_packed + (static_cast<int64_t>(c.e) * NB + min(n_hi / BNH, NB - 1)) * KS * kQHalfBytes;
         for (int ks = 0; ks < KS; ++ks) {
           if (!wait_or_abort(&s->ld_empty[stage], phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* a_dst = smem + static_cast<size_t>(stage) * kLoadBytes;
           uint8_t* q_dst = a_dst + kABytes;
           mbar_arrive_expect_tx(&s->ld_full[stage], kLoadBytes);
           tma_load_2d(a_dst, &tm_a, &s->ld_full[stage], ks * BK, c.m0);
-          tma_load_2d(q_dst, &tm_q, &s->ld_full[stage], ks * (BK / 2), row_lo);
-          tma_load_2d(q_dst + kQHalfBytes, &tm_q, &s->ld_full[stage], ks * (BK / 2), row_hi);
+          bulk_load_1d(q_dst, q_lo + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->ld_full[stage]);
+          bulk_load_1d(q_dst + kQHalfBytes, q_hi + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->ld_full[stage]);
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == kLoadStages) { stage = 0; phase ^= 1; }
@@ -297,9 +299,10 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             z_next = __ldg(p.b_zeros + idx);
           }
           if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
+          // a chunk is [word quad 0..1][row][16 bytes]: consecutive threads read consecutive pieces
           const uint4* q_src = reinterpret_cast<const uint4*>(smem + static_cast<size_t>(ls) * kLoadBytes + kABytes +
-                                                              half * kQHalfBytes + nr * (BK / 2));
-          const uint4 q0 = q_src[0], q1 = q_src[1];
+                                                              half * kQHalfBytes + nr * 16);
+          const uint4 q0 = q_src[0], q1 = q_src[kQHalfBytes / 32];
           __syncwarp();
           if (lane == 0) mbar_arrive(&s->ld_empty[ls]);  // the codes are in registers
           if (!wait_or_abort(&s->dq_empty[ds], dq_phase ^ 1, s, p)) { ok = false; break; }
@@ -434,19 +437,8 @@ CUresult make_tmap_a(EncodeTiledFn encode, CUtensorMap* m, const void* base, uin
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-CUresult make_tmap_q(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint64_t rows, uint64_t bytes_per_row) {
-  // u8 tensor [rows, K/2] row-major; box = 32 bytes x 128 rows, dense (no swizzle) in shared memory.
-  const cuuint64_t dims[2] = {bytes_per_row, rows};
-  const cuuint64_t strides[1] = {bytes_per_row};
-  const cuuint32_t box[2] = {BK / 2, BNH};
-  const cuuint32_t estr[2] = {1, 1};
-  return encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-}
-
 template <int MODE>
-cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tq, const W4Params& p, int grid) {
+cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& p, int grid) {
   static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
   bool& attr_set = attr_set_dev[L.device & 63];
   if (!attr_set) {
@@ -456,7 +448,7 @@ cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMa
     attr_set = true;
   }
   ++*L.launches;
-  return launch_pdl(gemm_w4a16_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tq, p);
+  return launch_pdl(gemm_w4a16_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, p);
 }
 
 }  // namespace
@@ -464,15 +456,14 @@ cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMa
 cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err) {
   *cu_err = CUDA_SUCCESS;
   if (a.rows_total == 0) return cudaSuccess;
-  CUtensorMap ta, tq;
+  CUtensorMap ta;
   CUresult r = make_tmap_a(encode, &ta, a.a_bf16, static_cast<uint64_t>(a.rows_total), static_cast<uint64_t>(a.K));
-  if (r == CUDA_SUCCESS)
-    r = make_tmap_q(encode, &tq, a.b_packed, static_cast<uint64_t>(a.E * a.N), static_cast<uint64_t>(a.K / 2));
   if (r != CUDA_SUCCESS) {
     *cu_err = r;
     return cudaErrorUnknown;
   }
   W4Params p{};
+  p.b_packed = a.b_packed;
   p.b_scales = a.b_scales;
   p.b_zeros = a.b_zeros;
   p.offsets = a.offsets;
@@ -492,9 +483,9 @@ cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW
   const int64_t m_tiles_max = a.rows_total / BM + a.E;
   const int grid = static_cast<int>(std::min<int64_t>(L.sm_count, m_tiles_max * p.n_tiles));
   switch (a.mode) {
-    case kModeLinear: return launch_mode<kModeLinear>(L, ta, tq, p, grid);
-    case kModeGateUp: return launch_mode<kModeGateUp>(L, ta, tq, p, grid);
-    case kModeDown: return launch_mode<kModeDown>(L, ta, tq, p, grid);
+    case kModeLinear: return launch_mode<kModeLinear>(L, ta, p, grid);
+    case kModeGateUp: return launch_mode<kModeGateUp>(L, ta, p, grid);
+    case kModeDown: return launch_mode<kModeDown>(L, ta, p, grid);
   }
   return cudaErrorInvalidValue;
 }

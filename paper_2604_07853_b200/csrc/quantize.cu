@@ -129,8 +129,12 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
 // s = bf16(max(hi - lo, 2^-40) / 15), z = clamp(rint(-lo / s), 0, 15).  8 threads per group, 16
 // elements (two 32-bit words of codes) each.  Inside a word the eight codes e0..e7 sit in the
 // nibble order e0 e2 e4 e6 e1 e3 e5 e7 (low nibble first), so that (word >> 4j) & 0x000F000F
-// yields the adjacent pair (e_2j, e_2j+1) in the two halves of a register.  Scales (bf16 bits)
-// and zero points are stored group-major, [E][K/128][N], contiguous along the weight rows.
+// yields the adjacent pair (e_2j, e_2j+1) in the two halves of a register.  The words are
+// stored tile-major: the codes of 128 weight rows x 64 K-elements form one contiguous 4 KB chunk
+// (what one K-step of the GEMM consumes for one half tile, fetched by a single bulk copy), laid
+// out inside as [word quad 0..1][row 0..127][16 bytes] so that the 128 threads that expand it
+// read consecutive 16-byte pieces.  Scales (bf16 bits) and zero points are stored group-major,
+// [E][K/128][N], contiguous along the weight rows.
 __device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float zf) {
   const uint32_t in[4] = {v.x, v.y, v.z, v.w};
   uint32_t word = 0;
@@ -187,9 +191,14 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
   const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
   const uint2 out = make_uint2(w4_word(v0, s, zf), w4_word(v1, s, zf));
   if (!live) return;
-  *reinterpret_cast<uint2*>(packed + row * (K / 2) + g * (kBlock / 2) + sub * 8) = out;
+  const int64_t e = row / N, n = row % N;
+  {
+    const int64_t ks = g * 2 + (sub >> 2);  // K-step of 64 elements
+    const int64_t chunk = (e * (N / kBlock) + n / kBlock) * (K / 64) + ks;
+    const int quad = (sub & 3) >> 1, piece = sub & 1;  // words 2(sub%4), 2(sub%4)+1 of the K-step's eight
+    *reinterpret_cast<uint2*>(packed + chunk * 4096 + quad * 2048 + (n % kBlock) * 16 + piece * 8) = out;
+  }
   if (sub == 0) {
-    const int64_t e = row / N, n = row % N;
     const int64_t idx = (e * kb + g) * N + n;
     scales[idx] = static_cast<uint16_t>(s_bits);
     zeros[idx] = static_cast<uint8_t>(zf);
