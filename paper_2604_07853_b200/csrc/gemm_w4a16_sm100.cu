@@ -14,16 +14,16 @@
 // weight rows for linear/down, gate rows and the matching up rows for gate_up (SwiGLU in the
 // epilogue).  One K-step is 64 elements = one 128-byte swizzle span of bf16.
 //
-// Structure of a CTA (512 threads, one CTA per SM, persistent, static tile list):
-//   warp 12     TMA producer: per K-step the A box (128 rows x 64 bf16, SWIZZLE_128B) and two
+// Structure of a CTA (704 threads, one CTA per SM, persistent, static tile list):
+//   warp 20     TMA producer: per K-step the A box (128 rows x 64 bf16, SWIZZLE_128B) and two
 //               4 KB chunks of packed codes (128 weight rows x 64 K-elements each, contiguous
 //               in the tile-major weight storage: one bulk copy per half) into a ring of load stages;
-//   warps 4-11  dequantization: thread n owns weight row n of the tile; it reads its 32 bytes
+//   warps 4-19  dequantization, two groups of 8 warps on alternate K-steps: thread n owns weight row n of the tile; it reads its 32 bytes
 //               of codes, forms pairs (w >> 4j) & 0x000F000F | 0x43004300 = bf16x2 (128 + q),
 //               subtracts 128 + z (exact), multiplies by s (one rounding: the bf16 of the exact
 //               product), and writes the 128-byte row of the bf16 B tile in the 128-byte swizzle
 //               the tensor core expects; a proxy fence, then the warp arrives on the stage;
-//   warp 13     MMA issuer: 4 x tcgen05.mma kind::f16 (128 x 256 x 16) per K-step into one of
+//   warp 21     MMA issuer: 4 x tcgen05.mma kind::f16 (128 x 256 x 16) per K-step into one of
 //               two 256-column TMEM accumulators; tcgen05.commit frees the stages, and after
 //               the last K-step publishes the accumulator;
 //   warps 0-3   epilogue: TMEM -> registers -> bf16 output (linear), SwiGLU -> h (gate_up),
@@ -51,10 +51,12 @@ constexpr int kLoadStages = 4;     // A + packed codes
 constexpr int kDqStages = 3;       // dequantized B tiles
 constexpr int kAccBufs = 2;
 constexpr int kEpiWarps = 4;       // warps 0-3 (TMEM quadrant = warp index)
-constexpr int kDqWarps = 8;        // warps 4-11
-constexpr int kTmaWarp = 12;
-constexpr int kMmaWarp = 13;
-constexpr int kThreads = 16 * 32;
+constexpr int kDqGroupWarps = 8;   // one warp per 32 weight rows of the tile
+constexpr int kDqGroups = 2;       // warps 4-11 expand the even K-steps, warps 12-19 the odd ones
+constexpr int kDqWarps = kDqGroups * kDqGroupWarps;
+constexpr int kTmaWarp = 20;
+constexpr int kMmaWarp = 21;
+constexpr int kThreads = 22 * 32;
 constexpr uint32_t kABytes = BM * BK * 2;        // 16 KB
 constexpr uint32_t kQHalfBytes = BNH * BK / 2;   // 4 KB: 128 rows x 32 bytes of codes
 constexpr uint32_t kQBytes = 2 * kQHalfBytes;    // 8 KB
@@ -155,10 +157,10 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < kLoadStages; ++i) {
       mbar_init(&s->ld_full[i], 1);
-      mbar_init(&s->ld_empty[i], kDqWarps + 1);  // the dequant warps (codes read) + the MMA commit (A read)
+      mbar_init(&s->ld_empty[i], kDqGroupWarps + 1);  // one group's dequant warps (codes read) + the MMA commit (A read)
     }
     for (int i = 0; i < kDqStages; ++i) {
-      mbar_init(&s->dq_full[i], kDqWarps);
+      mbar_init(&s->dq_full[i], kDqGroupWarps);
       mbar_init(&s->dq_empty[i], 1);
     }
     for (int i = 0; i < kAccBufs; ++i) {
@@ -260,11 +262,13 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
     }
   } else if (warp >= kEpiWarps && warp < kEpiWarps + kDqWarps) {
     // =============================== dequantization warps =============================
-    const int n = (warp - kEpiWarps) * 32 + lane;  // weight row of the tile, 0..255
+    // Two groups of 8 warps take alternate K-steps (a tile has an even number of them), so the
+    // latency of one step's loads, barrier waits and stores hides behind the other group's math.
+    const int grp = (warp - kEpiWarps) / kDqGroupWarps;
+    const int n = ((warp - kEpiWarps) % kDqGroupWarps) * 32 + lane;  // weight row of the tile, 0..255
     const int half = n >> 7, nr = n & 127;
-    const int KG = KS / 2;                         // 128-element groups along K
-    int ls = 0, ds = 0;
-    uint32_t ld_phase = 0, dq_phase = 0;
+    const int KG = KS / 2;                         // 128-element groups along K: one K-step of each per group of warps
+    uint32_t step0 = 0;                            // K-steps of this CTA before the current tile
     int cur_e = 0;
     bool ok = true;
     // (s, z) of group g of this thread's row in tile c; rows past N (dense, ragged N) clamp
@@ -283,21 +287,20 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
         const int Tn = T + num_ctas;
         const bool has_next = Tn < total_tiles;
         TileCoord cn = c;
-        uint32_t s2 = 0, zc2 = 0;
-        for (int ks = 0; ks < KS; ++ks) {
-          if ((ks & 1) == 0) {
-            s2 = s_next | (s_next << 16);
-            zc2 = (0x4300u | z_next) * 0x00010001u;  // bf16x2 of 128 + z
-            const int g = ks >> 1;
-            if (g + 1 < KG) {
-              idx = sz_index(c, g + 1);
-            } else if (has_next) {
-              cn = decode_tile(s->off, s->prefix, BM, Tn, cur_e);
-              idx = sz_index(cn, 0);
-            }
-            s_next = __ldg(p.b_scales + idx);
-            z_next = __ldg(p.b_zeros + idx);
+        for (int g = 0; g < KG; ++g) {
+          const uint32_t s2 = s_next | (s_next << 16);
+          const uint32_t zc2 = (0x4300u | z_next) * 0x00010001u;  // bf16x2 of 128 + z
+          if (g + 1 < KG) {
+            idx = sz_index(c, g + 1);
+          } else if (has_next) {
+            cn = decode_tile(s->off, s->prefix, BM, Tn, cur_e);
+            idx = sz_index(cn, 0);
           }
+          s_next = __ldg(p.b_scales + idx);
+          z_next = __ldg(p.b_zeros + idx);
+          const uint32_t step = step0 + 2 * g + grp;
+          const uint32_t ls = step % kLoadStages, ld_phase = (step / kLoadStages) & 1u;
+          const uint32_t ds = step % kDqStages, dq_phase = (step / kDqStages) & 1u;
           if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
           // a chunk is [word quad 0..1][row][16 bytes]: consecutive threads read consecutive pieces
           const uint4* q_src = reinterpret_cast<const uint4*>(smem + static_cast<size_t>(ls) * kLoadBytes + kABytes +
@@ -314,10 +317,9 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           fence_proxy_async_smem();  // generic-proxy stores -> visible to the tensor core's async proxy
           __syncwarp();
           if (lane == 0) mbar_arrive(&s->dq_full[ds]);
-          if (++ls == kLoadStages) { ls = 0; ld_phase ^= 1; }
-          if (++ds == kDqStages) { ds = 0; dq_phase ^= 1; }
         }
         if (!ok || !has_next) break;
+        step0 += static_cast<uint32_t>(KS);
         T = Tn;
         c = cn;
       }
