@@ -47,9 +47,6 @@ constexpr int BM = 128;            // rows per tile (UMMA M)
 constexpr int BNH = 128;           // columns per half tile
 constexpr int BN = 2 * BNH;        // UMMA N
 constexpr int BK = 64;             // bf16 elements per K-step (128 bytes)
-constexpr int kLoadStages = 4;     // A + packed codes
-constexpr int kDqStages = 3;       // dequantized B tiles
-constexpr int kAccBufs = 2;
 constexpr int kEpiWarps = 4;       // warps 0-3 (TMEM quadrant = warp index)
 constexpr int kDqGroupWarps = 8;   // one warp per 32 weight rows of the tile
 constexpr int kDqGroups = 2;       // warps 4-11 expand the even K-steps, warps 12-19 the odd ones
@@ -57,13 +54,33 @@ constexpr int kDqWarps = kDqGroups * kDqGroupWarps;
 constexpr int kTmaWarp = 20;
 constexpr int kMmaWarp = 21;
 constexpr int kThreads = 22 * 32;
-constexpr uint32_t kABytes = BM * BK * 2;        // 16 KB
+constexpr uint32_t kAHalfBytes = BM * BK * 2;    // 16 KB: 128 token rows x 64 bf16
 constexpr uint32_t kQHalfBytes = BNH * BK / 2;   // 4 KB: 128 rows x 32 bytes of codes
 constexpr uint32_t kQBytes = 2 * kQHalfBytes;    // 8 KB
-constexpr uint32_t kLoadBytes = kABytes + kQBytes;
 constexpr uint32_t kDqBytes = BN * BK * 2;       // 32 KB
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxExperts = 1024;
+
+// A tile holds MT x 128 token rows.  MT = 2 (training-sized groups) expands every weight tile
+// once for 256 rows -- half the shared-memory traffic per flop, which is what bounds this
+// kernel -- at the price of a single set of accumulators (the epilogue, ~2% of a tile, is not
+// overlapped).  MT = 1 (decode-sized groups) keeps two accumulator sets and wastes no MMA work
+// on rows that do not exist.
+// Codes ring: always an even number of stages, so each dequantization group meets only stages it
+// consumed itself the time before (a parity wait cannot tell two outstanding fills apart).
+constexpr int kQStages = 4;
+template <int MT>
+struct Cfg {
+  static constexpr int kRows = MT * BM;
+  static constexpr uint32_t kABytes = MT * kAHalfBytes;
+  static constexpr int kAStages = MT == 1 ? 4 : 3;      // token tiles (ring of its own, freed by the MMA)
+  static constexpr int kDqStages = MT == 1 ? 3 : 2;     // dequantized B tiles
+  static constexpr int kAccBufs = MT == 1 ? 2 : 1;      // sets of MT 256-column TMEM accumulators
+  static constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kAStages) * kABytes +
+                                       static_cast<size_t>(kQStages) * kQBytes +
+                                       static_cast<size_t>(kDqStages) * kDqBytes;
+};
+constexpr int kMaxAStages = 4, kMaxDqStages = 3, kMaxAccBufs = 2;
 
 struct W4Params {
   const uint8_t* b_packed;   // tile-major 4 KB chunks [E][N/128][K/64]
@@ -86,21 +103,23 @@ struct W4Params {
 };
 
 struct __align__(8) SmemTail {
-  uint64_t ld_full[kLoadStages];
-  uint64_t ld_empty[kLoadStages];
-  uint64_t dq_full[kDqStages];
-  uint64_t dq_empty[kDqStages];
-  uint64_t tmem_full[kAccBufs];
-  uint64_t tmem_empty[kAccBufs];
+  uint64_t a_full[kMaxAStages];
+  uint64_t a_empty[kMaxAStages];
+  uint64_t q_full[kQStages];
+  uint64_t q_empty[kQStages];
+  uint64_t dq_full[kMaxDqStages];
+  uint64_t dq_empty[kMaxDqStages];
+  uint64_t tmem_full[kMaxAccBufs];
+  uint64_t tmem_empty[kMaxAccBufs];
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
   int32_t prefix[kMaxExperts + 1];
 };
 
-constexpr size_t kSmemBytes =
-    1024 + static_cast<size_t>(kLoadStages) * kLoadBytes + static_cast<size_t>(kDqStages) * kDqBytes + sizeof(SmemTail);
-static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+template <int MT>
+constexpr size_t smem_bytes() { return Cfg<MT>::kSmemBytes + sizeof(SmemTail); }
+static_assert(smem_bytes<1>() <= 227 * 1024 && smem_bytes<2>() <= 227 * 1024, "shared memory budget");
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const W4Params& p) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -143,21 +162,29 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, uint32_t zc2, uint32_t
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-template <int MODE>
+template <int MODE, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
+  using C = Cfg<MT>;
+  constexpr int kAStages = C::kAStages, kDqStages = C::kDqStages, kAccBufs = C::kAccBufs;
+  constexpr uint32_t kABytes = C::kABytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* dq_base = smem + static_cast<size_t>(kLoadStages) * kLoadBytes;
+  uint8_t* q_base = smem + static_cast<size_t>(kAStages) * kABytes;
+  uint8_t* dq_base = q_base + static_cast<size_t>(kQStages) * kQBytes;
   SmemTail* s = reinterpret_cast<SmemTail*>(dq_base + static_cast<size_t>(kDqStages) * kDqBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
   pdl_trigger();
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kLoadStages; ++i) {
-      mbar_init(&s->ld_full[i], 1);
-      mbar_init(&s->ld_empty[i], kDqGroupWarps + 1);  // one group's dequant warps (codes read) + the MMA commit (A read)
+    for (int i = 0; i < kAStages; ++i) {
+      mbar_init(&s->a_full[i], 1);
+      mbar_init(&s->a_empty[i], 1);               // the MMA commit
+    }
+    for (int i = 0; i < kQStages; ++i) {
+      mbar_init(&s->q_full[i], 1);
+      mbar_init(&s->q_empty[i], kDqGroupWarps);   // the dequant warps of the group that expanded it
     }
     for (int i = 0; i < kDqStages; ++i) {
       mbar_init(&s->dq_full[i], kDqGroupWarps);
@@ -178,7 +205,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
     tmem_relinquish();
   }
   pdl_wait();  // nothing above read the predecessor's results
-  build_tile_list(s->off, s->prefix, p.offsets, p.rows_total, p.E, BM, p.n_tiles);
+  build_tile_list(s->off, s->prefix, p.offsets, p.rows_total, p.E, C::kRows, p.n_tiles);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -202,34 +229,46 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
   if (warp == kTmaWarp) {
     // =============================== TMA producer =====================================
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      uint32_t armed = 0, armed_parity = 0;
+      int as = 0, qs = 0;
+      uint32_t a_phase = 0, q_phase = 0;
+      uint32_t a_armed = 0, a_armed_parity = 0, q_armed = 0, q_armed_parity = 0;
       int cur_e = 0;
       bool ok = true;
       for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
-        const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+        const TileCoord c = decode_tile(s->off, s->prefix, C::kRows, T, cur_e);
         int n_lo, n_hi;
         b_rows(c, n_lo, n_hi);
         const int NB = p.N / BNH;  // 128-row blocks per expert; a half tile past N re-reads the last one
         const uint8_t* q_lo = p.b_packed + (static_cast<int64_t>(c.e) * NB + n_lo / BNH) * KS * kQHalfBytes;
         const uint8_t* q_hi = p.b_packed + (static_cast<int64_t>(c.e) * NB + min(n_hi / BNH, NB - 1)) * KS * kQHalfBytes;
         for (int ks = 0; ks < KS; ++ks) {
-          if (!wait_or_abort(&s->ld_empty[stage], phase ^ 1, s, p)) { ok = false; break; }
-          uint8_t* a_dst = smem + static_cast<size_t>(stage) * kLoadBytes;
-          uint8_t* q_dst = a_dst + kABytes;
-          mbar_arrive_expect_tx(&s->ld_full[stage], kLoadBytes);
-          tma_load_2d(a_dst, &tm_a, &s->ld_full[stage], ks * BK, c.m0);
-          bulk_load_1d(q_dst, q_lo + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->ld_full[stage]);
-          bulk_load_1d(q_dst + kQHalfBytes, q_hi + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->ld_full[stage]);
-          armed |= 1u << stage;
-          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
-          if (++stage == kLoadStages) { stage = 0; phase ^= 1; }
+          // codes first: their ring frees as soon as they are in registers, and for decode-sized
+          // calls they are the stream from HBM that has to run ahead
+          if (!wait_or_abort(&s->q_empty[qs], q_phase ^ 1, s, p)) { ok = false; break; }
+          uint8_t* q_dst = q_base + static_cast<size_t>(qs) * kQBytes;
+          mbar_arrive_expect_tx(&s->q_full[qs], kQBytes);
+          bulk_load_1d(q_dst, q_lo + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->q_full[qs]);
+          bulk_load_1d(q_dst + kQHalfBytes, q_hi + static_cast<int64_t>(ks) * kQHalfBytes, kQHalfBytes, &s->q_full[qs]);
+          q_armed |= 1u << qs;
+          q_armed_parity = (q_armed_parity & ~(1u << qs)) | (q_phase << qs);
+          if (++qs == kQStages) { qs = 0; q_phase ^= 1; }
+
+          if (!wait_or_abort(&s->a_empty[as], a_phase ^ 1, s, p)) { ok = false; break; }
+          uint8_t* a_dst = smem + static_cast<size_t>(as) * kABytes;
+          mbar_arrive_expect_tx(&s->a_full[as], kABytes);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            tma_load_2d(a_dst + mt * kAHalfBytes, &tm_a, &s->a_full[as], ks * BK, c.m0 + mt * BM);
+          a_armed |= 1u << as;
+          a_armed_parity = (a_armed_parity & ~(1u << as)) | (a_phase << as);
+          if (++as == kAStages) { as = 0; a_phase ^= 1; }
         }
       }
       if (!ok) {  // let copies in flight land before the CTA's shared memory is released
-        for (int i = 0; i < kLoadStages; ++i)
-          if (armed & (1u << i)) mbar_wait_bounded(&s->ld_full[i], (armed_parity >> i) & 1u, 20000000ull);
+        for (int i = 0; i < kAStages; ++i)
+          if (a_armed & (1u << i)) mbar_wait_bounded(&s->a_full[i], (a_armed_parity >> i) & 1u, 20000000ull);
+        for (int i = 0; i < kQStages; ++i)
+          if (q_armed & (1u << i)) mbar_wait_bounded(&s->q_full[i], (q_armed_parity >> i) & 1u, 20000000ull);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -241,20 +280,23 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
       bool ok = true;
       for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
         if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * MT) * BN;
         for (int ks = 0; ks < KS; ++ks) {
-          if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
+          if (!wait_or_abort(&s->a_full[ls], ld_phase, s, p)) { ok = false; break; }
           if (!wait_or_abort(&s->dq_full[ds], dq_phase, s, p)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint64_t a_desc = umma_desc_k_sw128(smem_u32(smem + static_cast<size_t>(ls) * kLoadBytes));
+          const uint64_t a_desc = umma_desc_k_sw128(smem_u32(smem + static_cast<size_t>(ls) * kABytes));
           const uint64_t b_desc = umma_desc_k_sw128(smem_u32(dq_base + static_cast<size_t>(ds) * kDqBytes));
 #pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
-            umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (ks > 0 || k4 > 0) ? 1u : 0u);
-          umma_commit(&s->ld_empty[ls]);
+          for (int mt = 0; mt < MT; ++mt)  // the 128-row halves of A share the expanded weight tile
+#pragma unroll
+            for (int k4 = 0; k4 < BK / 16; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
+              umma_bf16(d_tmem + mt * BN, a_desc + mt * (kAHalfBytes >> 4) + 2 * k4, b_desc + 2 * k4, idesc,
+                        (ks > 0 || k4 > 0) ? 1u : 0u);
+          umma_commit(&s->a_empty[ls]);
           umma_commit(&s->dq_empty[ds]);
           if (ks == KS - 1) umma_commit(&s->tmem_full[acc]);
-          if (++ls == kLoadStages) { ls = 0; ld_phase ^= 1; }
+          if (++ls == kAStages) { ls = 0; ld_phase ^= 1; }
           if (++ds == kDqStages) { ds = 0; dq_phase ^= 1; }
         }
         if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
@@ -280,7 +322,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
     };
     int T = first_tile;
     if (T < total_tiles) {
-      TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+      TileCoord c = decode_tile(s->off, s->prefix, C::kRows, T, cur_e);
       int64_t idx = sz_index(c, 0);
       uint32_t s_next = __ldg(p.b_scales + idx), z_next = __ldg(p.b_zeros + idx);
       for (;;) {
@@ -293,21 +335,21 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           if (g + 1 < KG) {
             idx = sz_index(c, g + 1);
           } else if (has_next) {
-            cn = decode_tile(s->off, s->prefix, BM, Tn, cur_e);
+            cn = decode_tile(s->off, s->prefix, C::kRows, Tn, cur_e);
             idx = sz_index(cn, 0);
           }
           s_next = __ldg(p.b_scales + idx);
           z_next = __ldg(p.b_zeros + idx);
           const uint32_t step = step0 + 2 * g + grp;
-          const uint32_t ls = step % kLoadStages, ld_phase = (step / kLoadStages) & 1u;
+          const uint32_t qs = step % kQStages, q_phase = (step / kQStages) & 1u;
           const uint32_t ds = step % kDqStages, dq_phase = (step / kDqStages) & 1u;
-          if (!wait_or_abort(&s->ld_full[ls], ld_phase, s, p)) { ok = false; break; }
+          if (!wait_or_abort(&s->q_full[qs], q_phase, s, p)) { ok = false; break; }
           // a chunk is [word quad 0..1][row][16 bytes]: consecutive threads read consecutive pieces
-          const uint4* q_src = reinterpret_cast<const uint4*>(smem + static_cast<size_t>(ls) * kLoadBytes + kABytes +
+          const uint4* q_src = reinterpret_cast<const uint4*>(q_base + static_cast<size_t>(qs) * kQBytes +
                                                               half * kQHalfBytes + nr * 16);
           const uint4 q0 = q_src[0], q1 = q_src[kQHalfBytes / 32];
           __syncwarp();
-          if (lane == 0) mbar_arrive(&s->ld_empty[ls]);  // the codes are in registers
+          if (lane == 0) mbar_arrive(&s->q_empty[qs]);  // the codes are in registers
           if (!wait_or_abort(&s->dq_empty[ds], dq_phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* row_dst = dq_base + static_cast<size_t>(ds) * kDqBytes + n * 128;
           const uint32_t words[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
@@ -333,19 +375,24 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
     uint32_t acc_phase = 0;
     int cur_e = 0;
     for (int T = first_tile; T < total_tiles; T += num_ctas) {
-      const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
-      const int row = c.m0 + r;
+      const TileCoord c = decode_tile(s->off, s->prefix, C::kRows, T, cur_e);
+      bool ok = true;
+#pragma unroll 1
+      for (int mt = 0; mt < MT; ++mt) {
+      const int row = c.m0 + mt * BM + r;
       const bool valid = row < c.m_end;
-      const bool warp_live = c.m0 + q * 32 < c.m_end;
+      const bool warp_live = c.m0 + mt * BM + q * 32 < c.m_end;
       float w = 0.0f;
       int64_t out_row = row;
       if (MODE == kModeDown && valid) {
         w = __ldg(p.pair_weights + row);
         out_row = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
       }
-      if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
-      tc_fence_after_sync();
-      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN);
+      if (mt == 0) {
+        if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) { ok = false; break; }
+        tc_fence_after_sync();
+      }
+      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>((acc * MT + mt) * BN);
       if (warp_live) {
         if (MODE == kModeGateUp) {
 #pragma unroll 1
@@ -412,6 +459,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           }
         }
       }
+      }  // mt
+      if (!ok) break;
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
@@ -439,18 +488,29 @@ CUresult make_tmap_a(EncodeTiledFn encode, CUtensorMap* m, const void* base, uin
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int MODE>
-cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& p, int grid) {
+template <int MODE, int MT>
+cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
   static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
   bool& attr_set = attr_set_dev[L.device & 63];
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kSmemBytes));
+    cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem_bytes<MT>()));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  // upper bound on the tile count (group sizes live on the device): each expert adds at most
+  // one partial row tile
+  const int64_t m_tiles_max = a.rows_total / Cfg<MT>::kRows + a.E;
+  const int grid = static_cast<int>(std::min<int64_t>(L.sm_count, m_tiles_max * p.n_tiles));
   ++*L.launches;
-  return launch_pdl(gemm_w4a16_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, p);
+  return launch_pdl(gemm_w4a16_kernel<MODE, MT>, static_cast<unsigned>(grid), kThreads, smem_bytes<MT>(), L.stream, ta, p);
+}
+
+template <int MODE>
+cudaError_t launch_mt(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
+  // groups of at most 128 rows on average (decode-sized calls): 128-row tiles
+  if (a.rows_total <= a.E * BM) return launch_mode<MODE, 1>(L, ta, p, a);
+  return launch_mode<MODE, 2>(L, ta, p, a);
 }
 
 }  // namespace
@@ -482,12 +542,10 @@ cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW
   p.pair_weights = a.pair_weights;
   p.status = L.d_status;
   p.wait_limit_ns = 2000000000ull;
-  const int64_t m_tiles_max = a.rows_total / BM + a.E;
-  const int grid = static_cast<int>(std::min<int64_t>(L.sm_count, m_tiles_max * p.n_tiles));
   switch (a.mode) {
-    case kModeLinear: return launch_mode<kModeLinear>(L, ta, p, grid);
-    case kModeGateUp: return launch_mode<kModeGateUp>(L, ta, p, grid);
-    case kModeDown: return launch_mode<kModeDown>(L, ta, p, grid);
+    case kModeLinear: return launch_mt<kModeLinear>(L, ta, p, a);
+    case kModeGateUp: return launch_mt<kModeGateUp>(L, ta, p, a);
+    case kModeDown: return launch_mt<kModeDown>(L, ta, p, a);
   }
   return cudaErrorInvalidValue;
 }
