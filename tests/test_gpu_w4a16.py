@@ -256,3 +256,82 @@ def test_moe_rows_do_not_depend_on_the_batch(ctx):
     full = dc.run(ctx)
     for rows in ([0], [255], list(range(100, 164)), list(range(0, 256, 5))):
         assert torch.equal(dc.run(ctx, rows=rows), full[rows])
+
+
+# ------------------------------------------------------------------------------ full size
+def test_moe_training_shape_sampled(ctx):
+    """M = 32768, Zipf(1.1), the shapes of the benchmark step: sampled sorted positions against
+    the oracle (teacher-forced on the GPU's own codes and intermediates), combine bit-exact on
+    sampled tokens, and the same tokens run as two halves give the same bytes."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    dev = torch.device("cuda", 0)
+    M, H, I, E, k = 32768, bench.H, bench.I, bench.E, bench.TOPK
+    w13, w2, x, ids, wts = bench.make_inputs(M, 1000, dev, zipf=True)
+    q13 = ctx.quantize_weight_w4(w13)
+    q2 = ctx.quantize_weight_w4(w2)
+    out, d = ctx.moe_fwd_w4a16(x, ids, wts, q13, q2, debug=True)
+    assert ctx.poll() == 0
+    ids_h, wts_h = ids.cpu().numpy(), wts.cpu().numpy()
+
+    # weight quantization: three experts, bit-exact (codes, scales, zero points)
+    p13, s13, z13 = host_weights(q13)
+    p2, s2, z2 = host_weights(q2)
+    for e in (0, 57, 127):
+        for w, (gp, gs, gz) in ((w13, (p13, s13, z13)), (w2, (p2, s2, z2))):
+            op, os_, oz = oracle.quantize_weight_w4(torch_to_bits(w[e]))
+            assert np.array_equal(gp[e], op) and np.array_equal(gs[e], os_) and np.array_equal(gz[e], oz)
+
+    off, srt, _ = oracle.permute(ids_h, E)
+    assert np.array_equal(d["expert_offsets"].cpu().numpy(), off)
+    assert np.array_equal(d["sorted_pair"].cpu().numpy(), srt)
+    sizes = np.diff(off)
+
+    rng = np.random.default_rng(0)
+    order = np.argsort(sizes)
+    picks = []
+    for e in (order[np.nonzero(sizes[order])[0][0]], order[E // 2], order[-1]):
+        picks += [off[e], off[e + 1] - 1, (off[e] + off[e + 1]) // 2, off[e] + min(129, sizes[e] - 1)]
+    picks += list(rng.integers(0, M * k, size=40))
+    picks = np.array(sorted(set(int(q) for q in picks)))
+    tok = srt[picks] // k
+    exp = ids_h.reshape(-1)[srt[picks]]
+    sel = torch.from_numpy(picks).cuda()
+    xs_bits = torch_to_bits(x[torch.from_numpy(tok).cuda()])
+    gu = torch_to_bits(d["gate_up"][sel])
+    hh = torch_to_bits(d["h"][sel])
+    dn = d["down_f32"][sel].cpu().numpy()
+    far = 0
+    what = {}
+    for i, e in enumerate(exp):
+        if e not in what:
+            what[e] = (oracle.dequant_w4(p13[e], s13[e], z13[e]), oracle.dequant_w4(p2[e], s2[e], z2[e]))
+        w13h, w2h = what[e]
+        o32, o16 = oracle.linear_bf16(xs_bits[i:i + 1], w13h)
+        bad = bf16_ulp_dist(gu[i:i + 1], o16) > 1
+        if bad.any():
+            tol = _norm_tol(xs_bits[i:i + 1], w13h)
+            g = inputs.bf16_bits_to_f32(gu[i:i + 1]).astype(np.float64)
+            assert (np.abs(g - o32)[bad] <= tol[bad] + np.abs(g[bad]) * 2.0 ** -8).all()
+        far += int(bad.sum())
+        assert bf16_ulp_dist(hh[i:i + 1], oracle.swiglu(gu[i:i + 1])).max() <= 1
+        o32, _ = oracle.linear_bf16(hh[i:i + 1], w2h)
+        assert (np.abs(dn[i:i + 1].astype(np.float64) - o32) <= _norm_tol(hh[i:i + 1], w2h)).all()
+    assert far <= 1e-3 * gu.size
+
+    pos = np.empty(M * k, dtype=np.int64)
+    pos[srt] = np.arange(M * k)
+    for t in rng.integers(0, M, size=24):
+        rows = torch.from_numpy(pos[t * k:(t + 1) * k]).cuda()
+        ref = oracle.combine(d["down_f32"][rows].cpu().numpy(), ids_h[t:t + 1], wts_h[t:t + 1])
+        assert np.array_equal(torch_to_bits(out[t:t + 1]), ref)
+
+    half = M // 2
+    a = ctx.moe_fwd_w4a16(x[:half], ids[:half], wts[:half], q13, q2).clone()
+    b = ctx.moe_fwd_w4a16(x[half:], ids[half:], wts[half:], q13, q2)
+    assert torch.equal(torch.cat([a, b]), out)
+    # decode-sized call on a slice of the same tokens (128-row tiles) gives the same rows
+    c = ctx.moe_fwd_w4a16(x[:256], ids[:256], wts[:256], q13, q2)
+    assert torch.equal(c, out[:256])
