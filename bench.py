@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-w4a16", action="store_true")
     ap.add_argument("--tokens", type=int, default=M_TRAIN,
                     help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
                          "only; the reported config names the size)")
@@ -322,6 +323,80 @@ def main():
                            "frac_fp8_peak_nominal_4500": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12 / 4500.0},
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches * world, "clocks": clocks,
     }
+
+    # ---------------- W4A16 variant of the same layer (4-bit weights, bf16 activations)
+    if not args.no_w4a16:
+        q13 = ctx.quantize_weight_w4(w13)
+        q2 = ctx.quantize_weight_w4(w2)
+        ws4 = torch.empty(ctx.moe_w4a16_workspace_bytes(M_TRAIN, H, I, E, TOPK), dtype=torch.uint8, device=dev)
+
+        def step4():
+            ctx.quantize_weight_w4(w13, out=q13)
+            ctx.quantize_weight_w4(w2, out=q2)
+            ctx.moe_fwd_w4a16(x, ids, wts, q13, q2, out=out, workspace=ws4)
+
+        steps4 = max(args.steps // 2, 10)
+        for _ in range(3):
+            step4()
+        barrier()
+        ev0.record()
+        for _ in range(steps4):
+            step4()
+        ev1.record()
+        barrier()
+        ms4 = max_over_ranks(ev0.elapsed_time(ev1)) / steps4
+        ctx.profile_begin(max_marks=steps4 * 16 + 8)
+        for _ in range(steps4):
+            step4()
+        st4 = ctx.profile_end()
+        ctx.check_device_status()
+        gu4 = st4["gate_up_gemm"][0] / max(st4["gate_up_gemm"][1], 1)
+        dn4 = st4["down_gemm"][0] / max(st4["down_gemm"][1], 1)
+        gu_tf = 2.0 * M_TRAIN * TOPK * H * 2 * I / (gu4 * 1e-3) / 1e12
+        dn_tf = 2.0 * M_TRAIN * TOPK * I * H / (dn4 * 1e-3) / 1e12
+        w4 = {
+            "workload": f"moe_ffn_train_M{M_TRAIN} with W4A16 weights (per-step 4-bit quantization + layer forward)",
+            "ms_per_step": ms4, "tokens_per_s": world * M_TRAIN / (ms4 * 1e-3),
+            "stage_ms": {k: v[0] / steps4 for k, v in st4.items() if v[1]},
+            "gate_up_tflops": gu_tf, "down_tflops": dn_tf,
+            "gate_up_frac_bf16_peak_measured_sustained": gu_tf / pk["bf16_sustained"],
+            "gate_up_frac_bf16_peak_measured_burst": gu_tf / pk["bf16_burst"],
+        }
+        # decode shape on pre-quantized weights; two weight copies alternated so that no step
+        # re-reads a copy that is resident in L2
+        _, _, xd4, idd4, wtd4 = make_inputs(M_DECODE, 2000 + rank, dev, zipf=False)
+        outd4 = torch.empty((M_DECODE, H), dtype=torch.bfloat16, device=dev)
+        sets4 = [(q13, q2), (tuple(t.clone() for t in q13), tuple(t.clone() for t in q2))]
+        dsteps4 = max(args.steps, 20) * 5
+
+        def dstep4(i):
+            a, b = sets4[i & 1]
+            ctx.moe_fwd_w4a16(xd4, idd4, wtd4, a, b, out=outd4, workspace=ws4)
+
+        for i in range(10):
+            dstep4(i)
+        barrier()
+        ev0.record()
+        for i in range(dsteps4):
+            dstep4(i)
+        ev1.record()
+        barrier()
+        d4_ms = max_over_ranks(ev0.elapsed_time(ev1)) / dsteps4
+        ctx.profile_begin(max_marks=dsteps4 * 8 + 8)
+        for i in range(dsteps4):
+            dstep4(i)
+        dst4 = ctx.profile_end()
+        ctx.check_device_status()
+        wbytes4 = sum(t.numel() * t.element_size() for t in (*q13, *q2)) + 2 * M_DECODE * H * 2
+        w4["decode"] = {
+            "workload": "moe_ffn_decode_M256 with W4A16 weights (pre-quantized, two copies alternated)",
+            "ms_per_step": d4_ms, "tokens_per_s": world * M_DECODE / (d4_ms * 1e-3),
+            "algorithmic_bytes": wbytes4, "gbs": wbytes4 / (d4_ms * 1e-3) / 1e9,
+            "frac_hbm_measured": wbytes4 / (d4_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+            "stage_ms": {k: v[0] / dsteps4 for k, v in dst4.items() if v[1]},
+        }
+        result["w4a16"] = w4
+        del q13, q2, sets4, ws4
 
     # ---------------- decode shape (rollout engine: weights already quantized)
     if not args.no_decode:

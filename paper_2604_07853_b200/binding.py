@@ -297,15 +297,19 @@ class Context:
         return (y, d) if debug else y
 
     # ------------------------------------------------------------------ W4A16
-    def quantize_weight_w4(self, w: torch.Tensor):
+    def quantize_weight_w4(self, w: torch.Tensor, out=None):
         """w bf16 [E, N, K] or [N, K] -> (packed u8 [.., N, K/2], scales bf16 [.., K/128, N],
-        zeros u8 [.., K/128, N]) in the library's storage order (see include/qarl.h)."""
+        zeros u8 [.., K/128, N]) in the library's storage order (see include/qarl.h).
+        out: an earlier result of this call to overwrite."""
         assert w.dtype == torch.bfloat16 and w.is_cuda and w.is_contiguous()
         shape = w.shape
         E, N, K = (1, *shape) if w.dim() == 2 else shape
-        packed = torch.empty((*shape[:-1], K // 2), dtype=torch.uint8, device=w.device)
-        scales = torch.empty((*shape[:-2], K // 128, N), dtype=torch.bfloat16, device=w.device)
-        zeros = torch.empty((*shape[:-2], K // 128, N), dtype=torch.uint8, device=w.device)
+        if out is not None:
+            packed, scales, zeros = out
+        else:
+            packed = torch.empty((*shape[:-1], K // 2), dtype=torch.uint8, device=w.device)
+            scales = torch.empty((*shape[:-2], K // 128, N), dtype=torch.bfloat16, device=w.device)
+            zeros = torch.empty((*shape[:-2], K // 128, N), dtype=torch.uint8, device=w.device)
         self._check(self.lib.qarl_quantize_weight_w4(self.h, _ptr(w), E, N, K, _ptr(packed), _ptr(scales),
                                                      _ptr(zeros), _stream()))
         return packed, scales, zeros

@@ -135,15 +135,32 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
 // out inside as [word quad 0..1][row 0..127][16 bytes] so that the 128 threads that expand it
 // read consecutive 16-byte pieces.  Scales (bf16 bits) and zero points are stored group-major,
 // [E][K/128][N], contiguous along the weight rows.
-__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float zf) {
+// rint(w / s) + z clamped to 0..15 for one element, equal to the IEEE-division form bit for bit
+// but without a division per element.  w and s are bf16 values (8 significant bits each), so the
+// exact quotient is either exactly half-way between two integers or at least 2^-14 (relative) away
+// from such a point: the product with inv = fl(1 / s) (relative error ~2^-23) then rounds to the
+// same integer except at exact ties, which the exact residual r = w - q0 s identifies
+// (2 r = +-s) and resolves to the even neighbour.  Rounding by adding and subtracting 1.5 * 2^23.
+__device__ __forceinline__ uint32_t w4_code(float w, float s, float inv, float zf) {
+  const float kMagic = 12582912.0f;
+  float q0 = __fsub_rn(__fadd_rn(__fmul_rn(w, inv), kMagic), kMagic);
+  const float r2 = 2.0f * __fmaf_rn(-q0, s, w);  // exact: q0 s has at most 13 significant bits
+  if (r2 == s || r2 == -s) {                     // tie between q0 and q0 + sign(r2)
+    const float other = r2 > 0.0f ? q0 + 1.0f : q0 - 1.0f;
+    const float half = 0.5f * q0;
+    if (__fsub_rn(__fadd_rn(half, kMagic), kMagic) != half) q0 = other;  // q0 odd: the other one is even
+  }
+  const float v = fminf(fmaxf(q0 + zf, 0.0f), 15.0f);
+  return __float_as_uint(v + 8388608.0f) & 15u;  // integer 0..15 in the low mantissa bits
+}
+
+__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float inv, float zf) {
   const uint32_t in[4] = {v.x, v.y, v.z, v.w};
   uint32_t word = 0;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const float q0 = fminf(fmaxf(rintf(__fdiv_rn(bf16_bits_to_f32(in[j] & 0xFFFFu), s)) + zf, 0.0f), 15.0f);
-    const float q1 = fminf(fmaxf(rintf(__fdiv_rn(__uint_as_float(in[j] & 0xFFFF0000u), s)) + zf, 0.0f), 15.0f);
-    word |= static_cast<uint32_t>(q0) << (4 * j);
-    word |= static_cast<uint32_t>(q1) << (4 * j + 16);
+    word |= w4_code(bf16_bits_to_f32(in[j] & 0xFFFFu), s, inv, zf) << (4 * j);
+    word |= w4_code(__uint_as_float(in[j] & 0xFFFF0000u), s, inv, zf) << (4 * j + 16);
   }
   return word;
 }
@@ -189,7 +206,8 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
   const uint32_t s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
   const float s = bf16_bits_to_f32(s_bits);
   const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
-  const uint2 out = make_uint2(w4_word(v0, s, zf), w4_word(v1, s, zf));
+  const float inv = __fdiv_rn(1.0f, s);
+  const uint2 out = make_uint2(w4_word(v0, s, inv, zf), w4_word(v1, s, inv, zf));
   if (!live) return;
   const int64_t e = row / N, n = row % N;
   {

@@ -87,6 +87,26 @@ def test_quantizer_all_positive_and_all_negative_groups(ctx):
     assert np.array_equal(gs, os_) and np.array_equal(gz, oz)
 
 
+def test_quantizer_exact_ties_round_to_even(ctx):
+    """Multiples of s/2: every other value sits exactly half-way between two codes, where the
+    result must be the even neighbour (the oracle's rint of an exact IEEE quotient)."""
+    rng = np.random.default_rng(5)
+    w = rng.integers(-16, 15, size=(1, 128, 384)).astype(np.float32) * 0.125     # s = 3.75 / 15 = 0.25
+    w[:, :, ::128] = -2.0
+    w[:, :, 1::128] = 1.75
+    # other scales: the same pattern times powers of two and times 3 (s keeps 8 significant bits)
+    w[:, 32:64] *= 8.0
+    w[:, 64:96] *= 2.0 ** -10
+    w[:, 96:] *= 3.0
+    wb = inputs.f32_to_bf16_bits(w)
+    assert np.array_equal(inputs.bf16_bits_to_f32(wb), w)
+    op, os_, oz = oracle.quantize_weight_w4(wb)
+    assert os_[0, 0, 0] == np.float32(0.25) and os_[0, 100, 0] == np.float32(0.75)
+    gp, gs, gz = host_weights(ctx.quantize_weight_w4(bits_to_torch(wb)))
+    assert np.array_equal(unpack_linear(gp), unpack_linear(op))
+    assert np.array_equal(gs, os_) and np.array_equal(gz, oz)
+
+
 # ------------------------------------------------------------------------------ dense GEMM
 def check_linear(ctx, seed, m, n, k):
     """fp32: |gpu - oracle| <= 1e-3 * ||x_row|| * ||w^_col|| (the oracle sums exactly; the tensor
