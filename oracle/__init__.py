@@ -57,6 +57,8 @@ def lib() -> C.CDLL:
         L.oracle_linear_bf16.argtypes = [p, i64, i64, p, i64, p, p]
         L.oracle_moe_w4a16.restype = C.c_int
         L.oracle_moe_w4a16.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p]
+        L.oracle_linear_bwd.restype = None
+        L.oracle_linear_bwd.argtypes = [p, p, p, i64, i64, i64, p, p, p]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
     return _lib
@@ -271,3 +273,18 @@ def moe_w4a16(x_bits, ids, wts, w13_hat, w2_hat, dumps: bool = False):
     if rc:
         raise OracleError(rc)
     return (out, d) if dumps else out
+
+
+# ---------------------------------------------------------------------------- STE backward
+def linear_bwd(dy_bits, x_bits, w_bits):
+    """Backward of y = x . W^T on bf16 masters (straight-through past the quantizer):
+    -> (dX fp32 [M, K], dX bf16 bits, dW fp32 [N, K])."""
+    dy, x, w = _c(dy_bits, np.uint16), _c(x_bits, np.uint16), _c(w_bits, np.uint16)
+    M, N = dy.shape
+    K = x.shape[1]
+    assert x.shape == (M, K) and w.shape == (N, K)
+    dx32 = np.empty((M, K), dtype=np.float32)
+    dx16 = np.empty((M, K), dtype=np.uint16)
+    dw32 = np.empty((N, K), dtype=np.float32)
+    lib().oracle_linear_bwd(_ptr(dy), _ptr(x), _ptr(w), M, N, K, _ptr(dx32), _ptr(dx16), _ptr(dw32))
+    return dx32, dx16, dw32

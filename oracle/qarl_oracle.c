@@ -526,6 +526,45 @@ int oracle_moe_w4a16(const uint16_t *x, const int32_t *ids, const float *wts,
     return 0;
 }
 
+
+/* =======================================================================================
+ * Training-side backward of a quantized linear layer (Sec. 3.1 item 2: the forward runs in low
+ * bit, the backward in full precision; gradients pass the quantizer by the straight-through
+ * estimator and are applied to the bf16 master weights).  Reading: with y = x . W^T computed on
+ * Quant(W), the backward treats Quant as the identity and uses the bf16 masters themselves:
+ *   dX[m,k] = sum_n dY[m,n] W[n,k]      dW[n,k] = sum_m dY[m,n] X[m,k]
+ * bf16 operands; every product and the whole sum exact in double, rounded once to fp32
+ * (dX additionally to bf16, dW stays fp32 as the gradient a master-weight optimizer consumes).
+ * ===================================================================================== */
+void oracle_linear_bwd(const uint16_t *dy, const uint16_t *x, const uint16_t *w,
+                       int64_t M, int64_t N, int64_t K, float *dx32, uint16_t *dx16, float *dw32) {
+    float *dyf = (float *)malloc((size_t)(M > 0 ? M : 1) * N * sizeof(float));
+    for (int64_t i = 0; i < M * N; ++i) dyf[i] = bf16_to_f32(dy[i]);
+    if (dx32 || dx16) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m)
+            for (int64_t k = 0; k < K; ++k) {
+                double acc = 0.0;
+                for (int64_t n = 0; n < N; ++n)
+                    acc += (double)dyf[m * N + n] * (double)bf16_to_f32(w[n * K + k]);
+                float a = (float)acc;
+                if (dx32) dx32[m * K + k] = a;
+                if (dx16) dx16[m * K + k] = oracle_bf16_rne(a);
+            }
+    }
+    if (dw32) {
+#pragma omp parallel for schedule(static)
+        for (int64_t n = 0; n < N; ++n)
+            for (int64_t k = 0; k < K; ++k) {
+                double acc = 0.0;
+                for (int64_t m = 0; m < M; ++m)
+                    acc += (double)dyf[m * N + n] * (double)bf16_to_f32(x[m * K + k]);
+                dw32[n * K + k] = (float)acc;
+            }
+    }
+    free(dyf);
+}
+
 /* Number of OpenMP threads the oracle will use (reported beside its timing). */
 #ifdef _OPENMP
 #include <omp.h>
