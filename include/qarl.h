@@ -217,6 +217,22 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_id
                        void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
                        void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * Training-side backward of a quantized linear layer y = x . W^T (Sec. 3.1 item 2: the forward
+ * runs on Quant(W), the backward in full precision; the straight-through estimator treats Quant
+ * as the identity and the gradients belong to the bf16 master weights):
+ *   dX[m,k] = sum_n dY[m,n] W[n,k]  -> dx_bf16 [M, K] (and dx_f32 [M, K] if not NULL)
+ *   dW[n,k] = sum_m dY[m,n] X[m,k]  -> dw_f32 [N, K] (fp32, overwritten, not accumulated)
+ * in : dy_bf16 [M, N], x_bf16 [M, K], w_bf16 [N, K] (the masters, not the codes); device
+ *      pointers, 16-byte aligned; N % 8 == 0, K % 8 == 0, M >= 1.  Either output group may be
+ *      skipped: dx_bf16 == NULL && dx_f32 == NULL skips dX, dw_f32 == NULL skips dW.
+ * Two launches of one bf16 tensor-core GEMM that reads its operands in either orientation, so
+ * no transposed copy is made; fp32 accumulation in one fixed order (ascending n, resp. m): a
+ * row of dX depends only on that row of dY.  Needs no workspace. */
+int qarl_linear_bwd(qarl_ctx* ctx, const void* dy_bf16, const void* x_bf16, const void* w_bf16,
+                    int64_t M, int64_t N, int64_t K, void* dx_bf16, float* dx_f32, float* dw_f32,
+                    void* stream);
+
 /* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
  * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
  * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;
@@ -232,7 +248,9 @@ enum {
   QARL_STAGE_GATE_UP_GEMM = 4,
   QARL_STAGE_DOWN_GEMM = 5,
   QARL_STAGE_COMBINE = 6,
-  QARL_NUM_STAGES = 7
+  QARL_STAGE_BWD_DX = 7,
+  QARL_STAGE_BWD_DW = 8,
+  QARL_NUM_STAGES = 9
 };
 int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
 int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);

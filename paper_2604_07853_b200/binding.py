@@ -31,12 +31,12 @@ EXPORTS = [
     "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
-    "qarl_moe_fwd_w4a16",
+    "qarl_moe_fwd_w4a16", "qarl_linear_bwd",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
-          "combine"]
+          "combine", "bwd_dx", "bwd_dw"]
 
 
 class QarlError(RuntimeError):
@@ -108,6 +108,8 @@ def load() -> C.CDLL:
     L.qarl_moe_fwd_w4a16.restype = C.c_int
     L.qarl_moe_fwd_w4a16.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, sz,
                                      C.POINTER(MoeDebug), p]
+    L.qarl_linear_bwd.restype = C.c_int
+    L.qarl_linear_bwd.argtypes = [p, p, p, p, i64, i64, i64, p, p, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
     L.qarl_harness_rmsnorm.argtypes = [p, p, i64, i64, C.c_float, p, p]
     L.qarl_harness_wait_selftest.restype = C.c_int
@@ -356,3 +358,19 @@ class Context:
                                                 _ptr(y), _ptr(ws), ws.numel(),
                                                 C.byref(dbg) if dbg is not None else None, _stream()))
         return (y, d) if debug else y
+
+    # ------------------------------------------------------------------ backward
+    def linear_bwd(self, dy, x, w, want_dx_f32: bool = False, dx: bool = True, dw: bool = True):
+        """Straight-through backward of y = x . W^T on the bf16 masters ->
+        (dX bf16 [M, K] or None, dX fp32 or None, dW fp32 [N, K] or None)."""
+        for t in (dy, x, w):
+            assert t.dtype == torch.bfloat16 and t.is_cuda and t.is_contiguous()
+        M, N = dy.shape
+        K = x.shape[1]
+        assert x.shape == (M, K) and w.shape == (N, K)
+        dxo = torch.empty((M, K), dtype=torch.bfloat16, device=dy.device) if dx else None
+        dx32 = torch.empty((M, K), dtype=torch.float32, device=dy.device) if (dx and want_dx_f32) else None
+        dwo = torch.empty((N, K), dtype=torch.float32, device=dy.device) if dw else None
+        self._check(self.lib.qarl_linear_bwd(self.h, _ptr(dy), _ptr(x), _ptr(w), M, N, K, _ptr(dxo), _ptr(dx32),
+                                             _ptr(dwo), _stream()))
+        return dxo, dx32, dwo

@@ -1,5 +1,5 @@
-// C ABI entry points of the W4A16 path (4-bit group-quantized weights, bf16 activations):
-// argument checks, workspace planning, kernel sequencing.  No device memory is allocated here.
+// C ABI entry points of the W4A16 path (4-bit group-quantized weights, bf16 activations) and of
+// the full-precision backward: argument checks, workspace planning, kernel sequencing.  No device memory is allocated here.
 #include "api_util.cuh"
 
 namespace {
@@ -184,6 +184,57 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const f
     if (dbg->h_bf16 && (e = cudaMemcpyAsync(dbg->h_bf16, h, static_cast<size_t>(P) * I * sizeof(uint16_t),
                                             cudaMemcpyDeviceToDevice, L.stream)) != cudaSuccess)
       return cuda_fail(ctx, e, "copy h");
+  }
+  return QARL_OK;
+}
+
+int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w, int64_t M, int64_t N, int64_t K,
+                    void* dx, float* dx_f32, float* dw_f32, void* stream) {
+  if (!ctx || M < 0 || N <= 0 || K <= 0) return QARL_ERR_INVALID_ARG;
+  if (N % 8 || K % 8 || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll || K > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (M == 0) return QARL_OK;
+  if (!dy || !x || !w) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(w) || !aligned16(dx) || !aligned16(dx_f32) || !aligned16(dw_f32))
+    return QARL_ERR_MISALIGNED;
+  Launch L = make_launch(ctx, stream);
+  CUresult cu = CUDA_SUCCESS;
+  auto run = [&](const GemmBf16Args& a, const char* what) {
+    cudaError_t e = launch_gemm_bf16(L, ctx->encode, a, &cu);
+    if (cu != CUDA_SUCCESS) {
+      snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+      return static_cast<int>(QARL_ERR_CUDA);
+    }
+    return e == cudaSuccess ? static_cast<int>(QARL_OK) : cuda_fail(ctx, e, what);
+  };
+  mark(ctx, L.stream, -1);
+  if (dx || dx_f32) {
+    GemmBf16Args a{};
+    a.a = static_cast<const uint16_t*>(dy);  // A(m, n) = dY[m, n]: the contraction index n is contiguous
+    a.a_mn_major = false;
+    a.b = static_cast<const uint16_t*>(w);   // B(k, n) = W[n, k]: stored [n][k], the output index k is contiguous
+    a.b_mn_major = true;
+    a.Mo = M;
+    a.No = K;
+    a.Kc = N;
+    a.c_bf16 = static_cast<uint16_t*>(dx);
+    a.c_f32 = dx_f32;
+    const int rc = run(a, "linear_bwd dX");
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_BWD_DX);
+  }
+  if (dw_f32) {
+    GemmBf16Args a{};
+    a.a = static_cast<const uint16_t*>(dy);  // A(n, m) = dY[m, n]: stored [m][n], the output index n is contiguous
+    a.a_mn_major = true;
+    a.b = static_cast<const uint16_t*>(x);   // B(k, m) = X[m, k]
+    a.b_mn_major = true;
+    a.Mo = N;
+    a.No = K;
+    a.Kc = M;
+    a.c_f32 = dw_f32;
+    const int rc = run(a, "linear_bwd dW");
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_BWD_DW);
   }
   return QARL_OK;
 }

@@ -164,6 +164,17 @@ struct GemmW4Args {
 };
 cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err);
 
+// ---- dense bf16 GEMM (full-precision backward): C[i,j] = sum_c A(i,c) B(j,c) ---------------------
+struct GemmBf16Args {
+  const uint16_t* a;   // K-major: [Mo, Kc] row-major;  MN-major: [Kc, Mo] row-major
+  const uint16_t* b;   // K-major: [No, Kc] row-major;  MN-major: [Kc, No] row-major
+  bool a_mn_major, b_mn_major;
+  int64_t Mo, No, Kc;
+  uint16_t* c_bf16;    // [Mo, No] or nullptr
+  float* c_f32;        // [Mo, No] or nullptr
+};
+cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err);
+
 }  // namespace qarl
 
 // The opaque context of the C ABI (one per device).

@@ -1,0 +1,303 @@
+// Dense bf16 GEMM for sm_100a: the full-precision backward of the quantized linear layer
+// (Sec. 3.1 item 2: low-bit forward, backward in full precision on the bf16 master weights,
+// gradients passed through the quantizer by the straight-through estimator).
+//
+//   C[i, j] = sum over c ascending of A(i, c) * B(j, c),   fp32 accumulation in TMEM.
+//
+// Each operand is given as a row-major bf16 matrix in one of two orientations:
+//   K-major   memory [rows = i or j][cols = c]   (the contraction index is contiguous)
+//   MN-major  memory [rows = c][cols = i or j]   (the output index is contiguous)
+// so that no transposed copy of dY, X or W is ever made:
+//   dX[m, k] = sum_n dY[m, n] W[n, k]:  A = dY (K-major),  B = W  (MN-major, [c = n][j = k])
+//   dW[n, k] = sum_m dY[m, n] X[m, k]:  A = dY (MN-major, [c = m][i = n]),  B = X (MN-major)
+//
+// Tile 128 x 256 x 64.  TMA stages both operands with the 128-byte swizzle (a K-major tile is
+// one box of R rows x 128 bytes; an MN-major tile is one box of 64 c-rows x 128 bytes per 64
+// output indices); one thread issues 4 x tcgen05.mma kind::f16 (128 x 256 x 16) per stage with
+// the matching operand-major bits; two 256-column TMEM accumulators let the epilogue of a tile
+// overlap the main loop of the next.  Static persistent schedule, row tiles fastest.  One fixed
+// order of accumulation: a result does not depend on the grid or on the other rows.
+// Every wait is bounded (status word + CTA-wide abort flag), as in the other GEMMs.
+#include <algorithm>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace qarl {
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kAccBufs = 2;
+constexpr int kEpiWarps = 4;   // warps 0-3 (TMEM quadrant = warp index)
+constexpr int kTmaWarp = 4;
+constexpr int kMmaWarp = 5;
+constexpr int kThreads = 6 * 32;
+constexpr uint32_t kABytes = BM * BK * 2;   // 16 KB
+constexpr uint32_t kBBytes = BN * BK * 2;   // 32 KB
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kBlockBytes = 64 * BK * 2;  // one MN-major block: 64 output indices x 64 c-rows
+constexpr uint32_t kTmemCols = 512;
+
+struct Bf16Params {
+  int Mo, No, Kc;
+  uint16_t* c_bf16;   // [Mo, No] or nullptr
+  float* c_f32;       // [Mo, No] or nullptr
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+
+struct __align__(8) SmemTail {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+  uint64_t tmem_full[kAccBufs];
+  uint64_t tmem_empty[kAccBufs];
+  uint32_t tmem_addr;
+  int abort_flag;
+};
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + sizeof(SmemTail);
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const Bf16Params& p) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*reinterpret_cast<volatile int*>(&s->abort_flag)) return false;
+    if (globaltimer_ns() - t0 > p.wait_limit_ns) {
+      set_status(p.status, QARL_ERR_DEVICE_TIMEOUT);
+      *reinterpret_cast<volatile int*>(&s->abort_flag) = 1;
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
+  const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&b);
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                 const Bf16Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  SmemTail* s = reinterpret_cast<SmemTail*>(smem + static_cast<size_t>(kStages) * kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  pdl_trigger();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&s->full[i], 1);
+      mbar_init(&s->empty[i], 1);
+    }
+    for (int i = 0; i < kAccBufs; ++i) {
+      mbar_init(&s->tmem_full[i], 1);
+      mbar_init(&s->tmem_empty[i], kEpiWarps);
+    }
+    s->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == kTmaWarp && lane == 0) {
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_b);
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(&s->tmem_addr, kTmemCols);
+    tmem_relinquish();
+  }
+  pdl_wait();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = s->tmem_addr;
+  const int m_tiles = (p.Mo + BM - 1) / BM, n_tiles = (p.No + BN - 1) / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int KS = (p.Kc + BK - 1) / BK;  // a ragged last step reads zeros (TMA out-of-range fill)
+  const int grid = gridDim.x;
+
+  if (warp == kTmaWarp) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0, armed_parity = 0;
+      bool ok = true;
+      for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
+        const int i0 = (T % m_tiles) * BM, j0 = (T / m_tiles) * BN;
+        for (int ks = 0; ks < KS; ++ks) {
+          if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
+          uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
+          uint8_t* b_dst = a_dst + kABytes;
+          mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
+          if (A_MN) {
+#pragma unroll
+            for (int b = 0; b < BM / 64; ++b)
+              tma_load_2d(a_dst + b * kBlockBytes, &tm_a, &s->full[stage], i0 + 64 * b, ks * BK);
+          } else {
+            tma_load_2d(a_dst, &tm_a, &s->full[stage], ks * BK, i0);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int b = 0; b < BN / 64; ++b)
+              tma_load_2d(b_dst + b * kBlockBytes, &tm_b, &s->full[stage], j0 + 64 * b, ks * BK);
+          } else {
+            tma_load_2d(b_dst, &tm_b, &s->full[stage], ks * BK, j0);
+          }
+          armed |= 1u << stage;
+          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < kStages; ++i)
+          if (armed & (1u << i)) mbar_wait_bounded(&s->full[i], (armed_parity >> i) & 1u, 20000000ull);
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32_major(BM, BN, A_MN, B_MN);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
+        if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+        for (int ks = 0; ks < KS; ++ks) {
+          if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+          const uint64_t a_desc = A_MN ? umma_desc_mn_sw128(a_addr, kBlockBytes) : umma_desc_k_sw128(a_addr);
+          const uint64_t b_desc = B_MN ? umma_desc_mn_sw128(b_addr, kBlockBytes) : umma_desc_k_sw128(b_addr);
+          // 16 contraction elements further on: 32 bytes inside a K-major row, 16 rows of 128 bytes
+          // in an MN-major block (start-address field counts 16-byte units)
+          constexpr uint32_t a_step = A_MN ? (16 * 128) >> 4 : 32 >> 4;
+          constexpr uint32_t b_step = B_MN ? (16 * 128) >> 4 : 32 >> 4;
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 16; ++k4)
+            umma_bf16(d_tmem, a_desc + a_step * k4, b_desc + b_step * k4, idesc, (ks > 0 || k4 > 0) ? 1u : 0u);
+          umma_commit(&s->empty[stage]);
+          if (ks == KS - 1) umma_commit(&s->tmem_full[acc]);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else if (warp < kEpiWarps) {
+    const int r = warp * 32 + lane;
+    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int T = blockIdx.x; T < total_tiles; T += grid) {
+      const int i0 = (T % m_tiles) * BM, j0 = (T / m_tiles) * BN;
+      const int row = i0 + r;
+      const bool valid = row < p.Mo;
+      const bool warp_live = i0 + warp * 32 < p.Mo;
+      if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
+      tc_fence_after_sync();
+      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN);
+      if (warp_live) {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 16; ++ch) {
+          const int col = j0 + 16 * ch;
+          if (col >= p.No) break;
+          uint32_t v[16];
+          tmem_ld_x16(t0 + 16 * ch, v);
+          tmem_ld_wait();
+          if (valid) {
+            const bool whole = col + 16 <= p.No;  // No is a multiple of 8: a ragged last chunk holds 8 columns
+            if (p.c_f32) {
+              float4* fd = reinterpret_cast<float4*>(p.c_f32 + static_cast<int64_t>(row) * p.No + col);
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                if (j < 2 || whole)
+                  fd[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                      __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+            }
+            if (p.c_bf16) {
+              uint32_t ob[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) ob[j] = bf16x2_bits(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              uint4* od = reinterpret_cast<uint4*>(p.c_bf16 + static_cast<int64_t>(row) * p.No + col);
+              od[0] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+              if (whole) od[1] = make_uint4(ob[4], ob[5], ob[6], ob[7]);
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
+      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Tensor map of a row-major bf16 matrix [rows, cols] with a box of box_cols x box_rows elements.
+CUresult make_tmap(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                   uint32_t box_cols, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+template <bool A_MN, bool B_MN>
+cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p) {
+  static bool attr_set_dev[64] = {};
+  bool& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemBytes));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t tiles = static_cast<int64_t>((p.Mo + BM - 1) / BM) * ((p.No + BN - 1) / BN);
+  // full rounds only: with W = ceil(tiles / SMs) rounds, ceil(tiles / W) CTAs finish in W rounds
+  const int64_t rounds = (tiles + L.sm_count - 1) / L.sm_count;
+  const int grid = static_cast<int>((tiles + rounds - 1) / rounds);
+  ++*L.launches;
+  return launch_pdl(gemm_bf16_kernel<A_MN, B_MN>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err) {
+  *cu_err = CUDA_SUCCESS;
+  if (a.Mo == 0 || a.No == 0) return cudaSuccess;
+  CUtensorMap ta, tb;
+  CUresult r = a.a_mn_major ? make_tmap(encode, &ta, a.a, a.Kc, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a.Mo, a.Kc, BK, BM);
+  if (r == CUDA_SUCCESS)
+    r = a.b_mn_major ? make_tmap(encode, &tb, a.b, a.Kc, a.No, 64, BK) : make_tmap(encode, &tb, a.b, a.No, a.Kc, BK, BN);
+  if (r != CUDA_SUCCESS) {
+    *cu_err = r;
+    return cudaErrorUnknown;
+  }
+  Bf16Params p{};
+  p.Mo = static_cast<int>(a.Mo);
+  p.No = static_cast<int>(a.No);
+  p.Kc = static_cast<int>(a.Kc);
+  p.c_bf16 = a.c_bf16;
+  p.c_f32 = a.c_f32;
+  p.status = L.d_status;
+  p.wait_limit_ns = 2000000000ull;
+  if (a.a_mn_major) return a.b_mn_major ? launch_variant<true, true>(L, ta, tb, p) : launch_variant<true, false>(L, ta, tb, p);
+  return a.b_mn_major ? launch_variant<false, true>(L, ta, tb, p) : launch_variant<false, false>(L, ta, tb, p);
+}
+
+}  // namespace qarl

@@ -129,6 +129,21 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
   return d;
 }
 
+// Descriptor for an MN-major operand (the M or N index is the contiguous one in memory) staged
+// as 64-element column blocks: each block is what a TMA box of 64 elements (128 bytes) x R
+// k-rows with SWIZZLE_128B writes, i.e. groups of 8 k-rows 1024 bytes apart (stride byte
+// offset); the next 64-element block of the M/N index starts `lbo_bytes` further on (leading
+// byte offset).  Advancing K by 16 elements = 2 groups = +2048 bytes on the start address.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr >> 4) & 0x3FFF);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
 // Instruction descriptor for kind::f8f6f4 with e4m3 A and B (both K-major), fp32 D.
 __host__ __device__ constexpr uint32_t umma_idesc_e4m3_f32(int M, int N) {
   return (1u << 4)                              // D format: f32
@@ -146,6 +161,10 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N) {
          | (1u << 10)                           // B format: bf16
          | (static_cast<uint32_t>(N >> 3) << 17)
          | (static_cast<uint32_t>(M >> 4) << 24);
+}
+// The same with either operand MN-major (bit 15: A, bit 16: B).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32_major(int M, int N, bool a_mn, bool b_mn) {
+  return umma_idesc_bf16_f32(M, N) | (a_mn ? 1u << 15 : 0u) | (b_mn ? 1u << 16 : 0u);
 }
 // bf16 x bf16 -> fp32, K = 16 per instruction.
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
