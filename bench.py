@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-w4a16", action="store_true")
+    ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--tokens", type=int, default=M_TRAIN,
                     help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
                          "only; the reported config names the size)")
@@ -397,6 +398,41 @@ def main():
         }
         result["w4a16"] = w4
         del q13, q2, sets4, ws4
+
+    # ---------------- full-precision backward of the dense projection (QKV shape of the training configuration)
+    if not args.no_backward:
+        Mb, Nb, Kb = 8192, 5120, 2048
+        gen = torch.Generator(device=dev).manual_seed(3000 + rank)
+        dyb = torch.randn((Mb, Nb), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        xb = torch.randn((Mb, Kb), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        wb = (torch.randn((Nb, Kb), generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        bsteps = max(args.steps, 20)
+        for _ in range(3):
+            ctx.linear_bwd(dyb, xb, wb)
+        barrier()
+        ev0.record()
+        for _ in range(bsteps):
+            ctx.linear_bwd(dyb, xb, wb)
+        ev1.record()
+        barrier()
+        b_ms = max_over_ranks(ev0.elapsed_time(ev1)) / bsteps
+        ctx.profile_begin(max_marks=bsteps * 4 + 8)
+        for _ in range(bsteps):
+            ctx.linear_bwd(dyb, xb, wb)
+        bst = ctx.profile_end()
+        ctx.check_device_status()
+        fl = 2.0 * Mb * Nb * Kb
+        dx_ms = bst["bwd_dx"][0] / max(bst["bwd_dx"][1], 1)
+        dw_ms = bst["bwd_dw"][0] / max(bst["bwd_dw"][1], 1)
+        result["backward"] = {
+            "workload": (f"straight-through backward of the dense projection, M={Mb} N={Nb} K={Kb} (bf16 masters); "
+                         "213 MB of operands and results per step, larger than L2"),
+            "ms_per_step": b_ms, "dx_ms": dx_ms, "dw_ms": dw_ms,
+            "dx_tflops": fl / (dx_ms * 1e-3) / 1e12, "dw_tflops": fl / (dw_ms * 1e-3) / 1e12,
+            "dx_frac_bf16_peak_measured_burst": fl / (dx_ms * 1e-3) / 1e12 / pk["bf16_burst"],
+            "dw_frac_bf16_peak_measured_burst": fl / (dw_ms * 1e-3) / 1e12 / pk["bf16_burst"],
+        }
+        del dyb, xb, wb
 
     # ---------------- decode shape (rollout engine: weights already quantized)
     if not args.no_decode:

@@ -72,6 +72,16 @@ const char* qarl_last_cuda_error(qarl_ctx* ctx);
 int qarl_quantize_weight(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
                          uint8_t* codes, float* scales, void* stream);
 
+/* The same quantization, fused with publishing (Sec. 3.1 item 3: the low-bit tensors the
+ * training forward has just materialised are handed to the rollout engine as they are, with no
+ * second quantization pass).  pub_codes / pub_scales: a second destination of the same shapes,
+ * written from the same registers in the same launch -- the rollout engine's weight buffers:
+ * device memory of this GPU or peer-mapped memory of another one (plain stores).  Both NULL:
+ * identical to qarl_quantize_weight.  The two copies are bitwise equal by construction. */
+int qarl_quantize_weight_publish(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
+                                 uint8_t* codes, float* scales, uint8_t* pub_codes,
+                                 float* pub_scales, void* stream);
+
 /* Sec. 2.2 Quant, 1x128 groups along K.
  * in : x_bf16 device bf16 [M, K] with row stride ldx elements (ldx >= K, ldx % 8 == 0).
  * out: codes  device u8 [M, K] (dense);  scales device f32 [M, K/128]. */

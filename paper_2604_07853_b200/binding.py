@@ -31,7 +31,7 @@ EXPORTS = [
     "qarl_moe_workspace_bytes", "qarl_moe_fwd", "qarl_launch_count",
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
-    "qarl_moe_fwd_w4a16", "qarl_linear_bwd",
+    "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
@@ -108,6 +108,8 @@ def load() -> C.CDLL:
     L.qarl_moe_fwd_w4a16.restype = C.c_int
     L.qarl_moe_fwd_w4a16.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, sz,
                                      C.POINTER(MoeDebug), p]
+    L.qarl_quantize_weight_publish.restype = C.c_int
+    L.qarl_quantize_weight_publish.argtypes = [p, p, i64, i64, i64, p, p, p, p, p]
     L.qarl_linear_bwd.restype = C.c_int
     L.qarl_linear_bwd.argtypes = [p, p, p, p, i64, i64, i64, p, p, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
@@ -358,6 +360,14 @@ class Context:
                                                 _ptr(y), _ptr(ws), ws.numel(),
                                                 C.byref(dbg) if dbg is not None else None, _stream()))
         return (y, d) if debug else y
+
+    def quantize_weight_publish(self, w, codes, scales, pub_codes, pub_scales):
+        """quantize_weight writing a second, published copy of codes and scales in the same launch."""
+        assert w.dtype == torch.bfloat16 and w.is_cuda and w.is_contiguous()
+        E, N, K = (1, *w.shape) if w.dim() == 2 else w.shape
+        self._check(self.lib.qarl_quantize_weight_publish(self.h, _ptr(w), E, N, K, _ptr(codes), _ptr(scales),
+                                                          _ptr(pub_codes), _ptr(pub_scales), _stream()))
+        return codes, scales
 
     # ------------------------------------------------------------------ backward
     def linear_bwd(self, dy, x, w, want_dx_f32: bool = False, dx: bool = True, dw: bool = True):

@@ -167,7 +167,14 @@ int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches) {
 
 int qarl_quantize_weight(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* codes,
                          float* scales, void* stream) {
+  return qarl_quantize_weight_publish(ctx, w, E, N, K, codes, scales, nullptr, nullptr, stream);
+}
+
+int qarl_quantize_weight_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* codes,
+                                 float* scales, uint8_t* pub_codes, float* pub_scales, void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
+  if ((pub_codes == nullptr) != (pub_scales == nullptr)) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(pub_codes) || (reinterpret_cast<uintptr_t>(pub_scales) & 3u)) return QARL_ERR_MISALIGNED;
   if (N % kBlock || K % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E * (N / kBlock) * (K / kBlock) > 0x7FFFFFFFll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
@@ -175,7 +182,7 @@ int qarl_quantize_weight(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int
   if (!aligned16(w) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 3u)) return QARL_ERR_MISALIGNED;
   mark(ctx, static_cast<cudaStream_t>(stream), -1);
   cudaError_t e = launch_quantize_weight(make_launch(ctx, stream), static_cast<const uint16_t*>(w), E, N, K, codes,
-                                         scales);
+                                         scales, pub_codes, pub_scales);
   mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_WEIGHT);
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_weight");
 }

@@ -80,8 +80,10 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, 
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// pub_codes / pub_scales: optional second destination (the copy published to the rollout engine)
 cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
-                                   uint8_t* codes, float* scales);
+                                   uint8_t* codes, float* scales, uint8_t* pub_codes = nullptr,
+                                   float* pub_scales = nullptr);
 // dst_rows == nullptr: row m of the output is m.  Otherwise each input row t is written to
 // the `fanout` output rows dst_rows[t*fanout + j] (quantize once, scatter k times).
 // With dst_rows, pair_w [M*fanout] (the top-k weights by flat pair id) is scattered alongside

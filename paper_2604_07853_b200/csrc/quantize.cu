@@ -32,7 +32,9 @@ __device__ __forceinline__ void encode8(const uint4& v, float inv, uint32_t& c0,
 // reduction and the encode so the block is read from HBM once.
 __global__ void __launch_bounds__(256) quantize_weight_kernel(const uint16_t* __restrict__ w, int64_t N, int64_t K,
                                                               uint8_t* __restrict__ codes,
-                                                              float* __restrict__ scales) {
+                                                              float* __restrict__ scales,
+                                                              uint8_t* __restrict__ pub_codes,
+                                                              float* __restrict__ pub_scales) {
   pdl_trigger();
   pdl_wait();
   const int64_t kb = K / kBlock, nb = N / kBlock;
@@ -67,13 +69,18 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const uint16_t* __
 
   float inv;
   const float s = block_scale(bf16_bits_to_f32(m), &inv);
-  if (tid == 0) scales[blk] = s;
+  if (tid == 0) {
+    scales[blk] = s;
+    if (pub_scales) pub_scales[blk] = s;
+  }
 #pragma unroll
   for (int p = 0; p < 4; ++p) {
     uint4 out;
     encode8(v[p][0], inv, out.x, out.y);
     encode8(v[p][1], inv, out.z, out.w);
     *reinterpret_cast<uint4*>(codes + base + static_cast<int64_t>(r0 + 32 * p) * K) = out;
+    // the rollout engine's copy of the same tensors (Sec. 3.1 item 3), written from the same registers
+    if (pub_codes) *reinterpret_cast<uint4*>(pub_codes + base + static_cast<int64_t>(r0 + 32 * p) * K) = out;
   }
 }
 
@@ -248,11 +255,12 @@ __global__ void __launch_bounds__(256) scatter_rows_kernel(const uint16_t* __res
 }  // namespace
 
 cudaError_t launch_quantize_weight(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
-                                   uint8_t* codes, float* scales) {
+                                   uint8_t* codes, float* scales, uint8_t* pub_codes, float* pub_scales) {
   const int64_t blocks = E * (N / kBlock) * (K / kBlock);
   if (blocks == 0) return cudaSuccess;
   ++*L.launches;
-  return launch_pdl(quantize_weight_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, N, K, codes, scales);
+  return launch_pdl(quantize_weight_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, N, K, codes, scales,
+                    pub_codes, pub_scales);
 }
 
 cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, int64_t K, int64_t ldx,

@@ -94,3 +94,18 @@ def test_qkv_projection_shape_sampled(ctx):
     tol = 1e-3 * _norms(dy[:, feats], 0)[:, None] * _norms(x, 0)[None, :]
     g = dw32[torch.from_numpy(feats).cuda()].cpu().numpy().astype(np.float64)
     assert (np.abs(g - o_dw) <= tol).all()
+
+
+def test_quantize_weight_publish_writes_two_equal_copies(ctx):
+    """Sec. 3.1 item 3: the published tensors are the ones the training forward uses, bit for bit."""
+    rng = np.random.default_rng(9)
+    w = inputs.weight_bf16(rng, 3, 256, 384)
+    wt = bits_to_torch(w)
+    codes, scales = ctx.quantize_weight(wt)
+    c1, s1 = torch.zeros_like(codes), torch.zeros_like(scales)
+    c2, s2 = torch.zeros_like(codes), torch.zeros_like(scales)
+    ctx.quantize_weight_publish(wt, c1, s1, c2, s2)
+    assert torch.equal(c1, codes) and torch.equal(c2, codes)
+    assert torch.equal(s1, scales) and torch.equal(s2, scales)
+    oc, os_ = oracle.quantize_weight(w)
+    assert np.array_equal(c2.cpu().numpy(), oc) and np.array_equal(s2.cpu().numpy(), os_)
