@@ -59,6 +59,8 @@ def lib() -> C.CDLL:
         L.oracle_moe_w4a16.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p]
         L.oracle_linear_bwd.restype = None
         L.oracle_linear_bwd.argtypes = [p, p, p, i64, i64, i64, p, p, p]
+        L.oracle_tbpo.restype = None
+        L.oracle_tbpo.argtypes = [p, p, p, p, p, i64] + [C.c_double] * 4 + [p] * 6
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
     return _lib
@@ -288,3 +290,24 @@ def linear_bwd(dy_bits, x_bits, w_bits):
     dw32 = np.empty((N, K), dtype=np.float32)
     lib().oracle_linear_bwd(_ptr(dy), _ptr(x), _ptr(w), M, N, K, _ptr(dx32), _ptr(dx16), _ptr(dw32))
     return dx32, dx16, dw32
+
+
+# ---------------------------------------------------------------------------- TBPO
+TBPO_DEFAULTS = dict(eps_h=4e-4, delta_l=3e-4, delta_h=7e-4, cap=2.0)   # the paper's hyper-parameter table
+
+
+def tbpo(lp_cur, lp_old_learner, lp_old_sampler, offsets, adv, eps_h=4e-4, delta_l=3e-4, delta_h=7e-4, cap=2.0):
+    """Sequence-level TBPO surrogate over B packed responses (offsets int64 [B+1] into the flat
+    fp32 token arrays) -> dict(r, w, J float64 [B], flags int32 [B], grad fp32 [T], loss float)."""
+    a, b, c = (_c(v, np.float32) for v in (lp_cur, lp_old_learner, lp_old_sampler))
+    off, adv = _c(offsets, np.int64), _c(adv, np.float32)
+    B = adv.shape[0]
+    T = a.shape[0]
+    assert off.shape == (B + 1,) and off[0] == 0 and off[-1] == T and b.shape == c.shape == (T,)
+    r, w, J = (np.empty(B, dtype=np.float64) for _ in range(3))
+    flags = np.empty(B, dtype=np.int32)
+    grad = np.zeros(T, dtype=np.float32)
+    loss = np.zeros(1, dtype=np.float64)
+    lib().oracle_tbpo(_ptr(a), _ptr(b), _ptr(c), _ptr(off), _ptr(adv), B, eps_h, delta_l, delta_h, cap,
+                      _ptr(r), _ptr(w), _ptr(J), _ptr(flags), _ptr(grad), _ptr(loss))
+    return dict(r=r, w=w, J=J, flags=flags, grad=grad, loss=float(loss[0]))

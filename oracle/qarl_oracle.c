@@ -565,6 +565,66 @@ void oracle_linear_bwd(const uint16_t *dy, const uint16_t *x, const uint16_t *w,
     free(dyf);
 }
 
+
+/* =======================================================================================
+ * TBPO: the sequence-level surrogate of Sec. 3.2 ("Trust Band Policy Optimization"; ratio and
+ * weight as written out in the appendix "Detail of TBPO").  For a response o of L tokens:
+ *   a = (1/L) sum_t (log pi_current-learner - log pi_old-learner)(o_t),  r = exp(a)   (r_seq-prox)
+ *   b = (1/L) sum_t (log pi_old-learner - log pi_old-sampler)(o_t),      w = exp(b)   (w_seq-mismatch)
+ *   w~ = two-sided cap of w with c > 1 (Eq. "tis");  r~ = clip(r, 0, 1 + eps_h) if A >= 0,
+ *   clip(r, 1 - delta_l, 1 + delta_h) if A < 0 (Eq. "clip");  J = w~ r~ A.
+ * Readings: the cap is printed as clip(w, [-log c, log c]): taken in the log domain, i.e.
+ * w~ = exp(clip(b, -log c, log c)) in [1/c, c].  The batch objective is the mean of J over the B
+ * responses (the expectation over sampled responses), loss = -mean J.  A clipped r~ is a constant:
+ * the response then sends no gradient (the paper's "mask out the entire response"); bounds are
+ * inclusive (lo <= r <= hi passes the gradient).  w~ carries no gradient (neither old policy depends
+ * on theta).  Gradient of the loss with respect to every token log-prob of the current learner in
+ * response i:  -(1/B) w~ A r / L  if r is inside its band, else 0.  An empty response (L = 0)
+ * contributes J = 0 and still counts in B.  All arithmetic in double on fp32 inputs; the token
+ * differences are formed in double, summed in token order.
+ * flags: bit 0 = r outside its band (no gradient), bit 1 = w capped, bit 2 = empty response.
+ * ===================================================================================== */
+void oracle_tbpo(const float *lp_cur, const float *lp_old_learner, const float *lp_old_sampler,
+                 const int64_t *offsets, const float *adv, int64_t B,
+                 double eps_h, double delta_l, double delta_h, double cap,
+                 double *r_seq, double *w_seq, double *j_seq, int32_t *flags, float *grad, double *loss) {
+    double total = 0.0;
+    double logc = log(cap);
+    for (int64_t i = 0; i < B; ++i) {
+        int64_t t0 = offsets[i], t1 = offsets[i + 1], L = t1 - t0;
+        if (L <= 0) {
+            r_seq[i] = 1.0; w_seq[i] = 1.0; j_seq[i] = 0.0; flags[i] = 4;
+            continue;
+        }
+        double sa = 0.0, sb = 0.0;
+        for (int64_t t = t0; t < t1; ++t) {
+            sa += (double)lp_cur[t] - (double)lp_old_learner[t];
+            sb += (double)lp_old_learner[t] - (double)lp_old_sampler[t];
+        }
+        double a = sa / (double)L, b = sb / (double)L;
+        double r = exp(a), w = exp(b);
+        int f = 0;
+        double bc = b;
+        if (bc > logc) { bc = logc; f |= 2; }
+        if (bc < -logc) { bc = -logc; f |= 2; }
+        double wt = exp(bc);
+        double A = (double)adv[i];
+        double lo = A >= 0.0 ? 0.0 : 1.0 - delta_l;
+        double hi = A >= 0.0 ? 1.0 + eps_h : 1.0 + delta_h;
+        double rt = r;
+        if (rt < lo) { rt = lo; f |= 1; }
+        if (rt > hi) { rt = hi; f |= 1; }
+        double J = wt * rt * A;
+        r_seq[i] = r; w_seq[i] = w; j_seq[i] = J; flags[i] = f;
+        total += J;
+        if (grad) {
+            float g = (f & 1) ? 0.0f : (float)(-(wt * A * r) / ((double)L * (double)B));
+            for (int64_t t = t0; t < t1; ++t) grad[t] = g;
+        }
+    }
+    *loss = B > 0 ? -total / (double)B : 0.0;
+}
+
 /* Number of OpenMP threads the oracle will use (reported beside its timing). */
 #ifdef _OPENMP
 #include <omp.h>
