@@ -196,6 +196,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-w4a16", action="store_true")
     ap.add_argument("--no-backward", action="store_true")
+    ap.add_argument("--no-tbpo", action="store_true")
     ap.add_argument("--tokens", type=int, default=M_TRAIN,
                     help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
                          "only; the reported config names the size)")
@@ -433,6 +434,35 @@ def main():
             "dw_frac_bf16_peak_measured_burst": fl / (dw_ms * 1e-3) / 1e12 / pk["bf16_burst"],
         }
         del dyb, xb, wb
+
+    # ---------------- TBPO sequence-level loss over a packed batch of responses
+    if not args.no_tbpo:
+        from paper_2604_07853_b200 import inputs as gen_inputs
+        lens = gen_inputs.tbpo_lengths(4000 + rank, 4096)
+        tcase = [torch.from_numpy(a).to(dev) for a in gen_inputs.tbpo_case(4000 + rank, lens)]
+        Tt, Bt = int(tcase[0].shape[0]), int(tcase[4].shape[0])
+        tws = torch.empty(max(int(ctx.lib.qarl_tbpo_workspace_bytes(Bt, Tt)), 256), dtype=torch.uint8, device=dev)
+        tout = ctx.tbpo_loss(*tcase, workspace=tws)
+        tsteps = max(args.steps, 20)
+        for _ in range(3):
+            ctx.tbpo_loss(*tcase, out=tout, workspace=tws)
+        barrier()
+        ev0.record()
+        for _ in range(tsteps):
+            ctx.tbpo_loss(*tcase, out=tout, workspace=tws)
+        ev1.record()
+        barrier()
+        t_ms = max_over_ranks(ev0.elapsed_time(ev1)) / tsteps
+        ctx.check_device_status()
+        tbytes = 16 * Tt + 8 * (Bt + 1) + 4 * Bt + 28 * Bt
+        result["tbpo"] = {
+            "workload": f"TBPO loss + per-token gradient, {Bt} packed responses, {Tt} tokens (lognormal lengths, <= 16384); "
+                        f"{tbytes / 1e6:.0f} MB per step, larger than L2",
+            "ms_per_step": t_ms, "tokens_per_s": world * Tt / (t_ms * 1e-3),
+            "algorithmic_bytes": tbytes, "gbs": tbytes / (t_ms * 1e-3) / 1e9,
+            "frac_hbm_measured": tbytes / (t_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "launches_per_step": 4,
+        }
+        del tcase, tout, tws
 
     # ---------------- decode shape (rollout engine: weights already quantized)
     if not args.no_decode:

@@ -243,6 +243,36 @@ int qarl_linear_bwd(qarl_ctx* ctx, const void* dy_bf16, const void* x_bf16, cons
                     int64_t M, int64_t N, int64_t K, void* dx_bf16, float* dx_f32, float* dw_f32,
                     void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * TBPO: the sequence-level surrogate of Sec. 3.2 over B packed responses (ratio and weight as
+ * written out in the appendix "Detail of TBPO").  Response i owns tokens
+ * [offsets[i], offsets[i+1]) of the flat arrays (offsets monotone, offsets[0] = 0,
+ * offsets[B] = T; prompt and padding tokens are simply not in the arrays).  With L its length:
+ *   a = (1/L) sum_t (lp_cur - lp_old_learner)[t]          r = exp(a)    r_seq-prox
+ *   b = (1/L) sum_t (lp_old_learner - lp_old_sampler)[t]  w = exp(b)    w_seq-mismatch
+ *   w~ = exp(clip(b, -log cap, log cap))                  (two-sided cap, taken in the log domain)
+ *   r~ = clip(r, 0, 1 + eps_h)            if adv[i] >= 0
+ *        clip(r, 1 - delta_l, 1 + delta_h) if adv[i] <  0
+ *   J = w~ r~ adv[i];   loss = -(1/B) sum_i J;
+ *   grad[t] = d loss / d lp_cur[t] = -(w~ adv r) / (L B) if r lies inside its band (bounds
+ *   inclusive), else 0: a response outside its band is masked from the update.
+ * An empty response has r = w = 1, J = 0 and counts in B.  All arithmetic in double on the fp32
+ * inputs, every sum in a fixed order (results do not depend on the grid).
+ * in : lp_* f32 [T], offsets i64 [B+1], adv f32 [B]: device pointers.  params: host struct
+ *      (the paper's table: eps_h 4e-4, delta_l 3e-4, delta_h 7e-4, cap 2).
+ * out: r_seq, w_seq, j_seq f64 [B]; flags i32 [B] (bit 0: r outside its band, bit 1: w capped,
+ *      bit 2: empty); grad f32 [T] (NULL: skipped); loss f64 [1]: device pointers, caller-owned.
+ * workspace: qarl_tbpo_workspace_bytes(B, T) bytes, 256-byte aligned. */
+typedef struct {
+  double eps_h, delta_l, delta_h, cap;
+} qarl_tbpo_params;
+size_t qarl_tbpo_workspace_bytes(int64_t B, int64_t T);
+int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learner,
+                   const float* lp_old_sampler, const int64_t* offsets, const float* adv, int64_t B,
+                   int64_t T, const qarl_tbpo_params* params, double* r_seq, double* w_seq,
+                   double* j_seq, int32_t* flags, float* grad, double* loss, void* workspace,
+                   size_t workspace_bytes, void* stream);
+
 /* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
  * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
  * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;
@@ -260,7 +290,8 @@ enum {
   QARL_STAGE_COMBINE = 6,
   QARL_STAGE_BWD_DX = 7,
   QARL_STAGE_BWD_DW = 8,
-  QARL_NUM_STAGES = 9
+  QARL_STAGE_TBPO = 9,
+  QARL_NUM_STAGES = 10
 };
 int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
 int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);

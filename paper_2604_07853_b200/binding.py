@@ -32,11 +32,12 @@ EXPORTS = [
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
+    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
-          "combine", "bwd_dx", "bwd_dw"]
+          "combine", "bwd_dx", "bwd_dw", "tbpo"]
 
 
 class QarlError(RuntimeError):
@@ -44,6 +45,10 @@ class QarlError(RuntimeError):
         self.status = status
         name = STATUS_NAMES.get(status, str(status))
         super().__init__(f"{name}{': ' + detail if detail else ''}")
+
+
+class TbpoParams(C.Structure):
+    _fields_ = [("eps_h", C.c_double), ("delta_l", C.c_double), ("delta_h", C.c_double), ("cap", C.c_double)]
 
 
 class MoeDebug(C.Structure):
@@ -110,6 +115,10 @@ def load() -> C.CDLL:
                                      C.POINTER(MoeDebug), p]
     L.qarl_quantize_weight_publish.restype = C.c_int
     L.qarl_quantize_weight_publish.argtypes = [p, p, i64, i64, i64, p, p, p, p, p]
+    L.qarl_tbpo_workspace_bytes.restype = sz
+    L.qarl_tbpo_workspace_bytes.argtypes = [i64, i64]
+    L.qarl_tbpo_loss.restype = C.c_int
+    L.qarl_tbpo_loss.argtypes = [p, p, p, p, p, p, i64, i64, C.POINTER(TbpoParams), p, p, p, p, p, p, p, sz, p]
     L.qarl_linear_bwd.restype = C.c_int
     L.qarl_linear_bwd.argtypes = [p, p, p, p, i64, i64, i64, p, p, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
@@ -384,3 +393,26 @@ class Context:
         self._check(self.lib.qarl_linear_bwd(self.h, _ptr(dy), _ptr(x), _ptr(w), M, N, K, _ptr(dxo), _ptr(dx32),
                                              _ptr(dwo), _stream()))
         return dxo, dx32, dwo
+
+    # ------------------------------------------------------------------ TBPO
+    def tbpo_loss(self, lp_cur, lp_old_learner, lp_old_sampler, offsets, adv, eps_h=4e-4, delta_l=3e-4,
+                  delta_h=7e-4, cap=2.0, want_grad: bool = True, out=None, workspace=None):
+        """Sequence-level TBPO surrogate over B packed responses -> dict(r, w, J f64 [B], flags i32 [B],
+        grad f32 [T] or None, loss f64 [1]) of device tensors.  out: an earlier result to overwrite."""
+        for t in (lp_cur, lp_old_learner, lp_old_sampler, adv):
+            assert t.dtype == torch.float32 and t.is_cuda and t.is_contiguous()
+        assert offsets.dtype == torch.int64 and offsets.is_cuda
+        B, T = adv.shape[0], lp_cur.shape[0]
+        dev = lp_cur.device
+        if out is None:
+            out = dict(r=torch.empty(B, dtype=torch.float64, device=dev), w=torch.empty(B, dtype=torch.float64, device=dev),
+                       J=torch.empty(B, dtype=torch.float64, device=dev), flags=torch.empty(B, dtype=torch.int32, device=dev),
+                       grad=torch.empty(T, dtype=torch.float32, device=dev) if want_grad else None,
+                       loss=torch.empty(1, dtype=torch.float64, device=dev))
+        ws = workspace if workspace is not None else self.workspace(max(int(self.lib.qarl_tbpo_workspace_bytes(B, T)), 256))
+        prm = TbpoParams(eps_h, delta_l, delta_h, cap)
+        self._check(self.lib.qarl_tbpo_loss(self.h, _ptr(lp_cur), _ptr(lp_old_learner), _ptr(lp_old_sampler),
+                                            _ptr(offsets), _ptr(adv), B, T, C.byref(prm), _ptr(out["r"]), _ptr(out["w"]),
+                                            _ptr(out["J"]), _ptr(out["flags"]), _ptr(out["grad"]), _ptr(out["loss"]),
+                                            _ptr(ws), ws.numel(), _stream()))
+        return out

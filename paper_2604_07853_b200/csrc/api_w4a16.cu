@@ -239,4 +239,45 @@ int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w,
   return QARL_OK;
 }
 
+size_t qarl_tbpo_workspace_bytes(int64_t B, int64_t T) {
+  if (B < 0 || T < 0) return 0;
+  return tbpo_workspace_bytes(B, T);
+}
+
+int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learner, const float* lp_old_sampler,
+                   const int64_t* offsets, const float* adv, int64_t B, int64_t T, const qarl_tbpo_params* prm,
+                   double* r_seq, double* w_seq, double* j_seq, int32_t* flags, float* grad, double* loss,
+                   void* workspace, size_t workspace_bytes, void* stream) {
+  if (!ctx || B < 0 || T < 0 || !prm || !loss) return QARL_ERR_INVALID_ARG;
+  if (!(prm->cap > 1.0) || prm->eps_h < 0.0 || prm->delta_l < 0.0 || prm->delta_h < 0.0) return QARL_ERR_INVALID_ARG;
+  if (B > 0x7FFFFF00ll || T / 2048 > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (B > 0 && (!offsets || !adv || !r_seq || !w_seq || !j_seq || !flags || !workspace)) return QARL_ERR_INVALID_ARG;
+  if (T > 0 && (!lp_cur || !lp_old_learner || !lp_old_sampler)) return QARL_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return QARL_ERR_MISALIGNED;
+  if (workspace_bytes < tbpo_workspace_bytes(B, T)) return QARL_ERR_WORKSPACE_TOO_SMALL;
+  TbpoArgs a{};
+  a.lp_cur = lp_cur;
+  a.lp_old_learner = lp_old_learner;
+  a.lp_old_sampler = lp_old_sampler;
+  a.offsets = offsets;
+  a.adv = adv;
+  a.B = B;
+  a.T = T;
+  a.eps_h = prm->eps_h;
+  a.delta_l = prm->delta_l;
+  a.delta_h = prm->delta_h;
+  a.cap = prm->cap;
+  a.r_seq = r_seq;
+  a.w_seq = w_seq;
+  a.j_seq = j_seq;
+  a.flags = flags;
+  a.grad = grad;
+  a.loss = loss;
+  a.workspace = workspace;
+  mark(ctx, static_cast<cudaStream_t>(stream), -1);
+  cudaError_t e = launch_tbpo(make_launch(ctx, stream), a);
+  mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_TBPO);
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "tbpo_loss");
+}
+
 }  // extern "C"

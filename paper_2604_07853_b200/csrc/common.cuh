@@ -177,6 +177,26 @@ struct GemmBf16Args {
 };
 cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err);
 
+// ---- TBPO sequence-level loss ------------------------------------------------------------------
+struct TbpoArgs {
+  const float* lp_cur;
+  const float* lp_old_learner;
+  const float* lp_old_sampler;
+  const int64_t* offsets;  // [B + 1]
+  const float* adv;        // [B]
+  int64_t B, T;
+  double eps_h, delta_l, delta_h, cap;
+  double* r_seq;
+  double* w_seq;
+  double* j_seq;
+  int32_t* flags;
+  float* grad;             // [T] or nullptr
+  double* loss;
+  void* workspace;
+};
+size_t tbpo_workspace_bytes(int64_t B, int64_t T);
+cudaError_t launch_tbpo(const Launch& L, const TbpoArgs& a);
+
 }  // namespace qarl
 
 // The opaque context of the C ABI (one per device).

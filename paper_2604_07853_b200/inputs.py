@@ -141,3 +141,30 @@ def config3() -> MoeCase:
 def config4(m: int = 32768) -> MoeCase:
     """MoE FFN layer at the training-forward shape: M = 32768, Zipf(1.1) popularity."""
     return moe_case(4, m, zipf_s=1.1)
+
+
+# --------------------------------------------------------------------------- TBPO loss inputs
+def tbpo_case(seed: int, lengths, drift: float = 5e-4, mismatch: float = 0.02):
+    """Packed per-token log-probs of B responses with the given lengths (a list/array of ints,
+    zeros allowed): the old sampler's (negative, heavy towards small magnitudes), the old
+    learner's = sampler + N(0, mismatch) (quantized-rollout mismatch), the current learner's =
+    old learner + a per-response shift N(0, drift) + token noise N(0, 2 drift) (one optimizer
+    step away, so that the sequence ratios straddle the 1e-3-wide trust bands), and
+    group-normalized-looking advantages N(0, 1).  Returns fp32 arrays and int64 offsets."""
+    rng = np.random.default_rng(seed)
+    lengths = np.asarray(lengths, dtype=np.int64)
+    off = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    T = int(off[-1])
+    smp = (-np.abs(rng.normal(0.0, 1.5, size=T)) - 0.01).astype(np.float32)
+    old = (smp + rng.normal(0.0, mismatch, size=T)).astype(np.float32)
+    shift = np.repeat(rng.normal(0.0, drift, size=len(lengths)), lengths)
+    cur = (old + shift + rng.normal(0.0, 2 * drift, size=T)).astype(np.float32)
+    adv = rng.normal(0.0, 1.0, size=len(lengths)).astype(np.float32)
+    return cur, old, smp, off, adv
+
+
+def tbpo_lengths(seed: int, b: int, mean_len: int = 4096, max_len: int = 16384) -> np.ndarray:
+    """Response lengths: lognormal around mean_len (sigma 0.8), clipped to [16, max_len]."""
+    rng = np.random.default_rng(seed)
+    l = rng.lognormal(np.log(mean_len) - 0.32, 0.8, size=b)
+    return np.clip(l, 16, max_len).astype(np.int64)
