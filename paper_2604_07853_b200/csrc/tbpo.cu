@@ -5,15 +5,15 @@
 //   w~ = exp(clip(b, -log c, log c));  r~ = clip(r, 0, 1 + eps_h) if A >= 0 else clip(r, 1 - delta_l, 1 + delta_h)
 //   J = w~ r~ A;   loss = -mean_i J;   d loss / d lp_cur[t] = -(w~ A r) / (L B) if r is inside its band, else 0.
 // HBM-bound: 12 bytes read and 4 written per token.  The token axis is cut into fixed chunks
-// of 2048 tokens so that the work is balanced whatever the response lengths are:
-//   map      (thread per response)  first[k] = the response that holds token 2048 k; empty responses are finished here
+// of 8192 tokens so that the work is balanced whatever the response lengths are:
+//   map      (thread per response)  first[k] = the response that holds token 8192 k; empty responses are finished here
 //   partial  (CTA per chunk)        for every response that overlaps the chunk, the sums of the two token
 //                                   differences over the overlap, in double, to slot (response + chunk)
 //                                   -- unique, because both indices only grow along the token axis
-//   finish   (CTA per chunk)        per overlapping response: add its partials in chunk order, form r, w, J,
-//                                   flags in double; the chunk that holds the response's first token stores
-//                                   them; every chunk writes the gradient of its own tokens
-//   loss     (one CTA)              -mean J in a fixed order
+//   stats    (thread per response)  add the response's partials in chunk order, form r, w, J, flags and the
+//                                   gradient value its tokens share, in double; the last CTA to finish adds
+//                                   all J in index order: loss = -mean J
+//   grad     (CTA per chunk)        streams the per-response gradient value over the response's tokens
 // Every sum has a fixed order: results do not depend on the grid or on timing.
 #include <math.h>
 
@@ -22,7 +22,8 @@
 namespace qarl {
 namespace {
 
-constexpr int kChunk = 2048;
+constexpr int kChunk = 8192;
+constexpr int kSub = 2048;  // tokens per pass of a CTA: 8 per thread, loads issued together
 constexpr int kThreads = 256;
 
 struct TbpoParams {
@@ -41,6 +42,8 @@ struct TbpoParams {
   double* loss;
   int32_t* first;    // [nchunks]
   double2* partial;  // [B + nchunks]
+  float* gval;       // [B] gradient value shared by the response's tokens
+  unsigned int* ticket;  // CTAs of the stats kernel that have finished
 };
 
 __device__ __forceinline__ int64_t clamp_off(const TbpoParams& p, int64_t i) {
@@ -51,6 +54,7 @@ __global__ void __launch_bounds__(kThreads) tbpo_map_kernel(const TbpoParams p) 
   pdl_trigger();
   pdl_wait();
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i == 0) *p.ticket = 0;
   if (i >= p.B) return;
   const int64_t t0 = clamp_off(p, i), t1 = clamp_off(p, i + 1);
   if (t1 <= t0) {  // empty response: J = 0, still counted in B
@@ -58,6 +62,7 @@ __global__ void __launch_bounds__(kThreads) tbpo_map_kernel(const TbpoParams p) 
     p.w_seq[i] = 1.0;
     p.j_seq[i] = 0.0;
     p.flags[i] = 4;
+    p.gval[i] = 0.0f;
     return;
   }
   for (int64_t k = (t0 + kChunk - 1) / kChunk; k * kChunk < t1; ++k) p.first[k] = static_cast<int32_t>(i);
@@ -95,27 +100,83 @@ __global__ void __launch_bounds__(kThreads) tbpo_partial_kernel(const TbpoParams
     if (t0 >= hi) break;
     const int64_t s0 = max(t0, lo), s1 = min(clamp_off(p, i + 1), hi);
     double2 acc = make_double2(0.0, 0.0);
-    // up to 8 tokens per thread with the loads issued together
-    float c[8], o[8], q[8];
+    for (int64_t base = s0; base < s1; base += kSub) {
+      float c[8], o[8], q[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int64_t t = s0 + threadIdx.x + u * kThreads;
-      const bool in = t < s1;
-      c[u] = in ? __ldg(p.lp_cur + t) : 0.0f;
-      o[u] = in ? __ldg(p.lp_old + t) : 0.0f;
-      q[u] = in ? __ldg(p.lp_smp + t) : 0.0f;
-    }
+      for (int u = 0; u < 8; ++u) {
+        const int64_t t = base + threadIdx.x + u * kThreads;
+        const bool in = t < s1;
+        c[u] = in ? __ldg(p.lp_cur + t) : 0.0f;
+        o[u] = in ? __ldg(p.lp_old + t) : 0.0f;
+        q[u] = in ? __ldg(p.lp_smp + t) : 0.0f;
+      }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {  // differences formed in double: exact
-      acc.x += static_cast<double>(c[u]) - static_cast<double>(o[u]);
-      acc.y += static_cast<double>(o[u]) - static_cast<double>(q[u]);
+      for (int u = 0; u < 8; ++u) {  // differences formed in double: exact
+        acc.x += static_cast<double>(c[u]) - static_cast<double>(o[u]);
+        acc.y += static_cast<double>(o[u]) - static_cast<double>(q[u]);
+      }
     }
     const double2 s = block_sum(acc, warp_part);
     if (threadIdx.x == 0 && s1 > s0) p.partial[i + k] = s;
   }
 }
 
-__global__ void __launch_bounds__(kThreads) tbpo_finish_kernel(const TbpoParams p) {
+__global__ void __launch_bounds__(kThreads) tbpo_stats_kernel(const TbpoParams p) {
+  __shared__ double part[kThreads];
+  __shared__ bool last;
+  pdl_trigger();
+  pdl_wait();
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < p.B) {
+    const int64_t t0 = clamp_off(p, i), t1 = clamp_off(p, i + 1);
+    if (t1 > t0) {
+      double sa = 0.0, sb = 0.0;
+      for (int64_t kk = t0 / kChunk; kk * kChunk < t1; ++kk) {  // the response's partials in chunk order
+        const double2 v = p.partial[i + kk];
+        sa += v.x;
+        sb += v.y;
+      }
+      const double L = static_cast<double>(t1 - t0);
+      const double a = sa / L, b = sb / L;
+      const double r = exp(a);
+      int f = 0;
+      double bc = b;
+      if (bc > p.log_cap) { bc = p.log_cap; f |= 2; }
+      if (bc < -p.log_cap) { bc = -p.log_cap; f |= 2; }
+      const double wt = exp(bc);
+      const double A = static_cast<double>(__ldg(p.adv + i));
+      const double band_lo = A >= 0.0 ? 0.0 : 1.0 - p.delta_l;
+      const double band_hi = A >= 0.0 ? 1.0 + p.eps_h : 1.0 + p.delta_h;
+      double rt = r;
+      if (rt < band_lo) { rt = band_lo; f |= 1; }
+      if (rt > band_hi) { rt = band_hi; f |= 1; }
+      p.r_seq[i] = r;
+      p.w_seq[i] = (f & 2) ? exp(b) : wt;
+      p.j_seq[i] = wt * rt * A;
+      p.flags[i] = f;
+      p.gval[i] = (f & 1) ? 0.0f : static_cast<float>(-(wt * A * r) / (L * static_cast<double>(p.B)));
+    }
+  }
+  // The last CTA to get here adds every J in one fixed order (thread j takes j, j + 256, ...; then a
+  // tree): which CTA that is varies, what it computes does not.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  double s = 0.0;
+  for (int64_t j = threadIdx.x; j < p.B; j += kThreads) s += __ldcg(p.j_seq + j);
+  part[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = kThreads / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *p.loss = -part[0] / static_cast<double>(p.B);
+}
+
+__global__ void __launch_bounds__(kThreads) tbpo_grad_kernel(const TbpoParams p) {
   pdl_trigger();
   pdl_wait();
   const int64_t k = blockIdx.x;
@@ -123,66 +184,39 @@ __global__ void __launch_bounds__(kThreads) tbpo_finish_kernel(const TbpoParams 
   for (int64_t i = min(max(static_cast<int64_t>(p.first[k]), int64_t(0)), p.B - 1); i < p.B; ++i) {
     const int64_t t0 = clamp_off(p, i);
     if (t0 >= hi) break;
-    const int64_t t1 = clamp_off(p, i + 1);
-    if (t1 <= t0) continue;  // empty responses lie between others on the token axis
-    const int64_t s0 = max(t0, lo), s1 = min(t1, hi);
+    const int64_t s0 = max(t0, lo), s1 = min(clamp_off(p, i + 1), hi);
     if (s1 <= s0) continue;
-    // every thread adds the response's partials in chunk order (a handful of L2 hits)
-    double sa = 0.0, sb = 0.0;
-    for (int64_t kk = t0 / kChunk; kk * kChunk < t1; ++kk) {
-      const double2 v = p.partial[i + kk];
-      sa += v.x;
-      sb += v.y;
-    }
-    const double L = static_cast<double>(t1 - t0);
-    const double a = sa / L, b = sb / L;
-    const double r = exp(a);
-    int f = 0;
-    double bc = b;
-    if (bc > p.log_cap) { bc = p.log_cap; f |= 2; }
-    if (bc < -p.log_cap) { bc = -p.log_cap; f |= 2; }
-    const double wt = exp(bc);
-    const double A = static_cast<double>(__ldg(p.adv + i));
-    const double band_lo = A >= 0.0 ? 0.0 : 1.0 - p.delta_l;
-    const double band_hi = A >= 0.0 ? 1.0 + p.eps_h : 1.0 + p.delta_h;
-    double rt = r;
-    if (rt < band_lo) { rt = band_lo; f |= 1; }
-    if (rt > band_hi) { rt = band_hi; f |= 1; }
-    if (threadIdx.x == 0 && s0 == t0) {  // this chunk holds the response's first token
-      p.r_seq[i] = r;
-      p.w_seq[i] = exp(b);
-      p.j_seq[i] = wt * rt * A;
-      p.flags[i] = f;
-    }
-    if (p.grad) {
-      const float g = (f & 1) ? 0.0f : static_cast<float>(-(wt * A * r) / (L * static_cast<double>(p.B)));
-      for (int64_t t = s0 + threadIdx.x; t < s1; t += kThreads) p.grad[t] = g;
-    }
+    const float g = __ldg(p.gval + i);
+    for (int64_t t = s0 + threadIdx.x; t < s1; t += kThreads) p.grad[t] = g;
   }
 }
 
-__global__ void __launch_bounds__(1024) tbpo_loss_kernel(const TbpoParams p) {
-  __shared__ double part[1024];
+__global__ void tbpo_zero_loss_kernel(const TbpoParams p) {
   pdl_trigger();
   pdl_wait();
-  double s = 0.0;
-  for (int64_t i = threadIdx.x; i < p.B; i += 1024) s += p.j_seq[i];
-  part[threadIdx.x] = s;
-  __syncthreads();
-  for (int o = 512; o > 0; o >>= 1) {
-    if (threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) *p.loss = p.B > 0 ? -part[0] / static_cast<double>(p.B) : 0.0;
+  *p.loss = 0.0;
 }
 
 }  // namespace
 
-size_t tbpo_workspace_bytes(int64_t B, int64_t T) {
+namespace {
+struct TbpoWs {
+  size_t first, partial, gval, ticket, total;
+};
+TbpoWs tbpo_plan(int64_t B, int64_t T) {
   const int64_t nchunks = (T + kChunk - 1) / kChunk;
-  const size_t first = (static_cast<size_t>(nchunks) * sizeof(int32_t) + 255) / 256 * 256;
-  return first + static_cast<size_t>(B + nchunks) * sizeof(double2);
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  TbpoWs w{};
+  w.first = 0;
+  w.partial = up(static_cast<size_t>(nchunks) * sizeof(int32_t));
+  w.gval = w.partial + up(static_cast<size_t>(B + nchunks) * sizeof(double2));
+  w.ticket = w.gval + up(static_cast<size_t>(B) * sizeof(float));
+  w.total = w.ticket + 256;
+  return w;
 }
+}  // namespace
+
+size_t tbpo_workspace_bytes(int64_t B, int64_t T) { return tbpo_plan(B, T).total; }
 
 cudaError_t launch_tbpo(const Launch& L, const TbpoArgs& a) {
   TbpoParams p{};
@@ -204,25 +238,33 @@ cudaError_t launch_tbpo(const Launch& L, const TbpoArgs& a) {
   p.grad = a.grad;
   p.loss = a.loss;
   const int64_t nchunks = (a.T + kChunk - 1) / kChunk;
-  p.first = static_cast<int32_t*>(a.workspace);
-  p.partial = reinterpret_cast<double2*>(static_cast<uint8_t*>(a.workspace) +
-                                         (static_cast<size_t>(nchunks) * sizeof(int32_t) + 255) / 256 * 256);
-  cudaError_t e = cudaSuccess;
-  if (a.B > 0) {
+  const TbpoWs w = tbpo_plan(a.B, a.T);
+  uint8_t* ws = static_cast<uint8_t*>(a.workspace);
+  p.first = reinterpret_cast<int32_t*>(ws + w.first);
+  p.partial = reinterpret_cast<double2*>(ws + w.partial);
+  p.gval = reinterpret_cast<float*>(ws + w.gval);
+  p.ticket = reinterpret_cast<unsigned int*>(ws + w.ticket);
+  if (a.B == 0) {  // no responses: the loss of an empty batch is 0
     ++*L.launches;
-    e = launch_pdl(tbpo_map_kernel, static_cast<unsigned>((a.B + kThreads - 1) / kThreads), kThreads, 0, L.stream, p);
-    if (e != cudaSuccess) return e;
+    return launch_pdl(tbpo_zero_loss_kernel, 1u, 1u, 0, L.stream, p);
   }
-  if (nchunks > 0 && a.B > 0) {
+  const unsigned resp_blocks = static_cast<unsigned>((a.B + kThreads - 1) / kThreads);
+  ++*L.launches;
+  cudaError_t e = launch_pdl(tbpo_map_kernel, resp_blocks, kThreads, 0, L.stream, p);
+  if (e != cudaSuccess) return e;
+  if (nchunks > 0) {
     ++*L.launches;
     e = launch_pdl(tbpo_partial_kernel, static_cast<unsigned>(nchunks), kThreads, 0, L.stream, p);
     if (e != cudaSuccess) return e;
-    ++*L.launches;
-    e = launch_pdl(tbpo_finish_kernel, static_cast<unsigned>(nchunks), kThreads, 0, L.stream, p);
-    if (e != cudaSuccess) return e;
   }
   ++*L.launches;
-  return launch_pdl(tbpo_loss_kernel, 1u, 1024u, 0, L.stream, p);
+  e = launch_pdl(tbpo_stats_kernel, resp_blocks, kThreads, 0, L.stream, p);
+  if (e != cudaSuccess) return e;
+  if (nchunks > 0 && a.grad) {
+    ++*L.launches;
+    e = launch_pdl(tbpo_grad_kernel, static_cast<unsigned>(nchunks), kThreads, 0, L.stream, p);
+  }
+  return e;
 }
 
 }  // namespace qarl
