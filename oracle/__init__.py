@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
         L.oracle_linear_bwd.argtypes = [p, p, p, i64, i64, i64, p, p, p]
         L.oracle_tbpo.restype = None
         L.oracle_tbpo.argtypes = [p, p, p, p, p, i64] + [C.c_double] * 4 + [p] * 6
+        L.oracle_router_topk.restype = None
+        L.oracle_router_topk.argtypes = [p, i64, i64, i64, p, p]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
     return _lib
@@ -311,3 +313,23 @@ def tbpo(lp_cur, lp_old_learner, lp_old_sampler, offsets, adv, eps_h=4e-4, delta
     lib().oracle_tbpo(_ptr(a), _ptr(b), _ptr(c), _ptr(off), _ptr(adv), B, eps_h, delta_l, delta_h, cap,
                       _ptr(r), _ptr(w), _ptr(J), _ptr(flags), _ptr(grad), _ptr(loss))
     return dict(r=r, w=w, J=J, flags=flags, grad=grad, loss=float(loss[0]))
+
+
+# ---------------------------------------------------------------------------- router
+def router_topk(logits, k: int):
+    """fp32 logits [M, E] -> (ids int32 [M, k] in descending-logit order, ties to the lower id;
+    weights fp32 [M, k] = softmax over the selected logits)."""
+    l = _c(logits, np.float32)
+    M, E = l.shape
+    assert 1 <= k <= E
+    ids = np.empty((M, k), dtype=np.int32)
+    wts = np.empty((M, k), dtype=np.float32)
+    lib().oracle_router_topk(_ptr(l), M, E, k, _ptr(ids), _ptr(wts))
+    return ids, wts
+
+
+def router(x_bits, w_router_bits, k: int):
+    """Router forward: logits = x . W_r^T (bf16 operands, exact sum -> fp32), then router_topk."""
+    logits, _ = linear_bf16(x_bits, w_router_bits)
+    ids, wts = router_topk(logits, k)
+    return logits, ids, wts

@@ -625,6 +625,36 @@ void oracle_tbpo(const float *lp_cur, const float *lp_old_learner, const float *
     *loss = B > 0 ? -total / (double)B : 0.0;
 }
 
+
+/* =======================================================================================
+ * Router of the MoE block ("router shift", Sec. 4.2: the routing decision is part of the forward
+ * the sampler and the learner must agree on).  The paper gives no formula; reading (the common
+ * top-k softmax router of the Qwen3-MoE family the paper trains): logits = x . W_r^T on bf16
+ * operands (exact sum, rounded once to fp32); the k largest logits of a token, ties to the lower
+ * expert id, in descending order; weights = softmax over the k selected fp32 logits (exp of
+ * logit - max in double, normalised, rounded to fp32).  The router stays in bf16: it is not
+ * quantized.
+ * ===================================================================================== */
+void oracle_router_topk(const float *logits, int64_t M, int64_t E, int64_t k, int32_t *ids, float *wts) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        const float *l = logits + m * E;
+        char *taken = (char *)calloc((size_t)E, 1);
+        double mx = 0.0, den = 0.0;
+        for (int64_t j = 0; j < k; ++j) {
+            int64_t best = -1;
+            for (int64_t e = 0; e < E; ++e)
+                if (!taken[e] && (best < 0 || l[e] > l[best])) best = e;   /* strict >: ties keep the lower id */
+            taken[best] = 1;
+            ids[m * k + j] = (int32_t)best;
+            if (j == 0) mx = (double)l[best];
+        }
+        for (int64_t j = 0; j < k; ++j) den += exp((double)l[ids[m * k + j]] - mx);
+        for (int64_t j = 0; j < k; ++j) wts[m * k + j] = (float)(exp((double)l[ids[m * k + j]] - mx) / den);
+        free(taken);
+    }
+}
+
 /* Number of OpenMP threads the oracle will use (reported beside its timing). */
 #ifdef _OPENMP
 #include <omp.h>
