@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--no-w4a16", action="store_true")
     ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--no-tbpo", action="store_true")
+    ap.add_argument("--no-router", action="store_true")
     ap.add_argument("--tokens", type=int, default=M_TRAIN,
                     help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
                          "only; the reported config names the size)")
@@ -325,6 +326,30 @@ def main():
                            "frac_fp8_peak_nominal_4500": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12 / 4500.0},
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches * world, "clocks": clocks,
     }
+
+    # ---------------- router (bf16 logits GEMM + top-k softmax) on the training batch
+    if not args.no_router:
+        gen = torch.Generator(device=dev).manual_seed(5000 + rank)
+        wr = (torch.randn((E, H), generator=gen, device=dev, dtype=torch.float32) * 0.05).to(torch.bfloat16)
+        rsteps = max(args.steps, 20)
+        for _ in range(3):
+            ctx.router_fwd(x, wr, TOPK)
+        barrier()
+        ev0.record()
+        for _ in range(rsteps):
+            ctx.router_fwd(x, wr, TOPK)
+        ev1.record()
+        barrier()
+        r_ms = max_over_ranks(ev0.elapsed_time(ev1)) / rsteps
+        ctx.check_device_status()
+        rbytes = M_TRAIN * H * 2 + E * H * 2 + 2 * M_TRAIN * E * 4 + M_TRAIN * TOPK * 8
+        result["router"] = {
+            "workload": f"router forward, M={M_TRAIN} H={H} E={E} top-{TOPK} (bf16 logits GEMM + top-k softmax, 2 launches)",
+            "ms_per_step": r_ms, "tokens_per_s": world * M_TRAIN / (r_ms * 1e-3),
+            "algorithmic_bytes": rbytes, "gbs": rbytes / (r_ms * 1e-3) / 1e9,
+            "frac_hbm_measured": rbytes / (r_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+        }
+        del wr
 
     # ---------------- W4A16 variant of the same layer (4-bit weights, bf16 activations)
     if not args.no_w4a16:

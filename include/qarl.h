@@ -273,6 +273,22 @@ int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learn
                    double* j_seq, int32_t* flags, float* grad, double* loss, void* workspace,
                    size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * Router of the MoE block (the paper names the "router shift" between sampler and learner,
+ * Sec. 4.2, but gives no formula; this is the top-k softmax router of the model family it
+ * trains).  The router is not quantized:
+ *   logits[m, e] = sum_h x[m, h] W_r[e, h]   bf16 operands, fp32 accumulation in a fixed order
+ *   topk_ids[m, :]     the k largest logits of token m in descending order, ties to the lower id
+ *   topk_weights[m, :] softmax over those k logits (fp32)
+ * in : x_bf16 [M, H], w_router_bf16 [E, H]: device, 16-byte aligned; H % 8 == 0, E % 8 == 0,
+ *      E <= 1024, 1 <= k <= min(E, 32).
+ * out: logits_f32 [M, E] (required: it is the GEMM's output buffer), topk_ids i32 [M, k],
+ *      topk_weights f32 [M, k]; caller-owned.  The outputs feed qarl_moe_fwd directly.
+ * A token's routing depends only on that token's row of x: bitwise the same for any M. */
+int qarl_router_fwd(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H,
+                    const void* w_router_bf16, int64_t E, int64_t k, float* logits_f32,
+                    int32_t* topk_ids, float* topk_weights, void* stream);
+
 /* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
  * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
  * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;
@@ -291,7 +307,8 @@ enum {
   QARL_STAGE_BWD_DX = 7,
   QARL_STAGE_BWD_DW = 8,
   QARL_STAGE_TBPO = 9,
-  QARL_NUM_STAGES = 10
+  QARL_STAGE_ROUTER = 10,
+  QARL_NUM_STAGES = 11
 };
 int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
 int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);

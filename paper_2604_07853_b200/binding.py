@@ -32,12 +32,12 @@ EXPORTS = [
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
-    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss",
+    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
-          "combine", "bwd_dx", "bwd_dw", "tbpo"]
+          "combine", "bwd_dx", "bwd_dw", "tbpo", "router"]
 
 
 class QarlError(RuntimeError):
@@ -119,6 +119,8 @@ def load() -> C.CDLL:
     L.qarl_tbpo_workspace_bytes.argtypes = [i64, i64]
     L.qarl_tbpo_loss.restype = C.c_int
     L.qarl_tbpo_loss.argtypes = [p, p, p, p, p, p, i64, i64, C.POINTER(TbpoParams), p, p, p, p, p, p, p, sz, p]
+    L.qarl_router_fwd.restype = C.c_int
+    L.qarl_router_fwd.argtypes = [p, p, i64, i64, p, i64, i64, p, p, p, p]
     L.qarl_linear_bwd.restype = C.c_int
     L.qarl_linear_bwd.argtypes = [p, p, p, p, i64, i64, i64, p, p, p, p]
     L.qarl_harness_rmsnorm.restype = C.c_int
@@ -416,3 +418,16 @@ class Context:
                                             _ptr(out["J"]), _ptr(out["flags"]), _ptr(out["grad"]), _ptr(out["loss"]),
                                             _ptr(ws), ws.numel(), _stream()))
         return out
+
+    # ------------------------------------------------------------------ router
+    def router_fwd(self, x, w_router, k: int):
+        """x bf16 [M, H], w_router bf16 [E, H] -> (logits f32 [M, E], ids i32 [M, k], weights f32 [M, k])."""
+        assert x.dtype == torch.bfloat16 and w_router.dtype == torch.bfloat16 and x.is_contiguous() and w_router.is_contiguous()
+        M, H = x.shape
+        E = w_router.shape[0]
+        logits = torch.empty((M, E), dtype=torch.float32, device=x.device)
+        ids = torch.empty((M, k), dtype=torch.int32, device=x.device)
+        wts = torch.empty((M, k), dtype=torch.float32, device=x.device)
+        self._check(self.lib.qarl_router_fwd(self.h, _ptr(x), M, H, _ptr(w_router), E, k, _ptr(logits), _ptr(ids),
+                                             _ptr(wts), _stream()))
+        return logits, ids, wts

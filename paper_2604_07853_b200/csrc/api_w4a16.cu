@@ -280,4 +280,32 @@ int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learn
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "tbpo_loss");
 }
 
+int qarl_router_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, const void* wr, int64_t E, int64_t k,
+                    float* logits, int32_t* ids, float* wts, void* stream) {
+  if (!ctx || M < 0 || H <= 0 || E <= 0 || k < 1 || k > 32 || k > E) return QARL_ERR_INVALID_ARG;
+  if (H % 8 || E % 8 || E > 1024 || M > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (M == 0) return QARL_OK;
+  if (!x || !wr || !logits || !ids || !wts) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(wr) || !aligned16(logits)) return QARL_ERR_MISALIGNED;
+  Launch L = make_launch(ctx, stream);
+  GemmBf16Args a{};
+  a.a = static_cast<const uint16_t*>(x);   // A(m, h) = x[m, h]
+  a.b = static_cast<const uint16_t*>(wr);  // B(e, h) = W_r[e, h]
+  a.Mo = M;
+  a.No = E;
+  a.Kc = H;
+  a.c_f32 = logits;
+  CUresult cu = CUDA_SUCCESS;
+  mark(ctx, L.stream, -1);
+  cudaError_t e = launch_gemm_bf16(L, ctx->encode, a, &cu);
+  if (cu != CUDA_SUCCESS) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+    return QARL_ERR_CUDA;
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "router logits");
+  if ((e = launch_router_topk(L, logits, M, E, k, ids, wts)) != cudaSuccess) return cuda_fail(ctx, e, "router top-k");
+  mark(ctx, L.stream, QARL_STAGE_ROUTER);
+  return QARL_OK;
+}
+
 }  // extern "C"

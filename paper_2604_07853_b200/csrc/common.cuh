@@ -177,6 +177,10 @@ struct GemmBf16Args {
 };
 cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err);
 
+// fp32 logits [M, E] -> top-k ids (descending, ties to the lower id) and softmax weights over the selection
+cudaError_t launch_router_topk(const Launch& L, const float* logits, int64_t M, int64_t E, int64_t k, int32_t* ids,
+                               float* wts);
+
 // ---- TBPO sequence-level loss ------------------------------------------------------------------
 struct TbpoArgs {
   const float* lp_cur;

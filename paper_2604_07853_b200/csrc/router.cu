@@ -1,0 +1,83 @@
+// Router of the MoE block: top-k experts of every token from its fp32 logits (ties to the lower
+// expert id, descending order) and the softmax over the selected logits.  One warp per token; lane l
+// keeps experts l, l + 32, ... in registers; k rounds of a warp arg-max.  The logits come from the
+// bf16 tensor-core GEMM (x . W_r^T, fp32 accumulation in a fixed order), so a token's routing
+// depends only on that token's row -- the same invariance the expert GEMMs have (App. C).
+#include <math.h>
+
+#include "common.cuh"
+
+namespace qarl {
+namespace {
+
+constexpr int kMaxPerLane = 32;  // E <= 1024
+
+__global__ void __launch_bounds__(256) router_topk_kernel(const float* __restrict__ logits, int64_t M, int E, int k,
+                                                          int32_t* __restrict__ ids, float* __restrict__ wts) {
+  pdl_trigger();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t m = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  if (m >= M) return;
+  const float* row = logits + m * E;
+  float v[kMaxPerLane];
+  const int per = (E + 31) / 32;
+#pragma unroll
+  for (int j = 0; j < kMaxPerLane; ++j) {
+    const int e = lane + 32 * j;
+    v[j] = (j < per && e < E) ? row[e] : -INFINITY;
+  }
+  uint32_t taken = 0;  // bit j: this lane's j-th expert was selected
+  float sel = 0.0f;    // lane j < k ends up holding the j-th selected logit
+  int sel_id = 0;
+  for (int r = 0; r < k; ++r) {
+    float best = -INFINITY;
+    int best_e = 0x7FFFFFFF;
+#pragma unroll
+    for (int j = 0; j < kMaxPerLane; ++j) {
+      if (j < per && !((taken >> j) & 1u)) {
+        const int e = lane + 32 * j;
+        if (e < E && (v[j] > best || best_e == 0x7FFFFFFF)) {  // ascending e within a lane: strict > keeps the lower id
+          best = v[j];
+          best_e = e;
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+      const int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, o);
+      if (oe != 0x7FFFFFFF && (best_e == 0x7FFFFFFF || ob > best || (ob == best && oe < best_e))) {
+        best = ob;
+        best_e = oe;
+      }
+    }
+    if ((best_e & 31) == lane) taken |= 1u << (best_e >> 5);
+    if (lane == r) {
+      sel = best;
+      sel_id = best_e;
+    }
+  }
+  // softmax over the k selected logits, in double: exp(l - max) / sum, rounded to fp32
+  const double mx = static_cast<double>(__shfl_sync(0xFFFFFFFFu, sel, 0));
+  double ex = lane < k ? exp(static_cast<double>(sel) - mx) : 0.0;
+  double den = ex;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+  if (lane < k) {
+    ids[m * k + lane] = sel_id;
+    wts[m * k + lane] = static_cast<float>(ex / den);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_router_topk(const Launch& L, const float* logits, int64_t M, int64_t E, int64_t k, int32_t* ids,
+                               float* wts) {
+  if (M == 0) return cudaSuccess;
+  ++*L.launches;
+  return launch_pdl(router_topk_kernel, static_cast<unsigned>((M * 32 + 255) / 256), 256, 0, L.stream, logits, M,
+                    static_cast<int>(E), static_cast<int>(k), ids, wts);
+}
+
+}  // namespace qarl
