@@ -10,8 +10,9 @@
 namespace qarl {
 namespace {
 
-constexpr int kMaxPerLane = 32;  // E <= 1024
-
+// PER = experts per lane (E <= 32 PER), a compile-time bound so that the selection loops unroll to
+// exactly the work the expert count needs.
+template <int PER>
 __global__ void __launch_bounds__(256) router_topk_kernel(const float* __restrict__ logits, int64_t M, int E, int k,
                                                           int32_t* __restrict__ ids, float* __restrict__ wts) {
   pdl_trigger();
@@ -20,12 +21,11 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const float* __restric
   const int64_t m = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   if (m >= M) return;
   const float* row = logits + m * E;
-  float v[kMaxPerLane];
-  const int per = (E + 31) / 32;
+  float v[PER];
 #pragma unroll
-  for (int j = 0; j < kMaxPerLane; ++j) {
+  for (int j = 0; j < PER; ++j) {
     const int e = lane + 32 * j;
-    v[j] = (j < per && e < E) ? row[e] : -INFINITY;
+    v[j] = e < E ? row[e] : -INFINITY;
   }
   uint32_t taken = 0;  // bit j: this lane's j-th expert was selected
   float sel = 0.0f;    // lane j < k ends up holding the j-th selected logit
@@ -34,8 +34,8 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const float* __restric
     float best = -INFINITY;
     int best_e = 0x7FFFFFFF;
 #pragma unroll
-    for (int j = 0; j < kMaxPerLane; ++j) {
-      if (j < per && !((taken >> j) & 1u)) {
+    for (int j = 0; j < PER; ++j) {
+      if (!((taken >> j) & 1u)) {
         const int e = lane + 32 * j;
         if (e < E && (v[j] > best || best_e == 0x7FFFFFFF)) {  // ascending e within a lane: strict > keeps the lower id
           best = v[j];
@@ -76,8 +76,15 @@ cudaError_t launch_router_topk(const Launch& L, const float* logits, int64_t M, 
                                float* wts) {
   if (M == 0) return cudaSuccess;
   ++*L.launches;
-  return launch_pdl(router_topk_kernel, static_cast<unsigned>((M * 32 + 255) / 256), 256, 0, L.stream, logits, M,
-                    static_cast<int>(E), static_cast<int>(k), ids, wts);
+  const unsigned grid = static_cast<unsigned>((M * 32 + 255) / 256);
+  const int Ei = static_cast<int>(E), ki = static_cast<int>(k);
+  const int per = static_cast<int>((E + 31) / 32);
+  if (per <= 1) return launch_pdl(router_topk_kernel<1>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
+  if (per <= 2) return launch_pdl(router_topk_kernel<2>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
+  if (per <= 4) return launch_pdl(router_topk_kernel<4>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
+  if (per <= 8) return launch_pdl(router_topk_kernel<8>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
+  if (per <= 16) return launch_pdl(router_topk_kernel<16>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
+  return launch_pdl(router_topk_kernel<32>, grid, 256, 0, L.stream, logits, M, Ei, ki, ids, wts);
 }
 
 }  // namespace qarl
