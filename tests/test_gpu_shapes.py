@@ -54,3 +54,29 @@ def test_argument_limits_are_rejected(ctx):
     with pytest.raises(binding.QarlError) as ei:
         ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s)                     # k = 33 > 32
     assert ei.value.status == -1
+
+
+def test_argument_limits_of_the_widened_entry_points(ctx):
+    """Bad shapes come back as status codes before anything is launched."""
+    bf = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.quantize_weight_w4(bf(1, 100, 128))                 # N % 128 != 0
+    assert ei.value.status == -2
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.quantize_weight_w4(bf(1, 128, 192))                 # K % 128 != 0
+    assert ei.value.status == -2
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.linear_bwd(bf(4, 12), bf(4, 16), bf(12, 16))         # N % 8 != 0
+    assert ei.value.status == -2
+    f32 = lambda *s: torch.zeros(s, dtype=torch.float32, device="cuda")
+    off = torch.tensor([0, 4], dtype=torch.int64, device="cuda")
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.tbpo_loss(f32(4), f32(4), f32(4), off, f32(1), cap=1.0)   # the cap must exceed 1
+    assert ei.value.status == -1
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.router_fwd(bf(4, 64), bf(8, 64), 9)                  # k > E
+    assert ei.value.status == -1
+    with pytest.raises(binding.QarlError) as ei:
+        ctx.router_fwd(bf(4, 64), bf(1032, 64), 8)               # E > 1024
+    assert ei.value.status == -2
+    assert ctx.poll() == 0
