@@ -243,6 +243,20 @@ int qarl_linear_bwd(qarl_ctx* ctx, const void* dy_bf16, const void* x_bf16, cons
                     int64_t M, int64_t N, int64_t K, void* dx_bf16, float* dx_f32, float* dw_f32,
                     void* stream);
 
+/* The same backward for an expert projection of the MoE layer, on the forward's expert-sorted row
+ * layout (expert e owns rows offsets[e] .. offsets[e+1]-1 of dy and x; offsets i32 [E+1] on the
+ * device, as qarl_moe_fwd's debug output expert_offsets gives them):
+ *   dX[p, k]   = sum_n dY[p, n] W_e[n, k]   for the expert e that owns row p   -> dx_bf16 / dx_f32 [P, K]
+ *   dW_e[n, k] = sum over the expert's rows p of dY[p, n] X[p, k]              -> dw_f32 [E, N, K]
+ * in : dy_bf16 [P, N], x_bf16 [P, K], w_bf16 [E, N, K] (masters); N % 64 == 0, K % 8 == 0,
+ *      1 <= E <= 1024.  An expert without rows gets dW_e = 0.  Outputs may be skipped as in
+ * qarl_linear_bwd.  No padding, no copies, no workspace; fixed accumulation order (a row of dX
+ * depends only on that row of dY; dW_e adds its rows in sorted order). */
+int qarl_grouped_linear_bwd(qarl_ctx* ctx, const void* dy_bf16, const void* x_bf16,
+                            const void* w_bf16, const int32_t* offsets, int64_t P, int64_t N,
+                            int64_t K, int64_t E, void* dx_bf16, float* dx_f32, float* dw_f32,
+                            void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * TBPO: the sequence-level surrogate of Sec. 3.2 over B packed responses (ratio and weight as
  * written out in the appendix "Detail of TBPO").  Response i owns tokens

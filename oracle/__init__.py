@@ -333,3 +333,19 @@ def router(x_bits, w_router_bits, k: int):
     logits, _ = linear_bf16(x_bits, w_router_bits)
     ids, wts = router_topk(logits, k)
     return logits, ids, wts
+
+
+def grouped_linear_bwd(dy_bits, x_bits, w_bits, offsets):
+    """linear_bwd per expert on expert-sorted rows: dy [P, N], x [P, K], w [E, N, K], offsets [E+1]
+    -> (dX fp32 [P, K], dX bf16 bits, dW fp32 [E, N, K]); an expert without rows has dW = 0."""
+    dy, x, w = _c(dy_bits, np.uint16), _c(x_bits, np.uint16), _c(w_bits, np.uint16)
+    P, K = x.shape
+    E, N, _ = w.shape
+    dx32 = np.zeros((P, K), dtype=np.float32)
+    dx16 = np.zeros((P, K), dtype=np.uint16)
+    dw32 = np.zeros((E, N, K), dtype=np.float32)
+    for e in range(E):
+        a, b = int(offsets[e]), int(offsets[e + 1])
+        if b > a:
+            dx32[a:b], dx16[a:b], dw32[e] = linear_bwd(dy[a:b], x[a:b], w[e])
+    return dx32, dx16, dw32

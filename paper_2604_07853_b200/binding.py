@@ -32,7 +32,7 @@ EXPORTS = [
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
-    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd",
+    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
@@ -119,6 +119,8 @@ def load() -> C.CDLL:
     L.qarl_tbpo_workspace_bytes.argtypes = [i64, i64]
     L.qarl_tbpo_loss.restype = C.c_int
     L.qarl_tbpo_loss.argtypes = [p, p, p, p, p, p, i64, i64, C.POINTER(TbpoParams), p, p, p, p, p, p, p, sz, p]
+    L.qarl_grouped_linear_bwd.restype = C.c_int
+    L.qarl_grouped_linear_bwd.argtypes = [p, p, p, p, p, i64, i64, i64, i64, p, p, p, p]
     L.qarl_router_fwd.restype = C.c_int
     L.qarl_router_fwd.argtypes = [p, p, i64, i64, p, i64, i64, p, p, p, p]
     L.qarl_linear_bwd.restype = C.c_int
@@ -394,6 +396,21 @@ class Context:
         dwo = torch.empty((N, K), dtype=torch.float32, device=dy.device) if dw else None
         self._check(self.lib.qarl_linear_bwd(self.h, _ptr(dy), _ptr(x), _ptr(w), M, N, K, _ptr(dxo), _ptr(dx32),
                                              _ptr(dwo), _stream()))
+        return dxo, dx32, dwo
+
+    def grouped_linear_bwd(self, dy, x, w, offsets, want_dx_f32: bool = False, dx: bool = True, dw: bool = True):
+        """Backward of an expert projection on expert-sorted rows: dy [P, N], x [P, K], w [E, N, K] bf16,
+        offsets i32 [E+1] -> (dX bf16 [P, K] or None, dX fp32 or None, dW fp32 [E, N, K] or None)."""
+        for t in (dy, x, w):
+            assert t.dtype == torch.bfloat16 and t.is_cuda and t.is_contiguous()
+        assert offsets.dtype == torch.int32 and offsets.is_cuda
+        P, N = dy.shape
+        E, _, K = w.shape
+        dxo = torch.empty((P, K), dtype=torch.bfloat16, device=w.device) if dx else None
+        dx32 = torch.empty((P, K), dtype=torch.float32, device=w.device) if (dx and want_dx_f32) else None
+        dwo = torch.empty((E, N, K), dtype=torch.float32, device=w.device) if dw else None
+        self._check(self.lib.qarl_grouped_linear_bwd(self.h, _ptr(dy), _ptr(x), _ptr(w), _ptr(offsets), P, N, K, E,
+                                                     _ptr(dxo), _ptr(dx32), _ptr(dwo), _stream()))
         return dxo, dx32, dwo
 
     # ------------------------------------------------------------------ TBPO

@@ -239,6 +239,68 @@ int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w,
   return QARL_OK;
 }
 
+int qarl_grouped_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w, const int32_t* offsets,
+                            int64_t P, int64_t N, int64_t K, int64_t E, void* dx, float* dx_f32, float* dw_f32,
+                            void* stream) {
+  if (!ctx || P < 0 || N <= 0 || K <= 0 || E < 1) return QARL_ERR_INVALID_ARG;
+  if (N % 64 || K % 8 || E > 1024 || P > 0x7FFFFF00ll || E * N > 0x7FFFFF00ll || E * K > 0x7FFFFF00ll)
+    return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (!w || !offsets || (P > 0 && (!dy || !x))) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(w) || !aligned16(dx) || !aligned16(dx_f32) || !aligned16(dw_f32))
+    return QARL_ERR_MISALIGNED;
+  Launch L = make_launch(ctx, stream);
+  CUresult cu = CUDA_SUCCESS;
+  auto run = [&](const GemmBf16Args& a, const char* what) {
+    cudaError_t e = launch_gemm_bf16(L, ctx->encode, a, &cu);
+    if (cu != CUDA_SUCCESS) {
+      snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+      return static_cast<int>(QARL_ERR_CUDA);
+    }
+    return e == cudaSuccess ? static_cast<int>(QARL_OK) : cuda_fail(ctx, e, what);
+  };
+  mark(ctx, L.stream, -1);
+  if ((dx || dx_f32) && P > 0) {
+    GemmBf16Args a{};
+    a.group = 1;
+    a.a = static_cast<const uint16_t*>(dy);  // A(p, n) = dY[p, n]
+    a.b = static_cast<const uint16_t*>(w);   // B_e(k, n) = W_e[n, k]: stored [n][k], MN-major
+    a.b_mn_major = true;
+    a.Mo = P;
+    a.No = K;
+    a.Kc = N;
+    a.E = E;
+    a.offsets = offsets;
+    a.c_bf16 = static_cast<uint16_t*>(dx);
+    a.c_f32 = dx_f32;
+    const int rc = run(a, "grouped_linear_bwd dX");
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_BWD_DX);
+  }
+  if (dw_f32) {
+    if (P == 0) {  // no rows at all: every dW_e is zero
+      cudaError_t e = cudaMemsetAsync(dw_f32, 0, static_cast<size_t>(E) * N * K * sizeof(float), L.stream);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "grouped_linear_bwd dW");
+      return QARL_OK;
+    }
+    GemmBf16Args a{};
+    a.group = 2;
+    a.a = static_cast<const uint16_t*>(dy);  // A(n, p) = dY[p, n]
+    a.a_mn_major = true;
+    a.b = static_cast<const uint16_t*>(x);   // B(k, p) = X[p, k]
+    a.b_mn_major = true;
+    a.Mo = N;
+    a.No = K;
+    a.E = E;
+    a.offsets = offsets;
+    a.rows_total = P;
+    a.c_f32 = dw_f32;
+    const int rc = run(a, "grouped_linear_bwd dW");
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_BWD_DW);
+  }
+  return QARL_OK;
+}
+
 size_t qarl_tbpo_workspace_bytes(int64_t B, int64_t T) {
   if (B < 0 || T < 0) return 0;
   return tbpo_workspace_bytes(B, T);

@@ -174,6 +174,15 @@ struct GemmBf16Args {
   int64_t Mo, No, Kc;
   uint16_t* c_bf16;    // [Mo, No] or nullptr
   float* c_f32;        // [Mo, No] or nullptr
+  // group = 0: dense.
+  // group = 1 (grouped rows): A [Mo = P rows, Kc] K-major in expert-sorted order, B [E, Kc, No] (MN-major) or
+  //   [E, No, Kc] (K-major); row p uses the B of the expert that owns it; C [P, No]; Kc % 64 == 0.
+  // group = 2 (grouped contraction): A [rows_total, Mo] and B [rows_total, No], both MN-major, expert-sorted
+  //   rows; C [E, Mo, No], C_e = sum over the expert's rows of A[p, :]^T B[p, :] (zeros for an empty expert).
+  int group = 0;
+  const int32_t* offsets = nullptr;  // [E + 1], device
+  int64_t E = 1;
+  int64_t rows_total = 0;
 };
 cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err);
 

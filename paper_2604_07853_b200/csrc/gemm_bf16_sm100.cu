@@ -11,6 +11,17 @@
 //   dX[m, k] = sum_n dY[m, n] W[n, k]:  A = dY (K-major),  B = W  (MN-major, [c = n][j = k])
 //   dW[n, k] = sum_m dY[m, n] X[m, k]:  A = dY (MN-major, [c = m][i = n]),  B = X (MN-major)
 //
+// Two grouped forms serve the expert GEMMs of the MoE layer, both on the forward's expert-sorted
+// row layout (expert e owns rows offsets[e] .. offsets[e+1]-1), with no padding and no copies:
+//   grouped rows         C[p, :] = A[p, :] . B_e  for the expert e that owns row p  (dX of an
+//                        expert projection: A = dY sorted, K-major; B = W [E, N, K], MN-major)
+//   grouped contraction  C_e = sum over the expert's rows p of A[p, :]^T B[p, :]  (dW of an
+//                        expert projection: both operands MN-major, the contraction runs over a
+//                        ragged row range).  The last 64-row step of an expert also holds rows of
+//                        the next expert: the MMA warp overwrites those rows of the staged A tile
+//                        with zeros (generic stores + proxy fence) before it issues the step, so
+//                        they contribute nothing whatever B holds there.
+//
 // Tile 128 x 256 x 64.  TMA stages both operands with the 128-byte swizzle (a K-major tile is
 // one box of R rows x 128 bytes; an MN-major tile is one box of 64 c-rows x 128 bytes per 64
 // output indices); one thread issues 4 x tcgen05.mma kind::f16 (128 x 256 x 16) per stage with
@@ -22,6 +33,7 @@
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "sched.cuh"
 
 namespace qarl {
 namespace {
@@ -40,9 +52,14 @@ constexpr uint32_t kBBytes = BN * BK * 2;   // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kBlockBytes = 64 * BK * 2;  // one MN-major block: 64 output indices x 64 c-rows
 constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxExperts = 1024;
+enum { kDense = 0, kGroupedRows = 1, kGroupedContraction = 2 };
 
 struct Bf16Params {
-  int Mo, No, Kc;
+  int Mo, No, Kc;           // grouped rows: Mo = total rows P;  grouped contraction: Kc unused (from offsets)
+  const int32_t* offsets;   // [E + 1] (grouped forms)
+  int E;
+  int rows_total;           // grouped contraction: P
   uint16_t* c_bf16;   // [Mo, No] or nullptr
   float* c_f32;       // [Mo, No] or nullptr
   int* status;
@@ -56,6 +73,8 @@ struct __align__(8) SmemTail {
   uint64_t tmem_empty[kAccBufs];
   uint32_t tmem_addr;
   int abort_flag;
+  int32_t off[kMaxExperts + 1];
+  int32_t prefix[kMaxExperts + 1];
 };
 constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + sizeof(SmemTail);
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
@@ -81,7 +100,7 @@ __device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&b);
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int GROUP>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const Bf16Params p) {
@@ -112,14 +131,61 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     tmem_relinquish();
   }
   pdl_wait();
+  const int n_tiles = (p.No + BN - 1) / BN;
+  const int m_tiles = GROUP == kGroupedRows ? 0 : (p.Mo + BM - 1) / BM;
+  if (GROUP == kGroupedRows) {
+    build_tile_list(s->off, s->prefix, p.offsets, p.Mo, p.E, BM, n_tiles);
+  } else if (GROUP == kGroupedContraction) {
+    for (int e = threadIdx.x; e <= p.E; e += kThreads) s->off[e] = min(max(p.offsets[e], 0), p.rows_total);
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = s->tmem_addr;
-  const int m_tiles = (p.Mo + BM - 1) / BM, n_tiles = (p.No + BN - 1) / BN;
-  const int total_tiles = m_tiles * n_tiles;
-  const int KS = (p.Kc + BK - 1) / BK;  // a ragged last step reads zeros (TMA out-of-range fill)
+  const int total_tiles = GROUP == kGroupedRows ? s->prefix[p.E]
+                        : GROUP == kGroupedContraction ? p.E * m_tiles * n_tiles : m_tiles * n_tiles;
   const int grid = gridDim.x;
+
+  // Everything a role needs to know about tile T.  i0 / j0: first output row / column; a_c0 / b_c0:
+  // first contraction coordinate of A / B; KS: 64-element contraction steps; last_valid: contraction
+  // elements of the last step that belong to this tile (64 = all); row_end: end of the rows that
+  // may be stored; c_off: element offset of this tile's output matrix.
+  struct Tile {
+    int i0, j0, a_c0, b_c0, KS, last_valid, row_end;
+    int64_t c_off;
+    int b_row0;  // K-major B: first row of the expert's block
+  };
+  auto tile_of = [&](int T, int& cur_e) {
+    Tile t{};
+    t.last_valid = BK;
+    if (GROUP == kDense) {
+      t.i0 = (T % m_tiles) * BM;
+      t.j0 = (T / m_tiles) * BN;
+      t.KS = (p.Kc + BK - 1) / BK;  // a ragged last step reads zeros (TMA out-of-range fill)
+      t.row_end = p.Mo;
+    } else if (GROUP == kGroupedRows) {
+      const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+      t.i0 = c.m0;
+      t.j0 = c.n_tile * BN;
+      t.KS = p.Kc / BK;             // Kc is a multiple of 64 here: a step never runs into the next expert's weights
+      t.a_c0 = 0;
+      t.b_c0 = c.e * p.Kc;          // MN-major B: the expert's [Kc, No] block starts at row e Kc
+      t.b_row0 = c.e * p.No;        // K-major B: the expert's [No, Kc] block starts at row e No
+      t.row_end = c.m_end;
+    } else {
+      const int per_e = m_tiles * n_tiles;
+      const int e = T / per_e, r = T % per_e;
+      t.i0 = (r % m_tiles) * BM;
+      t.j0 = (r / m_tiles) * BN;
+      const int rows = s->off[e + 1] - s->off[e];
+      t.KS = (rows + BK - 1) / BK;
+      t.last_valid = rows - (t.KS - 1) * BK;
+      t.a_c0 = t.b_c0 = s->off[e];
+      t.row_end = p.Mo;
+      t.c_off = static_cast<int64_t>(e) * p.Mo * p.No;
+    }
+    return t;
+  };
 
   if (warp == kTmaWarp) {
     if (lane == 0) {
@@ -127,9 +193,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       uint32_t phase = 0;
       uint32_t armed = 0, armed_parity = 0;
       bool ok = true;
+      int cur_e = 0;
       for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
-        const int i0 = (T % m_tiles) * BM, j0 = (T / m_tiles) * BN;
-        for (int ks = 0; ks < KS; ++ks) {
+        const Tile t = tile_of(T, cur_e);
+        const int i0 = t.i0, j0 = t.j0;
+        for (int ks = 0; ks < t.KS; ++ks) {
           if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
           uint8_t* b_dst = a_dst + kABytes;
@@ -137,16 +205,16 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           if (A_MN) {
 #pragma unroll
             for (int b = 0; b < BM / 64; ++b)
-              tma_load_2d(a_dst + b * kBlockBytes, &tm_a, &s->full[stage], i0 + 64 * b, ks * BK);
+              tma_load_2d(a_dst + b * kBlockBytes, &tm_a, &s->full[stage], i0 + 64 * b, t.a_c0 + ks * BK);
           } else {
-            tma_load_2d(a_dst, &tm_a, &s->full[stage], ks * BK, i0);
+            tma_load_2d(a_dst, &tm_a, &s->full[stage], t.a_c0 + ks * BK, i0);
           }
           if (B_MN) {
 #pragma unroll
             for (int b = 0; b < BN / 64; ++b)
-              tma_load_2d(b_dst + b * kBlockBytes, &tm_b, &s->full[stage], j0 + 64 * b, ks * BK);
+              tma_load_2d(b_dst + b * kBlockBytes, &tm_b, &s->full[stage], j0 + 64 * b, t.b_c0 + ks * BK);
           } else {
-            tma_load_2d(b_dst, &tm_b, &s->full[stage], ks * BK, j0);
+            tma_load_2d(b_dst, &tm_b, &s->full[stage], ks * BK, t.b_row0 + j0);
           }
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
@@ -159,18 +227,35 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       }
     }
   } else if (warp == kMmaWarp) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32_major(BM, BN, A_MN, B_MN);
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
-        if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
-        for (int ks = 0; ks < KS; ++ks) {
-          if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
+    // The whole warp follows the pipeline (so that it can zero the overhang rows of a ragged
+    // contraction step together); lane 0 issues the MMAs and commits.
+    constexpr uint32_t idesc = umma_idesc_bf16_f32_major(BM, BN, A_MN, B_MN);
+    int stage = 0, acc = 0;
+    uint32_t phase = 0, acc_phase = 0;
+    bool ok = true;
+    int cur_e = 0;
+    for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
+      const Tile t = tile_of(T, cur_e);
+      if (t.KS == 0) continue;  // an expert without rows: the epilogue writes zeros, no accumulator is used
+      if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+      for (int ks = 0; ks < t.KS; ++ks) {
+        if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
+        uint8_t* a_tile = smem + static_cast<size_t>(stage) * kStageBytes;
+        if (GROUP == kGroupedContraction && ks == t.KS - 1 && t.last_valid < BK) {
+          // rows last_valid .. 63 of both 64-column blocks of A belong to the next expert: make them zero
+          const int nrows = BK - t.last_valid;
+          for (int idx = lane; idx < 2 * nrows * 8; idx += 32) {
+            const int blk = idx / (nrows * 8), rem = idx % (nrows * 8);
+            *reinterpret_cast<uint4*>(a_tile + blk * kBlockBytes + (t.last_valid + rem / 8) * 128 + (rem % 8) * 16) =
+                make_uint4(0, 0, 0, 0);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncwarp();
+        if (lane == 0) {
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
+          const uint32_t a_addr = smem_u32(a_tile);
           const uint32_t b_addr = a_addr + kABytes;
           const uint64_t a_desc = A_MN ? umma_desc_mn_sw128(a_addr, kBlockBytes) : umma_desc_k_sw128(a_addr);
           const uint64_t b_desc = B_MN ? umma_desc_mn_sw128(b_addr, kBlockBytes) : umma_desc_k_sw128(b_addr);
@@ -182,24 +267,30 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           for (int k4 = 0; k4 < BK / 16; ++k4)
             umma_bf16(d_tmem, a_desc + a_step * k4, b_desc + b_step * k4, idesc, (ks > 0 || k4 > 0) ? 1u : 0u);
           umma_commit(&s->empty[stage]);
-          if (ks == KS - 1) umma_commit(&s->tmem_full[acc]);
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
+          if (ks == t.KS - 1) umma_commit(&s->tmem_full[acc]);
         }
-        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+        __syncwarp();
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
+      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
     }
   } else if (warp < kEpiWarps) {
     const int r = warp * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
     int acc = 0;
     uint32_t acc_phase = 0;
+    int cur_e = 0;
     for (int T = blockIdx.x; T < total_tiles; T += grid) {
-      const int i0 = (T % m_tiles) * BM, j0 = (T / m_tiles) * BN;
+      const Tile t = tile_of(T, cur_e);
+      const int i0 = t.i0, j0 = t.j0;
       const int row = i0 + r;
-      const bool valid = row < p.Mo;
-      const bool warp_live = i0 + warp * 32 < p.Mo;
-      if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
-      tc_fence_after_sync();
+      const bool valid = row < t.row_end;
+      const bool warp_live = i0 + warp * 32 < t.row_end;
+      const bool have_acc = t.KS > 0;
+      if (have_acc) {
+        if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
+        tc_fence_after_sync();
+      }
       const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN);
       if (warp_live) {
 #pragma unroll 1
@@ -207,12 +298,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           const int col = j0 + 16 * ch;
           if (col >= p.No) break;
           uint32_t v[16];
-          tmem_ld_x16(t0 + 16 * ch, v);
-          tmem_ld_wait();
+          if (have_acc) {
+            tmem_ld_x16(t0 + 16 * ch, v);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = 0u;
+          }
           if (valid) {
             const bool whole = col + 16 <= p.No;  // No is a multiple of 8: a ragged last chunk holds 8 columns
+            const int64_t at = t.c_off + static_cast<int64_t>(row) * p.No + col;
             if (p.c_f32) {
-              float4* fd = reinterpret_cast<float4*>(p.c_f32 + static_cast<int64_t>(row) * p.No + col);
+              float4* fd = reinterpret_cast<float4*>(p.c_f32 + at);
 #pragma unroll
               for (int j = 0; j < 4; ++j)
                 if (j < 2 || whole)
@@ -223,17 +320,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               uint32_t ob[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) ob[j] = bf16x2_bits(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-              uint4* od = reinterpret_cast<uint4*>(p.c_bf16 + static_cast<int64_t>(row) * p.No + col);
+              uint4* od = reinterpret_cast<uint4*>(p.c_bf16 + at);
               od[0] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
               if (whole) od[1] = make_uint4(ob[4], ob[5], ob[6], ob[7]);
             }
           }
         }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
-      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+      if (have_acc) {
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s->tmem_empty[acc]);
+        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
     }
   }
 
@@ -257,22 +356,23 @@ CUresult make_tmap(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint6
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <bool A_MN, bool B_MN>
-cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p) {
+template <bool A_MN, bool B_MN, int GROUP>
+cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p,
+                           int64_t tiles) {
   static bool attr_set_dev[64] = {};
   bool& attr_set = attr_set_dev[L.device & 63];
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kSmemBytes));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int64_t tiles = static_cast<int64_t>((p.Mo + BM - 1) / BM) * ((p.No + BN - 1) / BN);
   // full rounds only: with W = ceil(tiles / SMs) rounds, ceil(tiles / W) CTAs finish in W rounds
-  const int64_t rounds = (tiles + L.sm_count - 1) / L.sm_count;
-  const int grid = static_cast<int>((tiles + rounds - 1) / rounds);
+  // (for grouped rows `tiles` is an upper bound: the surplus CTAs find no tile and retire)
+  const int64_t rounds = std::max<int64_t>(1, (tiles + L.sm_count - 1) / L.sm_count);
+  const int grid = static_cast<int>(std::max<int64_t>(1, (tiles + rounds - 1) / rounds));
   ++*L.launches;
-  return launch_pdl(gemm_bf16_kernel<A_MN, B_MN>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
+  return launch_pdl(gemm_bf16_kernel<A_MN, B_MN, GROUP>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
 }
 
 }  // namespace
@@ -280,10 +380,15 @@ cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtenso
 cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err) {
   *cu_err = CUDA_SUCCESS;
   if (a.Mo == 0 || a.No == 0) return cudaSuccess;
+  const bool grouped_rows = a.group == 1, grouped_k = a.group == 2;
+  // rows of the tensors as TMA sees them
+  const int64_t a_rows = a.a_mn_major ? (grouped_k ? a.rows_total : a.Kc) : a.Mo;
+  const int64_t b_rows = a.b_mn_major ? (grouped_k ? a.rows_total : (grouped_rows ? a.E * a.Kc : a.Kc))
+                                      : (grouped_rows ? a.E * a.No : a.No);
   CUtensorMap ta, tb;
-  CUresult r = a.a_mn_major ? make_tmap(encode, &ta, a.a, a.Kc, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a.Mo, a.Kc, BK, BM);
+  CUresult r = a.a_mn_major ? make_tmap(encode, &ta, a.a, a_rows, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a_rows, a.Kc, BK, BM);
   if (r == CUDA_SUCCESS)
-    r = a.b_mn_major ? make_tmap(encode, &tb, a.b, a.Kc, a.No, 64, BK) : make_tmap(encode, &tb, a.b, a.No, a.Kc, BK, BN);
+    r = a.b_mn_major ? make_tmap(encode, &tb, a.b, b_rows, a.No, 64, BK) : make_tmap(encode, &tb, a.b, b_rows, a.Kc, BK, BN);
   if (r != CUDA_SUCCESS) {
     *cu_err = r;
     return cudaErrorUnknown;
@@ -292,12 +397,25 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   p.Mo = static_cast<int>(a.Mo);
   p.No = static_cast<int>(a.No);
   p.Kc = static_cast<int>(a.Kc);
+  p.offsets = a.offsets;
+  p.E = static_cast<int>(a.E);
+  p.rows_total = static_cast<int>(a.rows_total);
   p.c_bf16 = a.c_bf16;
   p.c_f32 = a.c_f32;
   p.status = L.d_status;
   p.wait_limit_ns = 2000000000ull;
-  if (a.a_mn_major) return a.b_mn_major ? launch_variant<true, true>(L, ta, tb, p) : launch_variant<true, false>(L, ta, tb, p);
-  return a.b_mn_major ? launch_variant<false, true>(L, ta, tb, p) : launch_variant<false, false>(L, ta, tb, p);
+  const int64_t n_tiles = (a.No + BN - 1) / BN;
+  if (grouped_rows) {  // A K-major; each expert adds at most one partial row tile
+    const int64_t tiles = (a.Mo / BM + a.E) * n_tiles;
+    return a.b_mn_major ? launch_variant<false, true, kGroupedRows>(L, ta, tb, p, tiles)
+                        : launch_variant<false, false, kGroupedRows>(L, ta, tb, p, tiles);
+  }
+  const int64_t m_tiles = (a.Mo + BM - 1) / BM;
+  if (grouped_k) return launch_variant<true, true, kGroupedContraction>(L, ta, tb, p, a.E * m_tiles * n_tiles);
+  const int64_t tiles = m_tiles * n_tiles;
+  if (a.a_mn_major)
+    return a.b_mn_major ? launch_variant<true, true, kDense>(L, ta, tb, p, tiles) : launch_variant<true, false, kDense>(L, ta, tb, p, tiles);
+  return a.b_mn_major ? launch_variant<false, true, kDense>(L, ta, tb, p, tiles) : launch_variant<false, false, kDense>(L, ta, tb, p, tiles);
 }
 
 }  // namespace qarl

@@ -109,3 +109,52 @@ def test_quantize_weight_publish_writes_two_equal_copies(ctx):
     assert torch.equal(s1, scales) and torch.equal(s2, scales)
     oc, os_ = oracle.quantize_weight(w)
     assert np.array_equal(c2.cpu().numpy(), oc) and np.array_equal(s2.cpu().numpy(), os_)
+
+
+# ------------------------------------------------------------------------------ grouped (expert) backward
+def check_grouped(ctx, seed, sizes, n, k, exact=False):
+    rng = np.random.default_rng(seed)
+    E = len(sizes)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    P = int(off[-1])
+    if exact:
+        mk = lambda *s: inputs.f32_to_bf16_bits(rng.integers(-4, 5, size=s).astype(np.float32))
+        dy, x, w = mk(P, n), mk(P, k), mk(E, n, k)
+    else:
+        dy, x = inputs.act_bf16(rng, P, n), inputs.act_bf16(rng, P, k)
+        w = inputs.weight_bf16(rng, E, n, k)
+    dx16, dx32, dw32 = ctx.grouped_linear_bwd(bits_to_torch(dy), bits_to_torch(x), bits_to_torch(w),
+                                              torch.from_numpy(off).cuda(), want_dx_f32=True)
+    assert ctx.poll() == 0
+    o_dx32, o_dx16, o_dw32 = oracle.grouped_linear_bwd(dy, x, w, off)
+    g_dx, g_dw = dx32.cpu().numpy(), dw32.cpu().numpy()
+    if exact:
+        assert np.array_equal(g_dx, o_dx32) and np.array_equal(g_dw, o_dw32)
+        return
+    for e in range(E):
+        a, b = off[e], off[e + 1]
+        tol = 1e-3 * _norms(dy[a:b], 1)[:, None] * _norms(w[e], 0)[None, :]
+        assert (np.abs(g_dx[a:b].astype(np.float64) - o_dx32[a:b]) <= tol).all()
+        tol = 1e-3 * _norms(dy[a:b], 0)[:, None] * _norms(x[a:b], 0)[None, :] if b > a else np.zeros((n, k))
+        assert (np.abs(g_dw[e].astype(np.float64) - o_dw32[e]) <= tol).all(), f"expert {e}"
+    assert np.array_equal(torch_to_bits(dx16), oracle.bf16_rne(g_dx))
+
+
+def test_grouped_exact_on_integer_data(ctx):
+    """Ragged groups around the 64-row step and the 128-row tile, empty experts first, last and in the
+    middle: every value exact, so one row leaking from a neighbouring expert cannot hide."""
+    check_grouped(ctx, 1, [0, 1, 63, 64, 65, 0, 127, 128, 129, 200, 0], 128, 264, exact=True)
+    check_grouped(ctx, 2, [5], 64, 8, exact=True)
+    check_grouped(ctx, 3, [0, 0, 7, 0], 192, 512, exact=True)
+
+
+def test_grouped_random_data(ctx):
+    check_grouped(ctx, 4, [300, 17, 0, 1000, 64, 129], 256, 512)
+
+
+def test_grouped_expert_projection_shapes(ctx):
+    """The two expert projections of the layer at a reduced expert count: down (N = 2048 -> K = 768)
+    and gate_up (N = 1536 -> K = 2048), Zipf-like group sizes."""
+    sizes = [900, 40, 333, 0, 128, 1, 77, 569]
+    check_grouped(ctx, 5, sizes, 2048, 768)
+    check_grouped(ctx, 6, sizes, 1536, 2048)

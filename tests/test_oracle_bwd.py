@@ -79,3 +79,23 @@ def test_rounding_is_one_rounding_of_the_exact_sum():
     assert np.array_equal(dx32, (dyf @ wf).astype(np.float32))
     assert np.array_equal(dw32, (dyf.T @ xf).astype(np.float32))
     assert np.array_equal(dx16, inputs.f32_to_bf16_bits(dx32))
+
+
+def test_grouped_backward_is_the_per_expert_backward():
+    """Adjoint identity per expert on integers, an empty expert, and E = 1 equals the dense call."""
+    rng = np.random.default_rng(4)
+    E, N, K = 4, 6, 5
+    off = np.array([0, 3, 3, 10, 12])
+    P = off[-1]
+    x, dy, w = _ints(rng, (P, K)), _ints(rng, (P, N)), _ints(rng, (E, N, K))
+    dx32, dx16, dw32 = oracle.grouped_linear_bwd(dy, x, w, off)
+    assert (dw32[1] == 0).all()
+    xf, dyf, wf = (inputs.bf16_bits_to_f32(a).astype(np.int64) for a in (x, dy, w))
+    for e in range(E):
+        a, b = off[e], off[e + 1]
+        y = xf[a:b] @ wf[e].T
+        lhs = int((dyf[a:b] * y).sum())
+        assert lhs == int((dx32[a:b].astype(np.int64) * xf[a:b]).sum()) == int((dw32[e].astype(np.int64) * wf[e]).sum())
+    d1 = oracle.grouped_linear_bwd(dy, x, w[:1], np.array([0, P]))
+    d0 = oracle.linear_bwd(dy, x, w[0])
+    assert np.array_equal(d1[0], d0[0]) and np.array_equal(d1[2][0], d0[2])
