@@ -458,7 +458,31 @@ def main():
             "dx_frac_bf16_peak_measured_burst": fl / (dx_ms * 1e-3) / 1e12 / pk["bf16_burst"],
             "dw_frac_bf16_peak_measured_burst": fl / (dw_ms * 1e-3) / 1e12 / pk["bf16_burst"],
         }
-        del dyb, xb, wb
+        # the expert gate_up projection of the training batch (expert-sorted rows, Zipf group sizes)
+        rows = torch.bincount(ids.flatten().to(torch.int64), minlength=E)
+        goff = torch.zeros(E + 1, dtype=torch.int32, device=dev)
+        goff[1:] = torch.cumsum(rows, 0).to(torch.int32)
+        Pg = M_TRAIN * TOPK
+        dyg = torch.randn((Pg, 2 * I), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        xg = torch.randn((Pg, H), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        gsteps = max(args.steps // 5, 5)
+        for _ in range(2):
+            ctx.grouped_linear_bwd(dyg, xg, w13, goff)
+        ctx.profile_begin(max_marks=gsteps * 4 + 8)
+        for _ in range(gsteps):
+            ctx.grouped_linear_bwd(dyg, xg, w13, goff)
+        gst = ctx.profile_end()
+        ctx.check_device_status()
+        gfl = 2.0 * Pg * 2 * I * H
+        gdx = gst["bwd_dx"][0] / max(gst["bwd_dx"][1], 1)
+        gdw = gst["bwd_dw"][0] / max(gst["bwd_dw"][1], 1)
+        result["backward"]["grouped"] = {
+            "workload": f"backward of the expert gate_up projection, {Pg} expert-sorted rows, E={E}, N={2 * I}, K={H}",
+            "dx_ms": gdx, "dw_ms": gdw, "dx_tflops": gfl / (gdx * 1e-3) / 1e12, "dw_tflops": gfl / (gdw * 1e-3) / 1e12,
+            "dx_frac_bf16_peak_measured_sustained": gfl / (gdx * 1e-3) / 1e12 / pk["bf16_sustained"],
+            "dw_frac_bf16_peak_measured_sustained": gfl / (gdw * 1e-3) / 1e12 / pk["bf16_sustained"],
+        }
+        del dyb, xb, wb, dyg, xg
 
     # ---------------- TBPO sequence-level loss over a packed batch of responses
     if not args.no_tbpo:

@@ -63,6 +63,8 @@ def lib() -> C.CDLL:
         L.oracle_tbpo.argtypes = [p, p, p, p, p, i64] + [C.c_double] * 4 + [p] * 6
         L.oracle_router_topk.restype = None
         L.oracle_router_topk.argtypes = [p, i64, i64, i64, p, p]
+        L.oracle_swiglu_bwd.restype = None
+        L.oracle_swiglu_bwd.argtypes = [p, p, i64, i64, p]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_num_threads.argtypes = []
     return _lib
@@ -349,3 +351,52 @@ def grouped_linear_bwd(dy_bits, x_bits, w_bits, offsets):
         if b > a:
             dx32[a:b], dx16[a:b], dw32[e] = linear_bwd(dy[a:b], x[a:b], w[e])
     return dx32, dx16, dw32
+
+
+# ---------------------------------------------------------------------------- MoE layer backward
+def swiglu_bwd(gate_up_bits, dh_bits) -> np.ndarray:
+    """gate_up bf16 [P, 2I] (saved by the forward), dH bf16 [P, I] -> dGU bf16 bits [P, 2I]."""
+    gu, dh = _c(gate_up_bits, np.uint16), _c(dh_bits, np.uint16)
+    P, I2 = gu.shape
+    out = np.empty((P, I2), dtype=np.uint16)
+    lib().oracle_swiglu_bwd(_ptr(gu), _ptr(dh), P, I2 // 2, _ptr(out))
+    return out
+
+
+def _bf16f(bits):
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def moe_bwd(x_bits, ids, wts, w13_bits, w2_bits, gate_up_bits, h_bits, dout_bits, y32=None):
+    """Full-precision backward of the routed MoE FFN layer (straight-through past both quantizers) on
+    the bf16 masters w13 [E, 2I, H], w2 [E, H, I] and the bf16 activations the low-bit forward saved
+    in expert-sorted order (gate_up [P, 2I], h [P, I]); dout bf16 [M, H].  Steps, each rounding its
+    result to bf16 where a tensor crosses an op boundary:
+      dy[q]  = bf16(w_pair * dout[token])                      per sorted pair q
+      dH     = bf16(dy . W2_e),     dW2_e  = dy^T h            (fp32)
+      dGU    = swiglu_bwd(gate_up, dH)
+      dXs    = bf16(dGU . W13_e),   dW13_e = dGU^T x_sorted    (fp32)
+      dX[t]  = bf16(sum of the token's k rows of dXs in ascending expert id)
+      dwts[t, j] = <dout[t], y32[q]>  (fp32; only if the forward's fp32 down output y32 [P, H], sorted, is given)
+    Returns dict(dx bf16 bits [M, H], dw13, dw2 fp32, dwts or None, and the intermediates)."""
+    ids, wts = _c(ids, np.int32), _c(wts, np.float32)
+    M, k = ids.shape
+    E = w13_bits.shape[0]
+    off, srt, pos = permute(ids, E)
+    tok = srt // k
+    dout = _bf16f(dout_bits)
+    dy = bf16_rne((wts.reshape(-1)[srt][:, None] * dout[tok]).astype(np.float32))
+    x_sorted = _c(x_bits, np.uint16)[tok]
+    _, dh16, dw2 = grouped_linear_bwd(dy, h_bits, w2_bits, off)
+    dgu = swiglu_bwd(gate_up_bits, dh16)
+    _, dxs16, dw13 = grouped_linear_bwd(dgu, x_sorted, w13_bits, off)
+    by_pair = np.empty((M * k, dxs16.shape[1]), dtype=np.float32)
+    by_pair[srt] = _bf16f(dxs16)
+    dx = combine(by_pair, ids, np.ones_like(wts))
+    dwts = None
+    if y32 is not None:
+        d = (dout[tok].astype(np.float64) * np.asarray(y32, dtype=np.float64)).sum(axis=1).astype(np.float32)
+        dwts = np.empty(M * k, dtype=np.float32)
+        dwts[srt] = d
+        dwts = dwts.reshape(M, k)
+    return dict(dx=dx, dw13=dw13, dw2=dw2, dwts=dwts, dy=dy, dh=dh16, dgu=dgu, dxs=dxs16, offsets=off, sorted_pair=srt)

@@ -288,6 +288,25 @@ void oracle_swiglu(const uint16_t *gate_up, int64_t P, int64_t I, uint16_t *h) {
         }
 }
 
+
+/* ---------------------------------------------------------------------------------------
+ * Backward of SwiGLU on the bf16 gate / up saved by the forward: with s = 1 / (1 + exp(-g)),
+ *   dG = dH * u * s * (1 + g (1 - s)),   dU = dH * g * s,
+ * evaluated in double, rounded once to fp32 and then to bf16.  dgu is [P, 2I], gate part first.
+ * ------------------------------------------------------------------------------------- */
+void oracle_swiglu_bwd(const uint16_t *gate_up, const uint16_t *dh, int64_t P, int64_t I, uint16_t *dgu) {
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < P; ++p)
+        for (int64_t i = 0; i < I; ++i) {
+            double g = (double)bf16_to_f32(gate_up[p * 2 * I + i]);
+            double u = (double)bf16_to_f32(gate_up[p * 2 * I + I + i]);
+            double d = (double)bf16_to_f32(dh[p * I + i]);
+            double s = 1.0 / (1.0 + exp(-g));
+            dgu[p * 2 * I + i] = oracle_bf16_rne((float)(d * u * s * (1.0 + g * (1.0 - s))));
+            dgu[p * 2 * I + I + i] = oracle_bf16_rne((float)(d * g * s));
+        }
+}
+
 /* ---------------------------------------------------------------------------------------
  * Top-k weighted combine.  For token t the k contributions are visited in ASCENDING EXPERT
  * ID (a canonical order that does not depend on the caller's slot order; parity unpinned

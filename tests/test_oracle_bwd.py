@@ -99,3 +99,89 @@ def test_grouped_backward_is_the_per_expert_backward():
     d1 = oracle.grouped_linear_bwd(dy, x, w[:1], np.array([0, P]))
     d0 = oracle.linear_bwd(dy, x, w[0])
     assert np.array_equal(d1[0], d0[0]) and np.array_equal(d1[2][0], d0[2])
+
+
+def _layer_f64(x, w13, w2, ids, wts):
+    """The layer as a smooth function in float64 (no quantization, no rounding): the function whose
+    derivative the straight-through backward approximates."""
+    M, k = ids.shape
+    I = w2.shape[2]
+    out = np.zeros((M, w2.shape[1]))
+    for t in range(M):
+        for j in range(k):
+            e = ids[t, j]
+            gu = w13[e] @ x[t]
+            g, u = gu[:I], gu[I:]
+            out[t] += wts[t, j] * (w2[e] @ (g / (1 + np.exp(-g)) * u))
+    return out
+
+
+def test_swiglu_bwd_is_the_derivative_of_swiglu():
+    rng = np.random.default_rng(5)
+    g = rng.normal(0, 1.5, size=(4, 16))
+    u = rng.normal(0, 1.0, size=(4, 16))
+    gu = inputs.f32_to_bf16_bits(np.concatenate([g, u], axis=1).astype(np.float32))
+    ones = inputs.f32_to_bf16_bits(np.ones((4, 16), np.float32))
+    d = inputs.bf16_bits_to_f32(oracle.swiglu_bwd(gu, ones)).astype(np.float64)
+    gq = inputs.bf16_bits_to_f32(gu).astype(np.float64)
+    gg, uu = gq[:, :16], gq[:, 16:]
+    f = lambda a, b: a / (1 + np.exp(-a)) * b
+    eps = 1e-6
+    assert np.allclose(d[:, :16], (f(gg + eps, uu) - f(gg - eps, uu)) / (2 * eps), rtol=1e-2, atol=1e-3)   # bf16 output
+    assert np.allclose(d[:, 16:], (f(gg, uu + eps) - f(gg, uu - eps)) / (2 * eps), rtol=1e-2, atol=1e-3)
+    # g = 0: silu'(0) = 1/2, silu(0) = 0
+    z = inputs.f32_to_bf16_bits(np.array([[0.0, 2.0]], np.float32))
+    out = inputs.bf16_bits_to_f32(oracle.swiglu_bwd(z, inputs.f32_to_bf16_bits(np.array([[3.0]], np.float32))))
+    assert out.tolist() == [[3.0, 0.0]]
+
+
+def test_layer_backward_against_numeric_derivatives_of_the_smooth_layer():
+    """L = <dOut, layer(x, W13, W2)>: central differences of the float64 layer w.r.t. entries of x, W13,
+    W2 and the routing weights against the oracle's backward (which rounds intermediates to bf16 and
+    uses the forward's saved activations): agreement to a few percent pins every index, transpose,
+    sign and the sorted-order bookkeeping."""
+    c = inputs.moe_case(31, 10, h=128, i=128, e=4, k=2)
+    rng = np.random.default_rng(31)
+    x = inputs.bf16_bits_to_f32(c.x).astype(np.float64)
+    w13 = inputs.bf16_bits_to_f32(c.w13).astype(np.float64)
+    w2 = inputs.bf16_bits_to_f32(c.w2).astype(np.float64)
+    wts = c.weights.astype(np.float64)
+    dout_bits = inputs.f32_to_bf16_bits(rng.normal(0, 1, size=(c.M, c.H)).astype(np.float32))
+    dout = inputs.bf16_bits_to_f32(dout_bits).astype(np.float64)
+    # saved activations of a forward in bf16 on the masters (what the backward is given), sorted order
+    off, srt, _ = oracle.permute(c.ids, c.E)
+    tok, exp = srt // c.k, c.ids.reshape(-1)[srt]
+    gu = np.stack([w13[e] @ x[t] for t, e in zip(tok, exp)])
+    gu_bits = inputs.f32_to_bf16_bits(gu.astype(np.float32))
+    h_bits = oracle.swiglu(gu_bits)
+    y32 = np.stack([w2[e] @ inputs.bf16_bits_to_f32(h_bits[q]).astype(np.float64) for q, e in enumerate(exp)]).astype(np.float32)
+    out = oracle.moe_bwd(c.x, c.ids, c.weights, c.w13, c.w2, gu_bits, h_bits, dout_bits, y32=y32)
+    L = lambda X, A, B, Wt: float((dout * _layer_f64(X, A, B, c.ids, Wt)).sum())
+    dx = inputs.bf16_bits_to_f32(out["dx"]).astype(np.float64)
+    scale = np.abs(dx).mean()
+
+    def close(num, got, ref_scale):
+        return abs(num - got) <= 0.03 * abs(num) + 0.02 * ref_scale
+
+    eps = 1e-4
+    for (t, hh) in [(0, 0), (3, 77), (9, 127), (5, 64)]:
+        e_ = np.zeros_like(x); e_[t, hh] = eps
+        num = (L(x + e_, w13, w2, wts) - L(x - e_, w13, w2, wts)) / (2 * eps)
+        assert close(num, dx[t, hh], scale), (t, hh, num, dx[t, hh])
+    used = np.unique(c.ids)
+    for e in used[:3]:
+        for (n, hh) in [(0, 0), (130, 5), (255, 127)]:
+            e_ = np.zeros_like(w13); e_[e, n, hh] = eps
+            num = (L(x, w13 + e_, w2, wts) - L(x, w13 - e_, w2, wts)) / (2 * eps)
+            assert close(num, out["dw13"][e, n, hh], np.abs(out["dw13"][e]).mean()), (e, n, hh)
+        for (hh, i) in [(0, 0), (100, 127), (64, 3)]:
+            e_ = np.zeros_like(w2); e_[e, hh, i] = eps
+            num = (L(x, w13, w2 + e_, wts) - L(x, w13, w2 - e_, wts)) / (2 * eps)
+            assert close(num, out["dw2"][e, hh, i], np.abs(out["dw2"][e]).mean()), (e, hh, i)
+    for (t, j) in [(0, 0), (4, 1), (9, 0)]:
+        e_ = np.zeros_like(wts); e_[t, j] = eps
+        num = (L(x, w13, w2, wts + e_) - L(x, w13, w2, wts - e_)) / (2 * eps)
+        assert close(num, out["dwts"][t, j], np.abs(out["dwts"]).mean()), (t, j)
+    # an expert no token chose has zero weight gradients
+    for e in set(range(c.E)) - set(used.tolist()):
+        assert (out["dw13"][e] == 0).all() and (out["dw2"][e] == 0).all()
