@@ -257,6 +257,30 @@ int qarl_grouped_linear_bwd(qarl_ctx* ctx, const void* dy_bf16, const void* x_bf
                             int64_t K, int64_t E, void* dx_bf16, float* dx_f32, float* dw_f32,
                             void* stream);
 
+/* Full-precision backward of the routed-expert FFN layer of qarl_moe_fwd (Sec. 3.1 item 2): the
+ * straight-through estimator passes the gradient through both quantizers, so the backward runs on
+ * the bf16 masters and on the bf16 activations the low-bit forward produced:
+ *   dy[q]   = bf16(topk_weights[pair] * dout[token])              per expert-sorted pair q
+ *   dH      = bf16(dy . W2_e)          dW2_e  = dy^T h            (fp32)
+ *   dGU     = SwiGLU backward of dH on the saved gate / up        (bf16)
+ *   dXs     = bf16(dGU . W13_e)        dW13_e = dGU^T x           (fp32)
+ *   dx[t]   = bf16(sum of the token's k rows of dXs in ascending expert id)
+ *   d_topk_weights[t, j] = <dout[t], y[q]>   (only if down_f32 and d_topk_weights are given)
+ * in : x_bf16 [M, H], topk_ids [M, k], topk_weights [M, k], w13_bf16 [E, 2I, H], w2_bf16 [E, H, I]
+ *      (masters), gate_up_bf16 [M*k, 2I] and h_bf16 [M*k, I] in expert-sorted order (the forward's
+ *      debug outputs of those names), dout_bf16 [M, H]; optional down_f32 [M*k, H] sorted.
+ * out: dx_bf16 [M, H], dw13_f32 [E, 2I, H], dw2_f32 [E, H, I] (overwritten; zeros for an expert
+ *      without tokens), optional d_topk_weights f32 [M, k].
+ * Limits as qarl_moe_fwd, and H % 64 == 0, I % 32 == 0.
+ * workspace: qarl_moe_bwd_workspace_bytes(M, H, I, E, k) bytes, 256-byte aligned. */
+size_t qarl_moe_bwd_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k);
+int qarl_moe_bwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
+                 const float* topk_weights, int64_t M, int64_t H, int64_t I, int64_t E, int64_t k,
+                 const void* w13_bf16, const void* w2_bf16, const void* gate_up_bf16,
+                 const void* h_bf16, const void* dout_bf16, const float* down_f32, void* dx_bf16,
+                 float* dw13_f32, float* dw2_f32, float* d_topk_weights, void* workspace,
+                 size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * TBPO: the sequence-level surrogate of Sec. 3.2 over B packed responses (ratio and weight as
  * written out in the appendix "Detail of TBPO").  Response i owns tokens
@@ -322,7 +346,8 @@ enum {
   QARL_STAGE_BWD_DW = 8,
   QARL_STAGE_TBPO = 9,
   QARL_STAGE_ROUTER = 10,
-  QARL_NUM_STAGES = 11
+  QARL_STAGE_BWD_ELEMENTWISE = 11,
+  QARL_NUM_STAGES = 12
 };
 int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
 int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);

@@ -32,12 +32,12 @@ EXPORTS = [
     "qarl_profile_begin", "qarl_profile_end", "qarl_linear_fwd_static",
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
-    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd",
+    "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd", "qarl_moe_bwd_workspace_bytes", "qarl_moe_bwd",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
-          "combine", "bwd_dx", "bwd_dw", "tbpo", "router"]
+          "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise"]
 
 
 class QarlError(RuntimeError):
@@ -121,6 +121,10 @@ def load() -> C.CDLL:
     L.qarl_tbpo_loss.argtypes = [p, p, p, p, p, p, i64, i64, C.POINTER(TbpoParams), p, p, p, p, p, p, p, sz, p]
     L.qarl_grouped_linear_bwd.restype = C.c_int
     L.qarl_grouped_linear_bwd.argtypes = [p, p, p, p, p, i64, i64, i64, i64, p, p, p, p]
+    L.qarl_moe_bwd_workspace_bytes.restype = sz
+    L.qarl_moe_bwd_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
+    L.qarl_moe_bwd.restype = C.c_int
+    L.qarl_moe_bwd.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p, p, sz, p]
     L.qarl_router_fwd.restype = C.c_int
     L.qarl_router_fwd.argtypes = [p, p, i64, i64, p, i64, i64, p, p, p, p]
     L.qarl_linear_bwd.restype = C.c_int
@@ -412,6 +416,27 @@ class Context:
         self._check(self.lib.qarl_grouped_linear_bwd(self.h, _ptr(dy), _ptr(x), _ptr(w), _ptr(offsets), P, N, K, E,
                                                      _ptr(dxo), _ptr(dx32), _ptr(dwo), _stream()))
         return dxo, dx32, dwo
+
+    def moe_bwd(self, x, topk_ids, topk_weights, w13, w2, gate_up, h, dout, down_f32=None, out=None, workspace=None):
+        """Backward of the routed-expert FFN layer on bf16 masters w13 [E, 2I, H], w2 [E, H, I] and the
+        forward's saved bf16 gate_up [P, 2I] / h [P, I] (expert-sorted) ->
+        dict(dx bf16 [M, H], dw13 f32, dw2 f32, dwts f32 [M, k] or None)."""
+        M, H = x.shape
+        k = topk_ids.shape[1]
+        E, I2, _ = w13.shape
+        I = I2 // 2
+        dev = x.device
+        if out is None:
+            out = dict(dx=torch.empty((M, H), dtype=torch.bfloat16, device=dev),
+                       dw13=torch.empty((E, 2 * I, H), dtype=torch.float32, device=dev),
+                       dw2=torch.empty((E, H, I), dtype=torch.float32, device=dev),
+                       dwts=torch.empty((M, k), dtype=torch.float32, device=dev) if down_f32 is not None else None)
+        ws = workspace if workspace is not None else self.workspace(max(int(self.lib.qarl_moe_bwd_workspace_bytes(M, H, I, E, k)), 256))
+        self._check(self.lib.qarl_moe_bwd(self.h, _ptr(x), _ptr(topk_ids), _ptr(topk_weights), M, H, I, E, k, _ptr(w13),
+                                          _ptr(w2), _ptr(gate_up), _ptr(h), _ptr(dout), _ptr(down_f32), _ptr(out["dx"]),
+                                          _ptr(out["dw13"]), _ptr(out["dw2"]), _ptr(out["dwts"]), _ptr(ws), ws.numel(),
+                                          _stream()))
+        return out
 
     # ------------------------------------------------------------------ TBPO
     def tbpo_loss(self, lp_cur, lp_old_learner, lp_old_sampler, offsets, adv, eps_h=4e-4, delta_l=3e-4,

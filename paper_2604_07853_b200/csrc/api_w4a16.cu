@@ -17,6 +17,33 @@ int run_gemm_w4(qarl_ctx* ctx, const Launch& L, const GemmW4Args& a) {
   return QARL_OK;
 }
 
+// Workspace carve-up of qarl_moe_bwd.
+struct MoeBwdPlan {
+  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, x_sorted, dy, dh, dgu, dxs, total;
+};
+MoeBwdPlan plan_moe_bwd(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
+  const size_t P = static_cast<size_t>(M * k);
+  MoeBwdPlan p{};
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = o;
+    o = align_up(o + bytes, 256);
+    return at;
+  };
+  p.chunk_hist = take(static_cast<size_t>(permute_num_chunks(M * k)) * E * sizeof(int32_t));
+  p.offsets = take((E + 1) * sizeof(int32_t));
+  p.sorted_pair = take(P * sizeof(int32_t));
+  p.pos_of_pair = take(P * sizeof(int32_t));
+  p.sorted_w = take(P * sizeof(float));
+  p.x_sorted = take(P * H * sizeof(uint16_t));
+  p.dy = take(P * H * sizeof(uint16_t));
+  p.dh = take(P * I * sizeof(uint16_t));
+  p.dgu = take(P * 2 * I * sizeof(uint16_t));
+  p.dxs = take(P * H * sizeof(uint16_t));
+  p.total = o;
+  return p;
+}
+
 // Workspace carve-up of qarl_moe_fwd_w4a16; every slice starts on a 256-byte boundary.
 struct MoeW4Plan {
   size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, x_sorted, h, contrib, total;
@@ -298,6 +325,141 @@ int qarl_grouped_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const 
     if (rc != QARL_OK) return rc;
     mark(ctx, L.stream, QARL_STAGE_BWD_DW);
   }
+  return QARL_OK;
+}
+
+size_t qarl_moe_bwd_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
+  if (M <= 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0) return 0;
+  return plan_moe_bwd(M, H, I, E, k).total;
+}
+
+int qarl_moe_bwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H, int64_t I,
+                 int64_t E, int64_t k, const void* w13, const void* w2, const void* gate_up, const void* h,
+                 const void* dout, const float* down_f32, void* dx, float* dw13, float* dw2, float* dwts,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  if (!ctx || M < 0 || H <= 0 || I <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
+  if (H % 64 || I % 32 || E > 1024 || M * k >= 0x7FFFFF00ll || E * 2 * I > 0x7FFFFF00ll || E * H > 0x7FFFFF00ll)
+    return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (!w13 || !w2 || !dw13 || !dw2) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(w13) || !aligned16(w2) || !aligned16(dw13) || !aligned16(dw2)) return QARL_ERR_MISALIGNED;
+  Launch L = make_launch(ctx, stream);
+  cudaError_t e;
+  if (M == 0) {  // no tokens: the weight gradients are zero
+    if ((e = cudaMemsetAsync(dw13, 0, static_cast<size_t>(E) * 2 * I * H * sizeof(float), L.stream)) != cudaSuccess ||
+        (e = cudaMemsetAsync(dw2, 0, static_cast<size_t>(E) * H * I * sizeof(float), L.stream)) != cudaSuccess)
+      return cuda_fail(ctx, e, "moe_bwd");
+    return QARL_OK;
+  }
+  if (!x || !ids || !wts || !gate_up || !h || !dout || !dx || !workspace) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(gate_up) || !aligned16(h) || !aligned16(dout) || !aligned16(dx) ||
+      !aligned16(down_f32) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return QARL_ERR_MISALIGNED;
+  const MoeBwdPlan pl = plan_moe_bwd(M, H, I, E, k);
+  if (workspace_bytes < pl.total) return QARL_ERR_WORKSPACE_TOO_SMALL;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const int64_t P = M * k;
+  PermuteBuffers pb;
+  pb.chunk_hist = reinterpret_cast<int32_t*>(ws + pl.chunk_hist);
+  pb.offsets = reinterpret_cast<int32_t*>(ws + pl.offsets);
+  pb.sorted_pair = reinterpret_cast<int32_t*>(ws + pl.sorted_pair);
+  pb.pos_of_pair = reinterpret_cast<int32_t*>(ws + pl.pos_of_pair);
+  float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
+  uint16_t* x_sorted = reinterpret_cast<uint16_t*>(ws + pl.x_sorted);
+  uint16_t* dy = reinterpret_cast<uint16_t*>(ws + pl.dy);
+  uint16_t* dh = reinterpret_cast<uint16_t*>(ws + pl.dh);
+  uint16_t* dgu = reinterpret_cast<uint16_t*>(ws + pl.dgu);
+  uint16_t* dxs = reinterpret_cast<uint16_t*>(ws + pl.dxs);
+  const uint16_t* xb = static_cast<const uint16_t*>(x);
+  const uint16_t* doutb = static_cast<const uint16_t*>(dout);
+
+  mark(ctx, L.stream, -1);
+  if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
+  mark(ctx, L.stream, QARL_STAGE_PERMUTE);
+  if ((e = launch_scatter_rows(L, xb, M, H, x_sorted, pb.pos_of_pair, static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
+    return cuda_fail(ctx, e, "scatter_rows");
+  if ((e = launch_scatter_scale_rows(L, doutb, M, H, dy, pb.pos_of_pair, static_cast<int>(k), wts)) != cudaSuccess)
+    return cuda_fail(ctx, e, "scatter_scale_rows");
+  if (down_f32 && dwts && (e = launch_pair_dot(L, doutb, down_f32, pb.sorted_pair, P, H, k, dwts)) != cudaSuccess)
+    return cuda_fail(ctx, e, "pair_dot");
+  mark(ctx, L.stream, QARL_STAGE_BWD_ELEMENTWISE);
+
+  CUresult cu = CUDA_SUCCESS;
+  auto gemm = [&](const GemmBf16Args& a, const char* what, int stage) {
+    cudaError_t ge = launch_gemm_bf16(L, ctx->encode, a, &cu);
+    if (cu != CUDA_SUCCESS) {
+      snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+      return static_cast<int>(QARL_ERR_CUDA);
+    }
+    if (ge != cudaSuccess) return cuda_fail(ctx, ge, what);
+    mark(ctx, L.stream, stage);
+    return static_cast<int>(QARL_OK);
+  };
+  int rc;
+  {  // dH = dy . W2_e
+    GemmBf16Args a{};
+    a.group = 1;
+    a.a = dy;
+    a.b = static_cast<const uint16_t*>(w2);  // [E][c = h][j = i]
+    a.b_mn_major = true;
+    a.Mo = P;
+    a.No = I;
+    a.Kc = H;
+    a.E = E;
+    a.offsets = pb.offsets;
+    a.c_bf16 = dh;
+    if ((rc = gemm(a, "moe_bwd dH", QARL_STAGE_BWD_DX)) != QARL_OK) return rc;
+  }
+  {  // dW2_e = dy^T h
+    GemmBf16Args a{};
+    a.group = 2;
+    a.a = dy;
+    a.a_mn_major = true;
+    a.b = static_cast<const uint16_t*>(h);
+    a.b_mn_major = true;
+    a.Mo = H;
+    a.No = I;
+    a.E = E;
+    a.offsets = pb.offsets;
+    a.rows_total = P;
+    a.c_f32 = dw2;
+    if ((rc = gemm(a, "moe_bwd dW2", QARL_STAGE_BWD_DW)) != QARL_OK) return rc;
+  }
+  if ((e = launch_swiglu_bwd(L, static_cast<const uint16_t*>(gate_up), dh, P, I, dgu)) != cudaSuccess)
+    return cuda_fail(ctx, e, "swiglu_bwd");
+  mark(ctx, L.stream, QARL_STAGE_BWD_ELEMENTWISE);
+  {  // dXs = dGU . W13_e, stored by flat pair id for the combine
+    GemmBf16Args a{};
+    a.group = 1;
+    a.a = dgu;
+    a.b = static_cast<const uint16_t*>(w13);  // [E][c = n][j = h]
+    a.b_mn_major = true;
+    a.Mo = P;
+    a.No = H;
+    a.Kc = 2 * I;
+    a.E = E;
+    a.offsets = pb.offsets;
+    a.out_rows = pb.sorted_pair;
+    a.c_bf16 = dxs;
+    if ((rc = gemm(a, "moe_bwd dXs", QARL_STAGE_BWD_DX)) != QARL_OK) return rc;
+  }
+  {  // dW13_e = dGU^T x
+    GemmBf16Args a{};
+    a.group = 2;
+    a.a = dgu;
+    a.a_mn_major = true;
+    a.b = x_sorted;
+    a.b_mn_major = true;
+    a.Mo = 2 * I;
+    a.No = H;
+    a.E = E;
+    a.offsets = pb.offsets;
+    a.rows_total = P;
+    a.c_f32 = dw13;
+    if ((rc = gemm(a, "moe_bwd dW13", QARL_STAGE_BWD_DW)) != QARL_OK) return rc;
+  }
+  if ((e = launch_combine(L, dxs, ids, M, k, H, E, static_cast<uint16_t*>(dx))) != cudaSuccess)
+    return cuda_fail(ctx, e, "combine");
+  mark(ctx, L.stream, QARL_STAGE_COMBINE);
   return QARL_OK;
 }
 

@@ -183,8 +183,17 @@ struct GemmBf16Args {
   const int32_t* offsets = nullptr;  // [E + 1], device
   int64_t E = 1;
   int64_t rows_total = 0;
+  const int32_t* out_rows = nullptr;  // group = 1: C row of sorted row p is out_rows[p] (e.g. the flat pair id)
 };
 cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf16Args& a, CUresult* cu_err);
+
+// element-wise kernels of the MoE layer's backward
+cudaError_t launch_scatter_scale_rows(const Launch& L, const uint16_t* dout, int64_t M, int64_t H, uint16_t* dy,
+                                      const int32_t* dst_rows, int fanout, const float* pair_w);
+cudaError_t launch_swiglu_bwd(const Launch& L, const uint16_t* gate_up, const uint16_t* dh, int64_t P, int64_t I,
+                              uint16_t* dgu);
+cudaError_t launch_pair_dot(const Launch& L, const uint16_t* dout, const float* y, const int32_t* sorted_pair,
+                            int64_t P, int64_t H, int64_t k, float* dwts);
 
 // fp32 logits [M, E] -> top-k ids (descending, ties to the lower id) and softmax weights over the selection
 cudaError_t launch_router_topk(const Launch& L, const float* logits, int64_t M, int64_t E, int64_t k, int32_t* ids,

@@ -60,6 +60,7 @@ struct Bf16Params {
   const int32_t* offsets;   // [E + 1] (grouped forms)
   int E;
   int rows_total;           // grouped contraction: P
+  const int32_t* out_rows;  // grouped rows: output row of each sorted row (nullptr: the row itself)
   uint16_t* c_bf16;   // [Mo, No] or nullptr
   float* c_f32;       // [Mo, No] or nullptr
   int* status;
@@ -307,7 +308,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           }
           if (valid) {
             const bool whole = col + 16 <= p.No;  // No is a multiple of 8: a ragged last chunk holds 8 columns
-            const int64_t at = t.c_off + static_cast<int64_t>(row) * p.No + col;
+            int64_t orow = row;
+            if (GROUP == kGroupedRows && p.out_rows) orow = min(max(__ldg(p.out_rows + row), 0), p.Mo - 1);
+            const int64_t at = t.c_off + orow * p.No + col;
             if (p.c_f32) {
               float4* fd = reinterpret_cast<float4*>(p.c_f32 + at);
 #pragma unroll
@@ -400,6 +403,7 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   p.offsets = a.offsets;
   p.E = static_cast<int>(a.E);
   p.rows_total = static_cast<int>(a.rows_total);
+  p.out_rows = a.out_rows;
   p.c_bf16 = a.c_bf16;
   p.c_f32 = a.c_f32;
   p.status = L.d_status;

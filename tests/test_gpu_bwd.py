@@ -158,3 +158,71 @@ def test_grouped_expert_projection_shapes(ctx):
     sizes = [900, 40, 333, 0, 128, 1, 77, 569]
     check_grouped(ctx, 5, sizes, 2048, 768)
     check_grouped(ctx, 6, sizes, 1536, 2048)
+
+
+# ------------------------------------------------------------------------------ MoE layer backward
+def check_moe_bwd(ctx, case, seed):
+    """FP8 forward on the GPU (saving gate_up, h and the fp32 down output), then the backward; the
+    oracle's backward runs on the same saved tensors.  Intermediates cross op boundaries in bf16 on
+    both sides and may differ by one bf16 step where the GPU's fp32 accumulation order rounds the
+    other way, so the end-to-end bars are norms: 1 % on dx and the weight gradients per expert,
+    1e-4 on the routing-weight gradient (a plain fp32 dot product)."""
+    from util import to_dev
+    c = case
+    rng = np.random.default_rng(seed)
+    dout = inputs.f32_to_bf16_bits(rng.normal(0, 1, size=(c.M, c.H)).astype(np.float32))
+    xt, ids, wts = bits_to_torch(c.x), to_dev(c.ids), to_dev(c.weights)
+    w13t, w2t = bits_to_torch(c.w13), bits_to_torch(c.w2)
+    w13c, w13s = ctx.quantize_weight(w13t)
+    w2c, w2s = ctx.quantize_weight(w2t)
+    _, d = ctx.moe_fwd(xt, ids, wts, w13c, w13s, w2c, w2s, debug=True)
+    out = ctx.moe_bwd(xt, ids, wts, w13t, w2t, d["gate_up"], d["h"], bits_to_torch(dout), down_f32=d["down_f32"])
+    assert ctx.poll() == 0
+    ref = oracle.moe_bwd(c.x, c.ids, c.weights, c.w13, c.w2, torch_to_bits(d["gate_up"]), torch_to_bits(d["h"]), dout,
+                         y32=d["down_f32"].cpu().numpy())
+    rel = lambda g, r: np.linalg.norm(g.astype(np.float64) - r.astype(np.float64)) / max(np.linalg.norm(r.astype(np.float64)), 1e-30)
+    gdx = inputs.bf16_bits_to_f32(torch_to_bits(out["dx"]))
+    assert rel(gdx, inputs.bf16_bits_to_f32(ref["dx"])) < 1e-2
+    g13, g2 = out["dw13"].cpu().numpy(), out["dw2"].cpu().numpy()
+    sizes = np.diff(ref["offsets"])
+    for e in range(c.E):
+        if sizes[e] == 0:
+            assert (g13[e] == 0).all() and (g2[e] == 0).all()
+        else:
+            assert rel(g13[e], ref["dw13"][e]) < 1e-2 and rel(g2[e], ref["dw2"][e]) < 1e-2, e
+    assert rel(out["dwts"].cpu().numpy(), ref["dwts"]) < 1e-4
+    return out, ref
+
+
+def test_moe_layer_backward_small(ctx):
+    check_moe_bwd(ctx, inputs.moe_case(41, 24, h=256, i=128, e=8, k=2), 41)
+
+
+def test_moe_layer_backward_ragged_and_empty_experts(ctx):
+    check_moe_bwd(ctx, inputs.moe_case(42, 3, h=256, i=256, e=16, k=4), 42)
+    check_moe_bwd(ctx, inputs.moe_case(43, 333, h=512, i=256, e=4, k=2), 43)
+
+
+def test_moe_layer_backward_skewed(ctx):
+    check_moe_bwd(ctx, inputs.moe_case(44, 600, h=256, i=128, e=32, k=8, zipf_s=1.1), 44)
+
+
+def test_moe_layer_backward_token_rows_do_not_depend_on_the_batch(ctx):
+    """dx of a token depends only on that token (weight gradients of course add over the batch)."""
+    from util import to_dev
+    c = inputs.moe_case(45, 128, h=256, i=128, e=8, k=2)
+    rng = np.random.default_rng(45)
+    dout = bits_to_torch(inputs.f32_to_bf16_bits(rng.normal(0, 1, size=(c.M, c.H)).astype(np.float32)))
+    xt, ids, wts = bits_to_torch(c.x), to_dev(c.ids), to_dev(c.weights)
+    w13t, w2t = bits_to_torch(c.w13), bits_to_torch(c.w2)
+    w13c, w13s = ctx.quantize_weight(w13t)
+    w2c, w2s = ctx.quantize_weight(w2t)
+
+    def run(rows):
+        x_, i_, w_, d_ = (t[rows].contiguous() for t in (xt, ids, wts, dout))
+        _, d = ctx.moe_fwd(x_, i_, w_, w13c, w13s, w2c, w2s, debug=True)
+        return ctx.moe_bwd(x_, i_, w_, w13t, w2t, d["gate_up"], d["h"], d_)["dx"].clone()
+
+    full = run(list(range(128)))
+    for rows in ([0], [127], list(range(40, 72))):
+        assert torch.equal(run(rows), full[rows])
