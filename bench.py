@@ -482,6 +482,35 @@ def main():
             "dx_frac_bf16_peak_measured_sustained": gfl / (gdx * 1e-3) / 1e12 / pk["bf16_sustained"],
             "dw_frac_bf16_peak_measured_sustained": gfl / (gdw * 1e-3) / 1e12 / pk["bf16_sustained"],
         }
+        # backward of the whole routed-expert layer on the training batch (saved activations from one forward)
+        _, dbg = ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, debug=True, workspace=ws)
+        gu_saved, h_saved = dbg["gate_up"], dbg["h"]
+        del dbg
+        doutb = torch.randn((M_TRAIN, H), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        bws = torch.empty(ctx.lib.qarl_moe_bwd_workspace_bytes(M_TRAIN, H, I, E, TOPK), dtype=torch.uint8, device=dev)
+        bout = ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, workspace=bws)
+        msteps = max(args.steps // 5, 5)
+        ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, out=bout, workspace=bws)
+        barrier()
+        ev0.record()
+        for _ in range(msteps):
+            ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, out=bout, workspace=bws)
+        ev1.record()
+        barrier()
+        mb_ms = max_over_ranks(ev0.elapsed_time(ev1)) / msteps
+        ctx.profile_begin(max_marks=msteps * 16 + 8)
+        for _ in range(msteps):
+            ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, out=bout, workspace=bws)
+        mst = ctx.profile_end()
+        ctx.check_device_status()
+        bfl = 2.0 * M_TRAIN * FLOP_PER_TOKEN
+        result["backward"]["moe_layer"] = {
+            "workload": f"backward of the routed-expert layer, M={M_TRAIN} (4 grouped bf16 GEMMs + element-wise kernels)",
+            "ms_per_step": mb_ms, "tflops": bfl / (mb_ms * 1e-3) / 1e12,
+            "frac_bf16_peak_measured_sustained": bfl / (mb_ms * 1e-3) / 1e12 / pk["bf16_sustained"],
+            "stage_ms": {k_: v[0] / msteps for k_, v in mst.items() if v[1]},
+        }
+        del gu_saved, h_saved, doutb, bws, bout
         del dyb, xb, wb, dyg, xg
 
     # ---------------- TBPO sequence-level loss over a packed batch of responses
