@@ -60,6 +60,7 @@ struct Bf16Params {
   const int32_t* offsets;   // [E + 1] (grouped forms)
   int E;
   int rows_total;           // grouped contraction: P
+  int a3d, b3d;             // MN-major operand staged by one 3-D TMA box (64 columns x 64 rows x blocks)
   const int32_t* out_rows;  // grouped rows: output row of each sorted row (nullptr: the row itself)
   uint16_t* c_bf16;   // [Mo, No] or nullptr
   float* c_f32;       // [Mo, No] or nullptr
@@ -203,14 +204,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
           uint8_t* b_dst = a_dst + kABytes;
           mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
-          if (A_MN) {
+          if (A_MN && p.a3d) {
+            tma_load_3d(a_dst, &tm_a, &s->full[stage], 0, t.a_c0 + ks * BK, i0 / 64);
+          } else if (A_MN) {
 #pragma unroll
             for (int b = 0; b < BM / 64; ++b)
               tma_load_2d(a_dst + b * kBlockBytes, &tm_a, &s->full[stage], i0 + 64 * b, t.a_c0 + ks * BK);
           } else {
             tma_load_2d(a_dst, &tm_a, &s->full[stage], t.a_c0 + ks * BK, i0);
           }
-          if (B_MN) {
+          if (B_MN && p.b3d) {
+            tma_load_3d(b_dst, &tm_b, &s->full[stage], 0, t.b_c0 + ks * BK, j0 / 64);
+          } else if (B_MN) {
 #pragma unroll
             for (int b = 0; b < BN / 64; ++b)
               tma_load_2d(b_dst + b * kBlockBytes, &tm_b, &s->full[stage], j0 + 64 * b, t.b_c0 + ks * BK);
@@ -359,6 +364,20 @@ CUresult make_tmap(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint6
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+// An MN-major matrix [rows, cols] (cols % 64 == 0) seen as 64-column blocks: dims {64, rows, cols / 64};
+// one box of 64 x 64 x nblocks lands as nblocks consecutive 8 KB blocks, the layout the descriptor expects.
+// The issuing thread pays per TMA instruction, so one box per operand instead of one per block matters.
+CUresult make_tmap_mn3d(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                        uint32_t nblocks) {
+  const cuuint64_t dims[3] = {64, rows, cols / 64};
+  const cuuint64_t strides[2] = {cols * 2, 128};
+  const cuuint32_t box[3] = {64, BK, nblocks};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 template <bool A_MN, bool B_MN, int GROUP>
 cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p,
                            int64_t tiles) {
@@ -389,9 +408,12 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   const int64_t b_rows = a.b_mn_major ? (grouped_k ? a.rows_total : (grouped_rows ? a.E * a.Kc : a.Kc))
                                       : (grouped_rows ? a.E * a.No : a.No);
   CUtensorMap ta, tb;
-  CUresult r = a.a_mn_major ? make_tmap(encode, &ta, a.a, a_rows, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a_rows, a.Kc, BK, BM);
+  const bool a3d = a.a_mn_major && a.Mo % 64 == 0, b3d = a.b_mn_major && a.No % 64 == 0;
+  CUresult r = a3d ? make_tmap_mn3d(encode, &ta, a.a, a_rows, a.Mo, BM / 64)
+             : a.a_mn_major ? make_tmap(encode, &ta, a.a, a_rows, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a_rows, a.Kc, BK, BM);
   if (r == CUDA_SUCCESS)
-    r = a.b_mn_major ? make_tmap(encode, &tb, a.b, b_rows, a.No, 64, BK) : make_tmap(encode, &tb, a.b, b_rows, a.Kc, BK, BN);
+    r = b3d ? make_tmap_mn3d(encode, &tb, a.b, b_rows, a.No, BN / 64)
+      : a.b_mn_major ? make_tmap(encode, &tb, a.b, b_rows, a.No, 64, BK) : make_tmap(encode, &tb, a.b, b_rows, a.Kc, BK, BN);
   if (r != CUDA_SUCCESS) {
     *cu_err = r;
     return cudaErrorUnknown;
@@ -404,6 +426,8 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   p.E = static_cast<int>(a.E);
   p.rows_total = static_cast<int>(a.rows_total);
   p.out_rows = a.out_rows;
+  p.a3d = a3d;
+  p.b3d = b3d;
   p.c_bf16 = a.c_bf16;
   p.c_f32 = a.c_f32;
   p.status = L.d_status;
