@@ -41,15 +41,26 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
-constexpr int kAccBufs = 2;
+constexpr int kMaxStages = 4, kMaxAccBufs = 2;
 constexpr int kEpiWarps = 4;   // warps 0-3 (TMEM quadrant = warp index)
 constexpr int kTmaWarp = 4;
 constexpr int kMmaWarp = 5;
 constexpr int kThreads = 6 * 32;
-constexpr uint32_t kABytes = BM * BK * 2;   // 16 KB
+constexpr uint32_t kAHalfBytes = BM * BK * 2;   // 16 KB: 128 output rows x 64 contraction elements
 constexpr uint32_t kBBytes = BN * BK * 2;   // 32 KB
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
+// A tile holds MT x 128 output rows.  The kernel is bound by the bytes it can keep in flight from
+// L2/HBM (shared-memory capacity over load latency: throughput grew linearly with the ring depth),
+// so MT = 2 -- both 128-row halves share one B tile, a third fewer bytes per flop -- is the default;
+// it leaves one set of accumulators, i.e. an epilogue that is not overlapped, which only pays when
+// the contraction is long enough (MT = 1 for the ragged contraction of the grouped dW).
+template <int MT>
+struct Cfg {
+  static constexpr int kRows = MT * BM;
+  static constexpr uint32_t kABytes = MT * kAHalfBytes;
+  static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = MT == 1 ? 4 : 3;
+  static constexpr int kAccBufs = MT == 1 ? 2 : 1;
+};
 constexpr uint32_t kBlockBytes = 64 * BK * 2;  // one MN-major block: 64 output indices x 64 c-rows
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxExperts = 1024;
@@ -69,17 +80,18 @@ struct Bf16Params {
 };
 
 struct __align__(8) SmemTail {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
-  uint64_t tmem_full[kAccBufs];
-  uint64_t tmem_empty[kAccBufs];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t tmem_full[kMaxAccBufs];
+  uint64_t tmem_empty[kMaxAccBufs];
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
   int32_t prefix[kMaxExperts + 1];
 };
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + sizeof(SmemTail);
-static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+template <int MT>
+constexpr size_t smem_bytes() { return 1024 + static_cast<size_t>(Cfg<MT>::kStages) * Cfg<MT>::kStageBytes + sizeof(SmemTail); }
+static_assert(smem_bytes<1>() <= 227 * 1024 && smem_bytes<2>() <= 227 * 1024, "shared memory budget");
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const Bf16Params& p) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -102,12 +114,15 @@ __device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&b);
 }
 
-template <bool A_MN, bool B_MN, int GROUP>
+template <bool A_MN, bool B_MN, int GROUP, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const Bf16Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using C = Cfg<MT>;
+  constexpr int kStages = C::kStages, kAccBufs = C::kAccBufs, TM = C::kRows;
+  constexpr uint32_t kABytes = C::kABytes, kStageBytes = C::kStageBytes;
   SmemTail* s = reinterpret_cast<SmemTail*>(smem + static_cast<size_t>(kStages) * kStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -134,9 +149,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   }
   pdl_wait();
   const int n_tiles = (p.No + BN - 1) / BN;
-  const int m_tiles = GROUP == kGroupedRows ? 0 : (p.Mo + BM - 1) / BM;
+  const int m_tiles = GROUP == kGroupedRows ? 0 : (p.Mo + TM - 1) / TM;
   if (GROUP == kGroupedRows) {
-    build_tile_list(s->off, s->prefix, p.offsets, p.Mo, p.E, BM, n_tiles);
+    build_tile_list(s->off, s->prefix, p.offsets, p.Mo, p.E, TM, n_tiles);
   } else if (GROUP == kGroupedContraction) {
     for (int e = threadIdx.x; e <= p.E; e += kThreads) s->off[e] = min(max(p.offsets[e], 0), p.rows_total);
   }
@@ -161,12 +176,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     Tile t{};
     t.last_valid = BK;
     if (GROUP == kDense) {
-      t.i0 = (T % m_tiles) * BM;
+      t.i0 = (T % m_tiles) * TM;
       t.j0 = (T / m_tiles) * BN;
       t.KS = (p.Kc + BK - 1) / BK;  // a ragged last step reads zeros (TMA out-of-range fill)
       t.row_end = p.Mo;
     } else if (GROUP == kGroupedRows) {
-      const TileCoord c = decode_tile(s->off, s->prefix, BM, T, cur_e);
+      const TileCoord c = decode_tile(s->off, s->prefix, TM, T, cur_e);
       t.i0 = c.m0;
       t.j0 = c.n_tile * BN;
       t.KS = p.Kc / BK;             // Kc is a multiple of 64 here: a step never runs into the next expert's weights
@@ -177,7 +192,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     } else {
       const int per_e = m_tiles * n_tiles;
       const int e = T / per_e, r = T % per_e;
-      t.i0 = (r % m_tiles) * BM;
+      t.i0 = (r % m_tiles) * TM;
       t.j0 = (r / m_tiles) * BN;
       const int rows = s->off[e + 1] - s->off[e];
       t.KS = (rows + BK - 1) / BK;
@@ -208,9 +223,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             tma_load_3d(a_dst, &tm_a, &s->full[stage], 0, t.a_c0 + ks * BK, i0 / 64);
           } else if (A_MN) {
 #pragma unroll
-            for (int b = 0; b < BM / 64; ++b)
+            for (int b = 0; b < TM / 64; ++b)
               tma_load_2d(a_dst + b * kBlockBytes, &tm_a, &s->full[stage], i0 + 64 * b, t.a_c0 + ks * BK);
-          } else {
+          } else {  // one box of TM rows x 128 bytes
             tma_load_2d(a_dst, &tm_a, &s->full[stage], t.a_c0 + ks * BK, i0);
           }
           if (B_MN && p.b3d) {
@@ -244,14 +259,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const Tile t = tile_of(T, cur_e);
       if (t.KS == 0) continue;  // an expert without rows: the epilogue writes zeros, no accumulator is used
       if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
-      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * BN;
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * MT) * BN;
       for (int ks = 0; ks < t.KS; ++ks) {
         if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
         uint8_t* a_tile = smem + static_cast<size_t>(stage) * kStageBytes;
         if (GROUP == kGroupedContraction && ks == t.KS - 1 && t.last_valid < BK) {
           // rows last_valid .. 63 of both 64-column blocks of A belong to the next expert: make them zero
           const int nrows = BK - t.last_valid;
-          for (int idx = lane; idx < 2 * nrows * 8; idx += 32) {
+          for (int idx = lane; idx < (TM / 64) * nrows * 8; idx += 32) {
             const int blk = idx / (nrows * 8), rem = idx % (nrows * 8);
             *reinterpret_cast<uint4*>(a_tile + blk * kBlockBytes + (t.last_valid + rem / 8) * 128 + (rem % 8) * 16) =
                 make_uint4(0, 0, 0, 0);
@@ -270,8 +285,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           constexpr uint32_t a_step = A_MN ? (16 * 128) >> 4 : 32 >> 4;
           constexpr uint32_t b_step = B_MN ? (16 * 128) >> 4 : 32 >> 4;
 #pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4)
-            umma_bf16(d_tmem, a_desc + a_step * k4, b_desc + b_step * k4, idesc, (ks > 0 || k4 > 0) ? 1u : 0u);
+          for (int mt = 0; mt < MT; ++mt)  // the 128-row halves of A share the B tile
+#pragma unroll
+            for (int k4 = 0; k4 < BK / 16; ++k4)
+              umma_bf16(d_tmem + mt * BN, a_desc + mt * (kAHalfBytes >> 4) + a_step * k4, b_desc + b_step * k4, idesc,
+                        (ks > 0 || k4 > 0) ? 1u : 0u);
           umma_commit(&s->empty[stage]);
           if (ks == t.KS - 1) umma_commit(&s->tmem_full[acc]);
         }
@@ -288,16 +306,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     int cur_e = 0;
     for (int T = blockIdx.x; T < total_tiles; T += grid) {
       const Tile t = tile_of(T, cur_e);
-      const int i0 = t.i0, j0 = t.j0;
-      const int row = i0 + r;
-      const bool valid = row < t.row_end;
-      const bool warp_live = i0 + warp * 32 < t.row_end;
+      const int j0 = t.j0;
       const bool have_acc = t.KS > 0;
       if (have_acc) {
         if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
         tc_fence_after_sync();
       }
-      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+      for (int mt = 0; mt < MT; ++mt) {
+      const int i0 = t.i0 + mt * BM;
+      const int row = i0 + r;
+      const bool valid = row < t.row_end;
+      const bool warp_live = i0 + warp * 32 < t.row_end;
+      const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>((acc * MT + mt) * BN);
       if (warp_live) {
 #pragma unroll 1
         for (int ch = 0; ch < BN / 16; ++ch) {
@@ -335,6 +356,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           }
         }
       }
+      }  // mt
       if (have_acc) {
         tc_fence_before_sync();
         __syncwarp();
@@ -378,14 +400,14 @@ CUresult make_tmap_mn3d(EncodeTiledFn encode, CUtensorMap* m, const void* base, 
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <bool A_MN, bool B_MN, int GROUP>
+template <bool A_MN, bool B_MN, int GROUP, int MT>
 cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p,
                            int64_t tiles) {
   static bool attr_set_dev[64] = {};
   bool& attr_set = attr_set_dev[L.device & 63];
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kSmemBytes));
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN, GROUP, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem_bytes<MT>()));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -394,7 +416,7 @@ cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtenso
   const int64_t rounds = std::max<int64_t>(1, (tiles + L.sm_count - 1) / L.sm_count);
   const int grid = static_cast<int>(std::max<int64_t>(1, (tiles + rounds - 1) / rounds));
   ++*L.launches;
-  return launch_pdl(gemm_bf16_kernel<A_MN, B_MN, GROUP>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
+  return launch_pdl(gemm_bf16_kernel<A_MN, B_MN, GROUP, MT>, static_cast<unsigned>(grid), kThreads, smem_bytes<MT>(), L.stream, ta, tb, p);
 }
 
 }  // namespace
@@ -403,14 +425,26 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   *cu_err = CUDA_SUCCESS;
   if (a.Mo == 0 || a.No == 0) return cudaSuccess;
   const bool grouped_rows = a.group == 1, grouped_k = a.group == 2;
+  // 256-row tiles pay (measured: 13 % less time per unit of work) when the tile count still fills the
+  // SMs' rounds; the grouped forms keep 128-row tiles (ragged groups waste more of a 256-row tile and
+  // the single accumulator set exposes the epilogue of short tiles).
+  int MT = 1;
+  if (a.group == 0 && a.Mo > BM) {
+    const int64_t n_t = (a.No + BN - 1) / BN;
+    const int64_t t1 = (a.Mo + BM - 1) / BM * n_t, t2 = (a.Mo + 2 * BM - 1) / (2 * BM) * n_t;
+    const double cost1 = static_cast<double>((t1 + L.sm_count - 1) / L.sm_count);
+    const double cost2 = static_cast<double>((t2 + L.sm_count - 1) / L.sm_count) * 2.0 * 0.87;
+    if (cost2 < cost1) MT = 2;
+  }
+  const int TM = MT * BM;
   // rows of the tensors as TMA sees them
   const int64_t a_rows = a.a_mn_major ? (grouped_k ? a.rows_total : a.Kc) : a.Mo;
   const int64_t b_rows = a.b_mn_major ? (grouped_k ? a.rows_total : (grouped_rows ? a.E * a.Kc : a.Kc))
                                       : (grouped_rows ? a.E * a.No : a.No);
   CUtensorMap ta, tb;
   const bool a3d = a.a_mn_major && a.Mo % 64 == 0, b3d = a.b_mn_major && a.No % 64 == 0;
-  CUresult r = a3d ? make_tmap_mn3d(encode, &ta, a.a, a_rows, a.Mo, BM / 64)
-             : a.a_mn_major ? make_tmap(encode, &ta, a.a, a_rows, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a_rows, a.Kc, BK, BM);
+  CUresult r = a3d ? make_tmap_mn3d(encode, &ta, a.a, a_rows, a.Mo, TM / 64)
+             : a.a_mn_major ? make_tmap(encode, &ta, a.a, a_rows, a.Mo, 64, BK) : make_tmap(encode, &ta, a.a, a_rows, a.Kc, BK, TM);
   if (r == CUDA_SUCCESS)
     r = b3d ? make_tmap_mn3d(encode, &tb, a.b, b_rows, a.No, BN / 64)
       : a.b_mn_major ? make_tmap(encode, &tb, a.b, b_rows, a.No, 64, BK) : make_tmap(encode, &tb, a.b, b_rows, a.Kc, BK, BN);
@@ -434,16 +468,24 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   p.wait_limit_ns = 2000000000ull;
   const int64_t n_tiles = (a.No + BN - 1) / BN;
   if (grouped_rows) {  // A K-major; each expert adds at most one partial row tile
-    const int64_t tiles = (a.Mo / BM + a.E) * n_tiles;
-    return a.b_mn_major ? launch_variant<false, true, kGroupedRows>(L, ta, tb, p, tiles)
-                        : launch_variant<false, false, kGroupedRows>(L, ta, tb, p, tiles);
+    const int64_t tiles = (a.Mo / TM + a.E) * n_tiles;
+    if (MT == 2)
+      return a.b_mn_major ? launch_variant<false, true, kGroupedRows, 2>(L, ta, tb, p, tiles)
+                          : launch_variant<false, false, kGroupedRows, 2>(L, ta, tb, p, tiles);
+    return a.b_mn_major ? launch_variant<false, true, kGroupedRows, 1>(L, ta, tb, p, tiles)
+                        : launch_variant<false, false, kGroupedRows, 1>(L, ta, tb, p, tiles);
   }
-  const int64_t m_tiles = (a.Mo + BM - 1) / BM;
-  if (grouped_k) return launch_variant<true, true, kGroupedContraction>(L, ta, tb, p, a.E * m_tiles * n_tiles);
+  const int64_t m_tiles = (a.Mo + TM - 1) / TM;
+  if (grouped_k) return launch_variant<true, true, kGroupedContraction, 1>(L, ta, tb, p, a.E * m_tiles * n_tiles);
   const int64_t tiles = m_tiles * n_tiles;
+  if (MT == 2) {
+    if (a.a_mn_major)
+      return a.b_mn_major ? launch_variant<true, true, kDense, 2>(L, ta, tb, p, tiles) : launch_variant<true, false, kDense, 2>(L, ta, tb, p, tiles);
+    return a.b_mn_major ? launch_variant<false, true, kDense, 2>(L, ta, tb, p, tiles) : launch_variant<false, false, kDense, 2>(L, ta, tb, p, tiles);
+  }
   if (a.a_mn_major)
-    return a.b_mn_major ? launch_variant<true, true, kDense>(L, ta, tb, p, tiles) : launch_variant<true, false, kDense>(L, ta, tb, p, tiles);
-  return a.b_mn_major ? launch_variant<false, true, kDense>(L, ta, tb, p, tiles) : launch_variant<false, false, kDense>(L, ta, tb, p, tiles);
+    return a.b_mn_major ? launch_variant<true, true, kDense, 1>(L, ta, tb, p, tiles) : launch_variant<true, false, kDense, 1>(L, ta, tb, p, tiles);
+  return a.b_mn_major ? launch_variant<false, true, kDense, 1>(L, ta, tb, p, tiles) : launch_variant<false, false, kDense, 1>(L, ta, tb, p, tiles);
 }
 
 }  // namespace qarl

@@ -45,7 +45,10 @@ constexpr int BM = 128;           // rows per tile (UMMA M)
 constexpr int BNH = 128;          // columns per half tile
 constexpr int BN = 2 * BNH;       // UMMA N
 constexpr int BK = 128;           // one K-block = one 128-byte swizzle span of e4m3
-constexpr int kStages = 3;
+#ifndef QARL_FP8_STAGES
+#define QARL_FP8_STAGES 3
+#endif
+constexpr int kStages = QARL_FP8_STAGES;
 constexpr int kAccBufs = 2;       // TMEM accumulators of 256 columns
 constexpr int kPromoWarps = 8;    // warps 0-7
 constexpr int kEpiWarps = 4;      // warps 8-11
