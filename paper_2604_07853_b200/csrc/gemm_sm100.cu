@@ -49,7 +49,10 @@ constexpr int BK = 128;           // one K-block = one 128-byte swizzle span of 
 #define QARL_FP8_STAGES 3
 #endif
 constexpr int kStages = QARL_FP8_STAGES;
-constexpr int kAccBufs = 2;       // TMEM accumulators of 256 columns
+#ifndef QARL_FP8_ACCBUFS
+#define QARL_FP8_ACCBUFS 2
+#endif
+constexpr int kAccBufs = QARL_FP8_ACCBUFS;       // TMEM accumulators of 256 columns
 constexpr int kPromoWarps = 8;    // warps 0-7
 constexpr int kEpiWarps = 4;      // warps 8-11
 constexpr int kTmaWarp = 12;
