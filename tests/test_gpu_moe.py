@@ -212,3 +212,25 @@ def test_empty_batch_and_argument_errors(ctx):
     with pytest.raises(binding.QarlError) as ei:
         ctx.moe_fwd(dc.x, dc.ids, dc.wts, dc.w13c, dc.w13s, dc.w2c, dc.w2s, workspace=small)
     assert ei.value.status == -4
+
+
+def test_layer_can_be_captured_in_a_cuda_graph(ctx):
+    """The layer makes no allocation, no synchronisation and no host read between its launches, so a
+    stream capture records it; a replay gives the bytes of the eager call."""
+    c = inputs.moe_case(13, 64, h=256, i=128, e=8, k=2)
+    dc = DeviceCase(ctx, c)
+    ref = dc.run(ctx).clone()
+    out = torch.empty_like(ref)
+    ws = ctx.workspace(ctx.moe_workspace_bytes(c.M, c.H, c.I, c.E, c.k))
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        ctx.moe_fwd(dc.x, dc.ids, dc.wts, dc.w13c, dc.w13s, dc.w2c, dc.w2s, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        ctx.moe_fwd(dc.x, dc.ids, dc.wts, dc.w13c, dc.w13s, dc.w2c, dc.w2s, out=out, workspace=ws)
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
+    assert ctx.poll() == 0
