@@ -198,6 +198,7 @@ def main():
     ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--no-tbpo", action="store_true")
     ap.add_argument("--no-router", action="store_true")
+    ap.add_argument("--no-linear", action="store_true")
     ap.add_argument("--tokens", type=int, default=M_TRAIN,
                     help="tokens per GPU of the training-shape step (smaller values are for profiler captures "
                          "only; the reported config names the size)")
@@ -363,6 +364,47 @@ def main():
                            "frac_fp8_peak_nominal_4500": M_TRAIN * FLOP_PER_TOKEN / (layer_ms * 1e-3) / 1e12 / 4500.0},
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches * world, "clocks": clocks,
     }
+
+    # ---------------- dense projection (QKV of the training configuration): N = 5120, K = 2048, M = 8192 and 64
+    if not args.no_linear:
+        Nl, Kl = 5120, 2048
+        gen = torch.Generator(device=dev).manual_seed(6000 + rank)
+        wl = (torch.randn((Nl, Kl), generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        # 16 copies of the quantized weight (168 MB), used in turn: a small-M call never finds its weight in L2
+        copies = [ctx.quantize_weight(wl) for _ in range(16)]
+        lin = {}
+        for Ml in (8192, 64):
+            xl = torch.randn((Ml, Kl), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            yl = torch.empty((Ml, Nl), dtype=torch.bfloat16, device=dev)
+            lsteps = max(args.steps, 20) * (1 if Ml > 1000 else 5)
+            for i in range(5):
+                ctx.linear_fwd(xl, *copies[i % 16], out=yl)
+            barrier()
+            ev0.record()
+            for i in range(lsteps):
+                ctx.linear_fwd(xl, *copies[i % 16], out=yl)
+            ev1.record()
+            barrier()
+            l_ms = max_over_ranks(ev0.elapsed_time(ev1)) / lsteps
+            ctx.profile_begin(max_marks=lsteps * 4 + 8)
+            for i in range(lsteps):
+                ctx.linear_fwd(xl, *copies[i % 16], out=yl)
+            lst = ctx.profile_end()
+            ctx.check_device_status()
+            g_ms = lst["linear_gemm"][0] / max(lst["linear_gemm"][1], 1)
+            fl = 2.0 * Ml * Nl * Kl
+            lbytes = Nl * Kl + Nl * Kl // (128 * 128) * 4 + Ml * Kl * 2 + Ml * Nl * 2
+            lin[f"M{Ml}"] = {
+                "ms_per_call": l_ms, "gemm_ms": g_ms, "quantize_act_ms": lst["quantize_act"][0] / max(lst["quantize_act"][1], 1),
+                "gemm_tflops": fl / (g_ms * 1e-3) / 1e12,
+                "gemm_frac_fp8_peak_measured": fl / (g_ms * 1e-3) / 1e12 / (2.0 * pk["bf16_sustained"]),
+                "algorithmic_bytes": lbytes, "gbs": lbytes / (l_ms * 1e-3) / 1e9,
+                "frac_hbm_measured": lbytes / (l_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+            }
+            del xl, yl
+        result["linear"] = {"workload": f"dense FP8 projection N={Nl} K={Kl} (activation quantization + GEMM), "
+                                        "16 weight copies used in turn", **lin}
+        del wl, copies
 
     # ---------------- router (bf16 logits GEMM + top-k softmax) on the training batch
     if not args.no_router:
