@@ -149,7 +149,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   }
   pdl_wait();
   const int n_tiles = (p.No + BN - 1) / BN;
-  const int m_tiles = GROUP == kGroupedRows ? 0 : (p.Mo + TM - 1) / TM;
+  const int m_tiles = GROUP == kGroupedRows ? 1 : (p.Mo + TM - 1) / TM;  // grouped rows: tiles come from the offsets
   if (GROUP == kGroupedRows) {
     build_tile_list(s->off, s->prefix, p.offsets, p.Mo, p.E, TM, n_tiles);
   } else if (GROUP == kGroupedContraction) {
@@ -469,9 +469,6 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   const int64_t n_tiles = (a.No + BN - 1) / BN;
   if (grouped_rows) {  // A K-major; each expert adds at most one partial row tile
     const int64_t tiles = (a.Mo / TM + a.E) * n_tiles;
-    if (MT == 2)
-      return a.b_mn_major ? launch_variant<false, true, kGroupedRows, 2>(L, ta, tb, p, tiles)
-                          : launch_variant<false, false, kGroupedRows, 2>(L, ta, tb, p, tiles);
     return a.b_mn_major ? launch_variant<false, true, kGroupedRows, 1>(L, ta, tb, p, tiles)
                         : launch_variant<false, false, kGroupedRows, 1>(L, ta, tb, p, tiles);
   }
