@@ -147,27 +147,28 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
 // exact quotient is either exactly half-way between two integers or at least 2^-14 (relative) away
 // from such a point: the product with inv = fl(1 / s) (relative error ~2^-23) then rounds to the
 // same integer except at exact ties, which the exact residual r = w - q0 s identifies
-// (2 r = +-s) and resolves to the even neighbour.  Rounding by adding and subtracting 1.5 * 2^23.
-__device__ __forceinline__ uint32_t w4_code(float w, float s, float inv, float zf) {
-  const float kMagic = 12582912.0f;
-  float q0 = __fsub_rn(__fadd_rn(__fmul_rn(w, inv), kMagic), kMagic);
-  const float r2 = 2.0f * __fmaf_rn(-q0, s, w);  // exact: q0 s has at most 13 significant bits
-  if (r2 == s || r2 == -s) {                     // tie between q0 and q0 + sign(r2)
-    const float other = r2 > 0.0f ? q0 + 1.0f : q0 - 1.0f;
+// (2 r = +-s) and resolves to the even neighbour.
+__device__ __forceinline__ uint32_t w4_code(float w, float s, float inv, float zm) {
+  const float kMagic = 12582912.0f;               // 1.5 * 2^23: adding it rounds to an integer
+  float q0 = __fsub_rn(__fmaf_rn(w, inv, kMagic), kMagic);
+  const float r = __fmaf_rn(-q0, s, w);           // exact: q0 s has at most 13 significant bits
+  if (fabsf(__fadd_rn(r, r)) == s) {              // tie between q0 and q0 + sign(r)
+    const float other = r > 0.0f ? q0 + 1.0f : q0 - 1.0f;
     const float half = 0.5f * q0;
     if (__fsub_rn(__fadd_rn(half, kMagic), kMagic) != half) q0 = other;  // q0 odd: the other one is even
   }
-  const float v = fminf(fmaxf(q0 + zf, 0.0f), 15.0f);
-  return __float_as_uint(v + 8388608.0f) & 15u;  // integer 0..15 in the low mantissa bits
+  // zm = z + 2^23: the code is clamped in that domain, where the integer sits in the low mantissa bits
+  const float v = fminf(fmaxf(__fadd_rn(q0, zm), 8388608.0f), 8388623.0f);
+  return __float_as_uint(v) & 15u;
 }
 
-__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float inv, float zf) {
+__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float inv, float zm) {
   const uint32_t in[4] = {v.x, v.y, v.z, v.w};
   uint32_t word = 0;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    word |= w4_code(bf16_bits_to_f32(in[j] & 0xFFFFu), s, inv, zf) << (4 * j);
-    word |= w4_code(__uint_as_float(in[j] & 0xFFFF0000u), s, inv, zf) << (4 * j + 16);
+    word |= w4_code(bf16_bits_to_f32(in[j] & 0xFFFFu), s, inv, zm) << (4 * j);
+    word |= w4_code(__uint_as_float(in[j] & 0xFFFF0000u), s, inv, zm) << (4 * j + 16);
   }
   return word;
 }
@@ -214,7 +215,8 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
   const float s = bf16_bits_to_f32(s_bits);
   const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
   const float inv = __fdiv_rn(1.0f, s);
-  const uint2 out = make_uint2(w4_word(v0, s, inv, zf), w4_word(v1, s, inv, zf));
+  const float zm = zf + 8388608.0f;
+  const uint2 out = make_uint2(w4_word(v0, s, inv, zm), w4_word(v1, s, inv, zm));
   if (!live) return;
   const int64_t e = row / N, n = row % N;
   {
