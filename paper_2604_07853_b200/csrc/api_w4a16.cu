@@ -77,7 +77,7 @@ int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, 
                             void* scales, uint8_t* zeros, void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
   if (K % kBlock || N % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
-  if (E * N * (K / kBlock) > (0x7FFFFFFFll << 5)) return QARL_ERR_UNSUPPORTED_SHAPE;
+  if (E * N * (K / kBlock) >= 0x10000000ll || E * N >= 0x7FFFFFFFll) return QARL_ERR_UNSUPPORTED_SHAPE;  // 32-bit group index x 8 threads
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
   if (!w || !packed || !scales || !zeros) return QARL_ERR_INVALID_ARG;
   if (!aligned16(w) || !aligned16(packed) || (reinterpret_cast<uintptr_t>(scales) & 1u)) return QARL_ERR_MISALIGNED;

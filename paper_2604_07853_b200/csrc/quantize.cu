@@ -190,11 +190,14 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
                                                                  uint8_t* __restrict__ zeros) {
   pdl_trigger();
   pdl_wait();
-  const int64_t kb = K / kBlock;
-  const int64_t gid = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;
-  const bool live = gid < rows * kb;
-  const int64_t gg = live ? gid : 0;
-  const int64_t row = gg / kb, g = gg % kb;
+  // 32-bit index arithmetic (the launcher guarantees fewer than 2^31 groups): 64-bit divisions
+  // would cost more instructions than the quantization itself
+  const uint32_t kb = static_cast<uint32_t>(K / kBlock);
+  const uint32_t gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  const bool live = gid < static_cast<uint32_t>(rows) * kb;
+  const uint32_t gg = live ? gid : 0u;
+  const uint32_t row32 = gg / kb, g32 = gg - row32 * kb;
+  const int64_t row = row32, g = g32;
   const int sub = threadIdx.x & 7;
   const uint4* src = reinterpret_cast<const uint4*>(w + row * K + g * kBlock + sub * 16);
   uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
@@ -218,12 +221,13 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
   const float zm = zf + 8388608.0f;
   const uint2 out = make_uint2(w4_word(v0, s, inv, zm), w4_word(v1, s, inv, zm));
   if (!live) return;
-  const int64_t e = row / N, n = row % N;
+  const uint32_t e32 = row32 / static_cast<uint32_t>(N);
+  const int64_t e = e32, n = row32 - e32 * static_cast<uint32_t>(N);
   {
     const int64_t ks = g * 2 + (sub >> 2);  // K-step of 64 elements
-    const int64_t chunk = (e * (N / kBlock) + n / kBlock) * (K / 64) + ks;
+    const int64_t chunk = (e * (N / kBlock) + (n >> 7)) * (K / 64) + ks;
     const int quad = (sub & 3) >> 1, piece = sub & 1;  // words 2(sub%4), 2(sub%4)+1 of the K-step's eight
-    *reinterpret_cast<uint2*>(packed + chunk * 4096 + quad * 2048 + (n % kBlock) * 16 + piece * 8) = out;
+    *reinterpret_cast<uint2*>(packed + chunk * 4096 + quad * 2048 + (n & (kBlock - 1)) * 16 + piece * 8) = out;
   }
   if (sub == 0) {
     const int64_t idx = (e * kb + g) * N + n;
