@@ -561,10 +561,11 @@ def main():
             "dx_frac_bf16_peak_measured_sustained": gfl / (gdx * 1e-3) / 1e12 / pk["bf16_sustained"],
             "dw_frac_bf16_peak_measured_sustained": gfl / (gdw * 1e-3) / 1e12 / pk["bf16_sustained"],
         }
-        # backward of the whole routed-expert layer on the training batch (saved activations from one forward)
-        _, dbg = ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, debug=True, workspace=ws)
-        gu_saved, h_saved = dbg["gate_up"], dbg["h"]
-        del dbg
+        # backward of the whole routed-expert layer on the training batch (activations saved by the forward)
+        saved = dict(gate_up=torch.empty((M_TRAIN * TOPK, 2 * I), dtype=torch.bfloat16, device=dev),
+                     h=torch.empty((M_TRAIN * TOPK, I), dtype=torch.bfloat16, device=dev))
+        ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, workspace=ws, save=saved)
+        gu_saved, h_saved = saved["gate_up"], saved["h"]
         doutb = torch.randn((M_TRAIN, H), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         bws = torch.empty(ctx.lib.qarl_moe_bwd_workspace_bytes(M_TRAIN, H, I, E, TOPK), dtype=torch.uint8, device=dev)
         bout = ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, workspace=bws)
@@ -589,7 +590,28 @@ def main():
             "frac_bf16_peak_measured_sustained": bfl / (mb_ms * 1e-3) / 1e12 / pk["bf16_sustained"],
             "stage_ms": {k_: v[0] / msteps for k_, v in mst.items() if v[1]},
         }
-        del gu_saved, h_saved, doutb, bws, bout
+        # one training step of the layer: quantize + publish-ready codes, low-bit forward that saves its
+        # activations, full-precision backward
+        def train_step():
+            ctx.quantize_weight(w13, w13c, w13s)
+            ctx.quantize_weight(w2, w2c, w2s)
+            ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, workspace=ws, save=saved)
+            ctx.moe_bwd(x, ids, wts, w13, w2, gu_saved, h_saved, doutb, out=bout, workspace=bws)
+        train_step()
+        barrier()
+        ev0.record()
+        for _ in range(msteps):
+            train_step()
+        ev1.record()
+        barrier()
+        ts_ms = max_over_ranks(ev0.elapsed_time(ev1)) / msteps
+        ctx.check_device_status()
+        result["backward"]["train_step"] = {
+            "workload": f"layer training step, M={M_TRAIN}: weight quantization + FP8 forward (saving gate_up, h) + bf16 backward",
+            "ms_per_step": ts_ms, "tokens_per_s": world * M_TRAIN / (ts_ms * 1e-3),
+            "tflops": 3.0 * M_TRAIN * FLOP_PER_TOKEN / (ts_ms * 1e-3) / 1e12,
+        }
+        del gu_saved, h_saved, saved, doutb, bws, bout
         del dyb, xb, wb, dyg, xg
 
     # ---------------- TBPO sequence-level loss over a packed batch of responses

@@ -286,8 +286,10 @@ class Context:
         return int(self.lib.qarl_moe_workspace_bytes(M, H, I, E, k))
 
     def moe_fwd(self, x, topk_ids, topk_weights, w13_codes, w13_scales, w2_codes, w2_scales,
-                out=None, debug: bool = False, workspace: torch.Tensor | None = None):
-        """One routed-expert FFN layer -> out bf16 [M, H] (and a dict of dumps if debug)."""
+                out=None, debug: bool = False, workspace: torch.Tensor | None = None, save=None):
+        """One routed-expert FFN layer -> out bf16 [M, H] (and a dict of dumps if debug).
+        save: dict(gate_up=bf16 [P, 2I], h=bf16 [P, I]) of caller-owned tensors that receive the
+        activations the backward needs (expert-sorted order), without the other dumps."""
         assert x.dtype == torch.bfloat16 and x.is_contiguous()
         assert topk_ids.dtype == torch.int32 and topk_weights.dtype == torch.float32
         M, H = x.shape
@@ -299,6 +301,8 @@ class Context:
         nbytes = self.moe_workspace_bytes(M, H, I, E, k)
         ws = workspace if workspace is not None else self.workspace(nbytes)
         d, dbg = None, None
+        if save is not None:
+            dbg = MoeDebug(None, None, save["gate_up"].data_ptr(), save["h"].data_ptr(), None, None, None)
         if debug:
             dev = x.device
             d = dict(expert_offsets=torch.zeros(E + 1, dtype=torch.int32, device=dev),
