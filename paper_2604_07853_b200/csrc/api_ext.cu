@@ -1,5 +1,6 @@
-// C ABI entry points of the W4A16 path (4-bit group-quantized weights, bf16 activations) and of
-// the full-precision backward: argument checks, workspace planning, kernel sequencing.  No device memory is allocated here.
+// C ABI entry points beyond the FP8 forward: the W4A16 path (4-bit group-quantized weights, bf16
+// activations), the full-precision backward (dense, per expert, whole layer), the TBPO loss and the
+// router: argument checks, workspace planning, kernel sequencing.  No device memory is allocated here.
 #include "api_util.cuh"
 
 namespace {
