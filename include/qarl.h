@@ -198,6 +198,13 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
  * scales (2-byte aligned), zeros, as above; caller-owned.  One kernel, every input byte read once. */
 int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
                             uint8_t* packed, void* scales_bf16, uint8_t* zeros, void* stream);
+/* The same, fused with publishing (Sec. 3.1 item 3): pub_* is a second destination of the same
+ * shapes (the rollout engine's buffers), written from the same registers in the same launch;
+ * all three NULL: identical to qarl_quantize_weight_w4.  The copies are bitwise equal. */
+int qarl_quantize_weight_w4_publish(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N,
+                                    int64_t K, uint8_t* packed, void* scales_bf16, uint8_t* zeros,
+                                    uint8_t* pub_packed, void* pub_scales_bf16, uint8_t* pub_zeros,
+                                    void* stream);
 
 /* y[m, n] = bf16( sum_k x[m,k] * w^[n,k] ), fp32 accumulation (Sec. 2.2 Dequant applied inside
  * the GEMM).  in: x_bf16 [M, K] 16-byte aligned; weights as produced by qarl_quantize_weight_w4

@@ -33,6 +33,7 @@ EXPORTS = [
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
     "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd", "qarl_moe_bwd_workspace_bytes", "qarl_moe_bwd",
+    "qarl_quantize_weight_w4_publish",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
@@ -125,6 +126,8 @@ def load() -> C.CDLL:
     L.qarl_moe_bwd_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
     L.qarl_moe_bwd.restype = C.c_int
     L.qarl_moe_bwd.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p, p, sz, p]
+    L.qarl_quantize_weight_w4_publish.restype = C.c_int
+    L.qarl_quantize_weight_w4_publish.argtypes = [p, p, i64, i64, i64, p, p, p, p, p, p, p]
     L.qarl_router_fwd.restype = C.c_int
     L.qarl_router_fwd.argtypes = [p, p, i64, i64, p, i64, i64, p, p, p, p]
     L.qarl_linear_bwd.restype = C.c_int
@@ -338,6 +341,15 @@ class Context:
         self._check(self.lib.qarl_quantize_weight_w4(self.h, _ptr(w), E, N, K, _ptr(packed), _ptr(scales),
                                                      _ptr(zeros), _stream()))
         return packed, scales, zeros
+
+    def quantize_weight_w4_publish(self, w, out, pub):
+        """quantize_weight_w4 writing a second, published copy (packed, scales, zeros) in the same launch."""
+        assert w.dtype == torch.bfloat16 and w.is_cuda and w.is_contiguous()
+        E, N, K = (1, *w.shape) if w.dim() == 2 else w.shape
+        self._check(self.lib.qarl_quantize_weight_w4_publish(self.h, _ptr(w), E, N, K, _ptr(out[0]), _ptr(out[1]),
+                                                             _ptr(out[2]), _ptr(pub[0]), _ptr(pub[1]), _ptr(pub[2]),
+                                                             _stream()))
+        return out
 
     def linear_fwd_w4a16(self, x, w_packed, w_scales, w_zeros, out=None, want_f32: bool = False):
         """y = x . w^T with 4-bit weights -> y bf16 [M, N] (and the fp32 accumulator if want_f32)."""

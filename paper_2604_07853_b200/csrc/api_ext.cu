@@ -76,7 +76,16 @@ extern "C" {
 
 int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
                             void* scales, uint8_t* zeros, void* stream) {
+  return qarl_quantize_weight_w4_publish(ctx, w, E, N, K, packed, scales, zeros, nullptr, nullptr, nullptr, stream);
+}
+
+int qarl_quantize_weight_w4_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                                    void* scales, uint8_t* zeros, uint8_t* pub_packed, void* pub_scales,
+                                    uint8_t* pub_zeros, void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
+  const int npub = (pub_packed != nullptr) + (pub_scales != nullptr) + (pub_zeros != nullptr);
+  if (npub != 0 && npub != 3) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(pub_packed) || (reinterpret_cast<uintptr_t>(pub_scales) & 1u)) return QARL_ERR_MISALIGNED;
   if (K % kBlock || N % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E * N * (K / kBlock) >= 0x10000000ll || E * N >= 0x7FFFFFFFll) return QARL_ERR_UNSUPPORTED_SHAPE;  // 32-bit group index x 8 threads
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
@@ -84,7 +93,8 @@ int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, 
   if (!aligned16(w) || !aligned16(packed) || (reinterpret_cast<uintptr_t>(scales) & 1u)) return QARL_ERR_MISALIGNED;
   mark(ctx, static_cast<cudaStream_t>(stream), -1);
   cudaError_t e = launch_quantize_weight_w4(make_launch(ctx, stream), static_cast<const uint16_t*>(w), E, N, K, packed,
-                                            static_cast<uint16_t*>(scales), zeros);
+                                            static_cast<uint16_t*>(scales), zeros, pub_packed,
+                                            static_cast<uint16_t*>(pub_scales), pub_zeros);
   mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_WEIGHT);
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_weight_w4");
 }

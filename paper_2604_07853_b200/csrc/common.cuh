@@ -142,7 +142,9 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
 
 // ---- W4A16 (4-bit group-quantized weights, bf16 activations) --------------------------------
 cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
-                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros);
+                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros,
+                                      uint8_t* pub_packed = nullptr, uint16_t* pub_scales = nullptr,
+                                      uint8_t* pub_zeros = nullptr);
 // bf16 row t of x [M, H] -> rows dst_rows[t*fanout + j] of out; pair weights scattered alongside.
 cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,
                                 const int32_t* dst_rows, int fanout, const float* pair_w, float* sorted_w);

@@ -187,7 +187,10 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
                                                                  int64_t N, int64_t K,
                                                                  uint8_t* __restrict__ packed,
                                                                  uint16_t* __restrict__ scales,
-                                                                 uint8_t* __restrict__ zeros) {
+                                                                 uint8_t* __restrict__ zeros,
+                                                                 uint8_t* __restrict__ pub_packed,
+                                                                 uint16_t* __restrict__ pub_scales,
+                                                                 uint8_t* __restrict__ pub_zeros) {
   pdl_trigger();
   pdl_wait();
   // 32-bit index arithmetic (the launcher guarantees fewer than 2^31 groups): 64-bit divisions
@@ -227,12 +230,18 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
     const int64_t ks = g * 2 + (sub >> 2);  // K-step of 64 elements
     const int64_t chunk = (e * (N / kBlock) + (n >> 7)) * (K / 64) + ks;
     const int quad = (sub & 3) >> 1, piece = sub & 1;  // words 2(sub%4), 2(sub%4)+1 of the K-step's eight
-    *reinterpret_cast<uint2*>(packed + chunk * 4096 + quad * 2048 + (n & (kBlock - 1)) * 16 + piece * 8) = out;
+    const int64_t at = chunk * 4096 + quad * 2048 + (n & (kBlock - 1)) * 16 + piece * 8;
+    *reinterpret_cast<uint2*>(packed + at) = out;
+    if (pub_packed) *reinterpret_cast<uint2*>(pub_packed + at) = out;  // the rollout engine's copy (Sec. 3.1 item 3)
   }
   if (sub == 0) {
     const int64_t idx = (e * kb + g) * N + n;
     scales[idx] = static_cast<uint16_t>(s_bits);
     zeros[idx] = static_cast<uint8_t>(zf);
+    if (pub_packed) {
+      pub_scales[idx] = static_cast<uint16_t>(s_bits);
+      pub_zeros[idx] = static_cast<uint8_t>(zf);
+    }
   }
 }
 
@@ -281,13 +290,14 @@ cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, i
 }
 
 cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
-                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros) {
+                                      uint8_t* packed, uint16_t* scales, uint8_t* zeros, uint8_t* pub_packed,
+                                      uint16_t* pub_scales, uint8_t* pub_zeros) {
   const int64_t groups = E * N * (K / kBlock);
   if (groups == 0) return cudaSuccess;
   const int64_t blocks = (groups * 8 + 255) / 256;
   ++*L.launches;
   return launch_pdl(quantize_weight_w4_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, E * N, N, K, packed,
-                    scales, zeros);
+                    scales, zeros, pub_packed, pub_scales, pub_zeros);
 }
 
 cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,

@@ -107,6 +107,18 @@ def test_quantizer_exact_ties_round_to_even(ctx):
     assert np.array_equal(gs, os_) and np.array_equal(gz, oz)
 
 
+def test_quantizer_publish_writes_two_equal_copies(ctx):
+    """Sec. 3.1 item 3: the published 4-bit tensors are the ones the training forward uses, bit for bit."""
+    rng = np.random.default_rng(8)
+    wt = bits_to_torch(inputs.weight_bf16(rng, 2, 256, 384))
+    ref = ctx.quantize_weight_w4(wt)
+    a = tuple(torch.zeros_like(t) for t in ref)
+    b = tuple(torch.zeros_like(t) for t in ref)
+    ctx.quantize_weight_w4_publish(wt, a, b)
+    for r, x, y in zip(ref, a, b):
+        assert torch.equal(r, x) and torch.equal(r, y)
+
+
 # ------------------------------------------------------------------------------ dense GEMM
 def check_linear(ctx, seed, m, n, k):
     """fp32: |gpu - oracle| <= 1e-3 * ||x_row|| * ||w^_col|| (the oracle sums exactly; the tensor
