@@ -53,6 +53,14 @@ def lib() -> C.CDLL:
         L.oracle_quantize_weight_w4.argtypes = [p, i64, i64, i64, p, p, p]
         L.oracle_dequant_w4.restype = None
         L.oracle_dequant_w4.argtypes = [p, p, p, i64, i64, p]
+        L.oracle_e2m1_decode.restype = C.c_double
+        L.oracle_e2m1_decode.argtypes = [C.c_uint8]
+        L.oracle_e2m1_encode.restype = C.c_uint8
+        L.oracle_e2m1_encode.argtypes = [C.c_float]
+        L.oracle_quantize_weight_fp4.restype = C.c_int
+        L.oracle_quantize_weight_fp4.argtypes = [p, i64, i64, i64, p, p]
+        L.oracle_dequant_fp4.restype = None
+        L.oracle_dequant_fp4.argtypes = [p, p, i64, i64, p]
         L.oracle_linear_bf16.restype = None
         L.oracle_linear_bf16.argtypes = [p, i64, i64, p, i64, p, p]
         L.oracle_moe_w4a16.restype = C.c_int
@@ -247,6 +255,42 @@ def dequant_w4(packed, scales, zeros) -> np.ndarray:
     rows = int(np.prod(packed.shape[:-1]))
     out = np.empty((*packed.shape[:-1], K), dtype=np.uint16)
     lib().oracle_dequant_w4(_ptr(packed), _ptr(scales), _ptr(zeros), rows, K, _ptr(out))
+    return out
+
+
+def e2m1_table() -> np.ndarray:
+    """The 16 e2m1 code values (code 8 is -0)."""
+    return np.array([lib().oracle_e2m1_decode(c) for c in range(16)], dtype=np.float64)
+
+
+def e2m1_encode(values) -> np.ndarray:
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    return np.array([lib().oracle_e2m1_encode(float(t)) for t in v.ravel()], dtype=np.uint8).reshape(v.shape)
+
+
+def quantize_weight_fp4(w_bits: np.ndarray):
+    """w bf16 bits [E, N, K] or [N, K] -> (packed u8 [.., N, K/2], scales f32 [.., N, K/128]);
+    e2m1 codes, one scale per 128 K-elements of a row."""
+    w = _c(w_bits, np.uint16)
+    squeeze = w.ndim == 2
+    if squeeze:
+        w = w[None]
+    E, N, K = w.shape
+    packed = np.empty((E, N, K // 2), dtype=np.uint8)
+    scales = np.empty((E, N, K // 128), dtype=np.float32)
+    rc = lib().oracle_quantize_weight_fp4(_ptr(w), E, N, K, _ptr(packed), _ptr(scales))
+    if rc:
+        raise OracleError(rc)
+    return (packed[0], scales[0]) if squeeze else (packed, scales)
+
+
+def dequant_fp4(packed, scales) -> np.ndarray:
+    """-> w^ bf16 bits, same leading shape, last dim K."""
+    packed, scales = _c(packed, np.uint8), _c(scales, np.float32)
+    K = packed.shape[-1] * 2
+    rows = int(np.prod(packed.shape[:-1]))
+    out = np.empty((*packed.shape[:-1], K), dtype=np.uint16)
+    lib().oracle_dequant_fp4(_ptr(packed), _ptr(scales), rows, K, _ptr(out))
     return out
 
 

@@ -492,6 +492,86 @@ void oracle_dequant_w4(const uint8_t *packed, const float *scales, const uint8_t
         }
 }
 
+/* =======================================================================================
+ * FP4 (e2m1) weight-only quantization (Sec. 2.2, "Floating-point quantization"):
+ *   s = max|W| / alpha,   W_q = [W / s]_FP4,   W^ = s * W_q,   alpha = 6 (largest finite e2m1 value).
+ * An e2m1 code has a sign bit (bit 3), two exponent bits (bits 2..1, bias 1) and one mantissa
+ * bit (bit 0); exponent field 0 is subnormal.  The eight magnitudes are 0, 0.5, 1, 1.5, 2, 3, 4, 6;
+ * there is no infinity and no NaN.
+ * Readings where the paper is silent (the same ones as for the integer format, so that the two
+ * 4-bit formats share storage and GEMM): one s per group of 128 consecutive K elements of one
+ * weight row; s = bf16( fl(max(amax, 2^-40) / 6) ), returned as the fp32 of that bf16 value;
+ * W / s is an IEEE fp32 division by the stored s; [.]_FP4 rounds to the nearest representable
+ * value, ties to the even code, and saturates at +-6; zero keeps the sign of W (code 8 for -0
+ * and for negative values that round to zero: it decodes to -0 = 0).  The GEMM consumes
+ * w^ = bf16(s * value): the value has two significant bits and s eight, so the product is exact
+ * before its one rounding.
+ * Packed layout as for the integer format: byte j of a row holds code 2j in its low nibble.
+ * ===================================================================================== */
+static const float E2M1_MAGNITUDES[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+double oracle_e2m1_decode(uint8_t code) {
+    int ee = (code >> 1) & 3, m = code & 1;
+    double mag = ee ? ldexp(1.0 + 0.5 * m, ee - 1) : 0.5 * m;
+    return (code & 8) ? -mag : mag;
+}
+
+/* Round a finite fp32 to e2m1: nearest magnitude, ties to the even code, saturating. */
+uint8_t oracle_e2m1_encode(float f) {
+    uint8_t sign = signbit(f) ? 8 : 0;
+    double a = fabs((double)f);
+    int best = 7;                                   /* everything at or above 6 saturates */
+    for (int c = 0; c < 7; ++c) {
+        double lo = E2M1_MAGNITUDES[c], hi = E2M1_MAGNITUDES[c + 1];
+        if (a > hi) continue;
+        double dl = a - lo, dh = hi - a;            /* a in [lo, hi]: both exact in double */
+        if (dl < dh) best = c;
+        else if (dl > dh) best = c + 1;
+        else best = (c & 1) ? c + 1 : c;            /* tie: the code with mantissa bit 0 */
+        break;
+    }
+    return (uint8_t)(sign | best);
+}
+
+int oracle_quantize_weight_fp4(const uint16_t *w, int64_t E, int64_t N, int64_t K,
+                               uint8_t *packed, float *scales) {
+    if (K % QBLOCK) return -2;
+    int64_t kb = K / QBLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < E * N; ++r)
+        for (int64_t g = 0; g < kb; ++g) {
+            const uint16_t *base = w + r * K + g * QBLOCK;
+            float amax = 0.0f;
+            for (int c = 0; c < QBLOCK; ++c) {
+                float v = fabsf(bf16_to_f32(base[c]));
+                if (v > amax) amax = v;
+            }
+            if (amax < AMAX_FLOOR) amax = AMAX_FLOOR;
+            float s = bf16_to_f32(oracle_bf16_rne(amax / 6.0f));
+            scales[r * kb + g] = s;
+            for (int c = 0; c < QBLOCK; c += 2) {
+                uint8_t q0 = oracle_e2m1_encode(bf16_to_f32(base[c]) / s);
+                uint8_t q1 = oracle_e2m1_encode(bf16_to_f32(base[c + 1]) / s);
+                packed[r * (K / 2) + (g * QBLOCK + c) / 2] = (uint8_t)(q0 | (q1 << 4));
+            }
+        }
+    return 0;
+}
+
+/* w^ bf16 bits [rows, K] from packed e2m1 codes and group scales (rows = E*N). */
+void oracle_dequant_fp4(const uint8_t *packed, const float *scales, int64_t rows, int64_t K,
+                        uint16_t *w_hat) {
+    int64_t kb = K / QBLOCK;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t b = packed[r * (K / 2) + k / 2];
+            uint8_t q = (k & 1) ? (b >> 4) : (b & 15);
+            float s = scales[r * kb + k / QBLOCK];
+            w_hat[r * K + k] = oracle_bf16_rne(s * (float)oracle_e2m1_decode(q));
+        }
+}
+
 /* y[m,n] = sum_k x[m,k] * w^[n,k]: bf16 operands, products and sum exact in double (each
  * product has <= 16 significant bits), rounded once to fp32, then to bf16.  The paper asks
  * only for "higher precision" accumulation; the GPU's tensor-core order is compared with this
