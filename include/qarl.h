@@ -235,6 +235,41 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_id
                        void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * FP4A16: e2m1 floating-point weight-only quantization with bf16 activations (Sec. 2.2,
+ * floating-point quantization: s = max|W| / alpha, W_q = [W / s]_FP4, W^ = s W_q, alpha = 6, the
+ * largest finite e2m1 value).  A code is sign (bit 3) | two exponent bits (bias 1) | one mantissa
+ * bit: magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6; no infinity, no NaN.  Choices the paper leaves
+ * open, fixed here as for the integer format: one s per 128 consecutive K elements of one weight
+ * row; s = bf16(max(amax, 2^-40) / 6); W / s is the IEEE fp32 quotient; [.]_FP4 rounds to the
+ * nearest value, ties to the even code, saturating at +-6; the sign bit is that of W (also on
+ * zero); the GEMM multiplies bf16 activations by w^ = bf16(s * value) and accumulates in fp32 in
+ * ascending k.  Storage: packed and scales exactly as for W4A16 above (same tile-major chunks,
+ * same nibble order, bf16 scales [E, K/128, N]); there are no zero points.
+ * ------------------------------------------------------------------------------------- */
+
+/* in : w_bf16 [E, N, K], 16-byte aligned, N % 128 == 0, K % 128 == 0.  out: packed (16-byte
+ * aligned), scales (2-byte aligned); caller-owned.  pub_packed / pub_scales_bf16: optional second
+ * destination written in the same launch (Sec. 3.1 item 3: the rollout engine's copy), both NULL
+ * or both set.  One kernel, every input byte read once.  Errors as qarl_quantize_weight_w4. */
+int qarl_quantize_weight_fp4(qarl_ctx* ctx, const void* w_bf16, int64_t E, int64_t N, int64_t K,
+                             uint8_t* packed, void* scales_bf16, uint8_t* pub_packed,
+                             void* pub_scales_bf16, void* stream);
+
+/* qarl_linear_fwd_w4a16 on e2m1 weights (E = 1): same shapes, limits, outputs, row invariance. */
+int qarl_linear_fwd_fp4a16(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t K,
+                           const uint8_t* w_packed, const void* w_scales_bf16, int64_t N,
+                           void* y_bf16, float* y_f32, void* stream);
+
+/* qarl_moe_fwd_w4a16 on e2m1 weights: same computation, limits, debug outputs and workspace
+ * (qarl_moe_w4a16_workspace_bytes). */
+int qarl_moe_fwd_fp4a16(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
+                        const float* topk_weights, int64_t M, int64_t H, int64_t I, int64_t E,
+                        int64_t k, const uint8_t* w13_packed, const void* w13_scales_bf16,
+                        const uint8_t* w2_packed, const void* w2_scales_bf16, void* out_bf16,
+                        void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
+                        void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * Training-side backward of a quantized linear layer y = x . W^T (Sec. 3.1 item 2: the forward
  * runs on Quant(W), the backward in full precision; the straight-through estimator treats Quant
  * as the identity and the gradients belong to the bf16 master weights):

@@ -33,7 +33,7 @@ EXPORTS = [
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
     "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd", "qarl_moe_bwd_workspace_bytes", "qarl_moe_bwd",
-    "qarl_quantize_weight_w4_publish",
+    "qarl_quantize_weight_w4_publish", "qarl_quantize_weight_fp4", "qarl_linear_fwd_fp4a16", "qarl_moe_fwd_fp4a16",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
@@ -126,6 +126,12 @@ def load() -> C.CDLL:
     L.qarl_moe_bwd_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
     L.qarl_moe_bwd.restype = C.c_int
     L.qarl_moe_bwd.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p, p, sz, p]
+    L.qarl_quantize_weight_fp4.restype = C.c_int
+    L.qarl_quantize_weight_fp4.argtypes = [p, p, i64, i64, i64, p, p, p, p, p]
+    L.qarl_linear_fwd_fp4a16.restype = C.c_int
+    L.qarl_linear_fwd_fp4a16.argtypes = [p, p, i64, i64, p, p, i64, p, p, p]
+    L.qarl_moe_fwd_fp4a16.restype = C.c_int
+    L.qarl_moe_fwd_fp4a16.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, sz, p, p]
     L.qarl_quantize_weight_w4_publish.restype = C.c_int
     L.qarl_quantize_weight_w4_publish.argtypes = [p, p, i64, i64, i64, p, p, p, p, p, p, p]
     L.qarl_router_fwd.restype = C.c_int
@@ -392,6 +398,63 @@ class Context:
                                                 _ptr(w2[0]), _ptr(w2[1]), _ptr(w2[2]),
                                                 _ptr(y), _ptr(ws), ws.numel(),
                                                 C.byref(dbg) if dbg is not None else None, _stream()))
+        return (y, d) if debug else y
+
+    # ------------------------------------------------------------------ FP4A16 (e2m1 weights)
+    def quantize_weight_fp4(self, w: torch.Tensor, out=None, pub=None):
+        """w bf16 [E, N, K] or [N, K] -> (packed u8 [.., N, K/2], scales bf16 [.., K/128, N]) of e2m1 codes in
+        the library's storage order.  out: an earlier result to overwrite; pub: a second (packed, scales)
+        destination written in the same launch."""
+        assert w.dtype == torch.bfloat16 and w.is_cuda and w.is_contiguous()
+        shape = w.shape
+        E, N, K = (1, *shape) if w.dim() == 2 else shape
+        if out is not None:
+            packed, scales = out
+        else:
+            packed = torch.empty((*shape[:-1], K // 2), dtype=torch.uint8, device=w.device)
+            scales = torch.empty((*shape[:-2], K // 128, N), dtype=torch.bfloat16, device=w.device)
+        pp, ps = pub if pub is not None else (None, None)
+        self._check(self.lib.qarl_quantize_weight_fp4(self.h, _ptr(w), E, N, K, _ptr(packed), _ptr(scales),
+                                                      _ptr(pp), _ptr(ps), _stream()))
+        return packed, scales
+
+    def linear_fwd_fp4a16(self, x, w_packed, w_scales, out=None, want_f32: bool = False):
+        """y = x . w^T with e2m1 weights -> y bf16 [M, N] (and the fp32 accumulator if want_f32)."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        M, K = x.shape
+        N = w_packed.shape[-2]
+        y = out if out is not None else torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        y32 = torch.empty((M, N), dtype=torch.float32, device=x.device) if want_f32 else None
+        self._check(self.lib.qarl_linear_fwd_fp4a16(self.h, _ptr(x), M, K, _ptr(w_packed), _ptr(w_scales), N,
+                                                    _ptr(y), _ptr(y32), _stream()))
+        return (y, y32) if want_f32 else y
+
+    def moe_fwd_fp4a16(self, x, topk_ids, topk_weights, w13, w2, out=None, debug: bool = False,
+                       workspace: torch.Tensor | None = None):
+        """One routed-expert FFN layer on e2m1 weights; w13 and w2 are (packed, scales)."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        assert topk_ids.dtype == torch.int32 and topk_weights.dtype == torch.float32
+        M, H = x.shape
+        k = topk_ids.shape[1]
+        E, I2, _ = w13[0].shape
+        I = I2 // 2
+        P = M * k
+        y = out if out is not None else torch.empty((M, H), dtype=torch.bfloat16, device=x.device)
+        ws = workspace if workspace is not None else self.workspace(self.moe_w4a16_workspace_bytes(M, H, I, E, k))
+        d, dbg = None, None
+        if debug:
+            dev = x.device
+            d = dict(expert_offsets=torch.zeros(E + 1, dtype=torch.int32, device=dev),
+                     sorted_pair=torch.zeros(P, dtype=torch.int32, device=dev),
+                     gate_up=torch.zeros((P, 2 * I), dtype=torch.bfloat16, device=dev),
+                     h=torch.zeros((P, I), dtype=torch.bfloat16, device=dev),
+                     down_f32=torch.zeros((P, H), dtype=torch.float32, device=dev))
+            dbg = MoeDebug(d["expert_offsets"].data_ptr(), d["sorted_pair"].data_ptr(),
+                           d["gate_up"].data_ptr(), d["h"].data_ptr(), None, None, d["down_f32"].data_ptr())
+        self._check(self.lib.qarl_moe_fwd_fp4a16(self.h, _ptr(x), _ptr(topk_ids), _ptr(topk_weights), M, H, I, E, k,
+                                                 _ptr(w13[0]), _ptr(w13[1]), _ptr(w2[0]), _ptr(w2[1]),
+                                                 _ptr(y), _ptr(ws), ws.numel(),
+                                                 C.byref(dbg) if dbg is not None else None, _stream()))
         return (y, d) if debug else y
 
     def quantize_weight_publish(self, w, codes, scales, pub_codes, pub_scales):

@@ -70,46 +70,39 @@ MoeW4Plan plan_moe_w4(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   return p;
 }
 
-}  // namespace
-
-extern "C" {
-
-int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
-                            void* scales, uint8_t* zeros, void* stream) {
-  return qarl_quantize_weight_w4_publish(ctx, w, E, N, K, packed, scales, zeros, nullptr, nullptr, nullptr, stream);
-}
-
-int qarl_quantize_weight_w4_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
-                                    void* scales, uint8_t* zeros, uint8_t* pub_packed, void* pub_scales,
-                                    uint8_t* pub_zeros, void* stream) {
+int quantize_w4(qarl_ctx* ctx, int fmt, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                void* scales, uint8_t* zeros, uint8_t* pub_packed, void* pub_scales, uint8_t* pub_zeros,
+                void* stream) {
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
+  const bool int4 = fmt == kFmtInt4;
   const int npub = (pub_packed != nullptr) + (pub_scales != nullptr) + (pub_zeros != nullptr);
-  if (npub != 0 && npub != 3) return QARL_ERR_INVALID_ARG;
+  if (npub != 0 && npub != (int4 ? 3 : 2)) return QARL_ERR_INVALID_ARG;
   if (!aligned16(pub_packed) || (reinterpret_cast<uintptr_t>(pub_scales) & 1u)) return QARL_ERR_MISALIGNED;
   if (K % kBlock || N % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (E * N * (K / kBlock) >= 0x10000000ll || E * N >= 0x7FFFFFFFll) return QARL_ERR_UNSUPPORTED_SHAPE;  // 32-bit group index x 8 threads
   if (E == 0 || N == 0 || K == 0) return QARL_OK;
-  if (!w || !packed || !scales || !zeros) return QARL_ERR_INVALID_ARG;
+  if (!w || !packed || !scales || (int4 && !zeros)) return QARL_ERR_INVALID_ARG;
   if (!aligned16(w) || !aligned16(packed) || (reinterpret_cast<uintptr_t>(scales) & 1u)) return QARL_ERR_MISALIGNED;
   mark(ctx, static_cast<cudaStream_t>(stream), -1);
-  cudaError_t e = launch_quantize_weight_w4(make_launch(ctx, stream), static_cast<const uint16_t*>(w), E, N, K, packed,
+  cudaError_t e = launch_quantize_weight_w4(make_launch(ctx, stream), fmt, static_cast<const uint16_t*>(w), E, N, K, packed,
                                             static_cast<uint16_t*>(scales), zeros, pub_packed,
                                             static_cast<uint16_t*>(pub_scales), pub_zeros);
   mark(ctx, static_cast<cudaStream_t>(stream), QARL_STAGE_QUANT_WEIGHT);
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "quantize_weight_w4");
 }
 
-int qarl_linear_fwd_w4a16(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wp, const void* ws,
-                          const uint8_t* wz, int64_t N, void* y, float* y_f32, void* stream) {
+int linear_w4(qarl_ctx* ctx, int fmt, const void* x, int64_t M, int64_t K, const uint8_t* wp, const void* ws,
+              const uint8_t* wz, int64_t N, void* y, float* y_f32, void* stream) {
   if (!ctx || M < 0 || K <= 0 || N <= 0) return QARL_ERR_INVALID_ARG;
   if (N % kBlock || K % kBlock || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
-  if (!x || !wp || !ws || !wz || !y) return QARL_ERR_INVALID_ARG;
+  if (!x || !wp || !ws || (fmt == kFmtInt4 && !wz) || !y) return QARL_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(wp) || !aligned16(y) || !aligned16(y_f32) ||
       (reinterpret_cast<uintptr_t>(ws) & 1u))
     return QARL_ERR_MISALIGNED;
   GemmW4Args a{};
   a.mode = kModeLinear;
+  a.fmt = fmt;
   a.a_bf16 = static_cast<const uint16_t*>(x);
   a.rows_total = M;
   a.K = K;
@@ -126,22 +119,17 @@ int qarl_linear_fwd_w4a16(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, co
   return rc;
 }
 
-size_t qarl_moe_w4a16_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
-  if (M <= 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0) return 0;
-  return plan_moe_w4(M, H, I, E, k).total;
-}
-
-int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
-                       int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w13z,
-                       const uint8_t* w2p, const void* w2s, const uint8_t* w2z, void* out, void* workspace,
-                       size_t workspace_bytes, const qarl_moe_debug* dbg, void* stream) {
+int moe_w4(qarl_ctx* ctx, int fmt, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
+           int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w13z,
+           const uint8_t* w2p, const void* w2s, const uint8_t* w2z, void* out, void* workspace,
+           size_t workspace_bytes, const qarl_moe_debug* dbg, void* stream) {
   if (!ctx || M < 0 || H <= 0 || I <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
   // the down tile spans 256 adjacent weight rows of one expert
   if (H % 256 || I % kBlock || E > 1024 || M * k >= 0x7FFFFF00ll || E * 2 * I > 0x7FFFFF00ll)
     return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
-  if (!x || !ids || !wts || !w13p || !w13s || !w13z || !w2p || !w2s || !w2z || !out || !workspace)
-    return QARL_ERR_INVALID_ARG;
+  if (!x || !ids || !wts || !w13p || !w13s || !w2p || !w2s || !out || !workspace) return QARL_ERR_INVALID_ARG;
+  if (fmt == kFmtInt4 && (!w13z || !w2z)) return QARL_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(w13p) || !aligned16(w2p) || !aligned16(out) ||
       (reinterpret_cast<uintptr_t>(w13s) & 1u) || (reinterpret_cast<uintptr_t>(w2s) & 1u) ||
       (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -172,6 +160,7 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const f
   uint16_t* h = reinterpret_cast<uint16_t*>(ws + pl.h);
   GemmW4Args g{};
   g.mode = kModeGateUp;
+  g.fmt = fmt;
   g.a_bf16 = x_sorted;
   g.rows_total = P;
   g.K = H;
@@ -190,6 +179,7 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const f
   uint16_t* contrib = reinterpret_cast<uint16_t*>(ws + pl.contrib);
   GemmW4Args d{};
   d.mode = kModeDown;
+  d.fmt = fmt;
   d.a_bf16 = h;
   d.rows_total = P;
   d.K = I;
@@ -224,6 +214,57 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const f
       return cuda_fail(ctx, e, "copy h");
   }
   return QARL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qarl_quantize_weight_w4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                            void* scales, uint8_t* zeros, void* stream) {
+  return quantize_w4(ctx, kFmtInt4, w, E, N, K, packed, scales, zeros, nullptr, nullptr, nullptr, stream);
+}
+
+int qarl_quantize_weight_w4_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                                    void* scales, uint8_t* zeros, uint8_t* pub_packed, void* pub_scales,
+                                    uint8_t* pub_zeros, void* stream) {
+  return quantize_w4(ctx, kFmtInt4, w, E, N, K, packed, scales, zeros, pub_packed, pub_scales, pub_zeros, stream);
+}
+
+int qarl_quantize_weight_fp4(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* packed,
+                             void* scales, uint8_t* pub_packed, void* pub_scales, void* stream) {
+  return quantize_w4(ctx, kFmtE2m1, w, E, N, K, packed, scales, nullptr, pub_packed, pub_scales, nullptr, stream);
+}
+
+int qarl_linear_fwd_w4a16(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wp, const void* ws,
+                          const uint8_t* wz, int64_t N, void* y, float* y_f32, void* stream) {
+  return linear_w4(ctx, kFmtInt4, x, M, K, wp, ws, wz, N, y, y_f32, stream);
+}
+
+int qarl_linear_fwd_fp4a16(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wp, const void* ws,
+                           int64_t N, void* y, float* y_f32, void* stream) {
+  return linear_w4(ctx, kFmtE2m1, x, M, K, wp, ws, nullptr, N, y, y_f32, stream);
+}
+
+int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
+                       int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w13z,
+                       const uint8_t* w2p, const void* w2s, const uint8_t* w2z, void* out, void* workspace,
+                       size_t workspace_bytes, const qarl_moe_debug* dbg, void* stream) {
+  return moe_w4(ctx, kFmtInt4, x, ids, wts, M, H, I, E, k, w13p, w13s, w13z, w2p, w2s, w2z, out, workspace,
+                workspace_bytes, dbg, stream);
+}
+
+int qarl_moe_fwd_fp4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
+                        int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w2p,
+                        const void* w2s, void* out, void* workspace, size_t workspace_bytes,
+                        const qarl_moe_debug* dbg, void* stream) {
+  return moe_w4(ctx, kFmtE2m1, x, ids, wts, M, H, I, E, k, w13p, w13s, nullptr, w2p, w2s, nullptr, out, workspace,
+                workspace_bytes, dbg, stream);
+}
+
+size_t qarl_moe_w4a16_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
+  if (M <= 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0) return 0;
+  return plan_moe_w4(M, H, I, E, k).total;
 }
 
 int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w, int64_t M, int64_t N, int64_t K,

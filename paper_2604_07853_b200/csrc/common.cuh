@@ -141,7 +141,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
 
 // ---- W4A16 (4-bit group-quantized weights, bf16 activations) --------------------------------
-cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
+// 4-bit weight formats (Sec. 2.2): unsigned integer codes with a zero point, or e2m1 floating point
+enum W4Format { kFmtInt4 = 0, kFmtE2m1 = 1 };
+cudaError_t launch_quantize_weight_w4(const Launch& L, int fmt, const uint16_t* w, int64_t E, int64_t N, int64_t K,
                                       uint8_t* packed, uint16_t* scales, uint8_t* zeros,
                                       uint8_t* pub_packed = nullptr, uint16_t* pub_scales = nullptr,
                                       uint8_t* pub_zeros = nullptr);
@@ -151,12 +153,13 @@ cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, i
 
 struct GemmW4Args {
   GemmMode mode;
+  int fmt;                  // W4Format
   const uint16_t* a_bf16;   // [rows_total, K]
   int64_t rows_total;
   int64_t K;
   const uint8_t* b_packed;  // [E, N, K/2]
   const uint16_t* b_scales; // bf16 bits [E, K/128, N]
-  const uint8_t* b_zeros;   // [E, K/128, N]
+  const uint8_t* b_zeros;   // [E, K/128, N] (integer format only)
   int64_t N;
   int64_t E;
   const int32_t* offsets;   // row groups per expert, or nullptr (dense)

@@ -160,9 +160,34 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, uint32_t zc2, uint32_t
                     dequant_pair(w >> 12, zc2, s2));
 }
 
+// e2m1 codes (Sec. 2.2, floating-point quantization): sign | 2 exponent bits (bias 1) | 1 mantissa bit.
+// Placed at bits 15 | 8..7 | 6 of a bf16, a code reads as its own value times 2^-126 (the code's
+// subnormals 0 and 0.5 land on bf16 subnormals), so two exact-or-once-rounded multiplications give
+// w^ = bf16(s * value): first by 2^a, exact, then by c = s 2^(126 - a); value has 2 significant bits and s
+// 8, so the last product is the single rounding.  a is chosen per group so that both factors stay
+// finite and normal for every bf16 s: a = min(127, E_s - 1) with E_s the exponent field of s.
+__device__ __forceinline__ void fp4_group_consts(uint32_t s_bits, uint32_t& c1x2, uint32_t& c2x2) {
+  const uint32_t es = (s_bits >> 7) & 0xFFu;
+  const uint32_t a = min(127u, es - 1u);
+  c1x2 = ((a + 127u) << 7) * 0x00010001u;
+  c2x2 = ((s_bits & 0x7Fu) | ((es + 126u - a) << 7)) * 0x00010001u;
+}
+__device__ __forceinline__ uint32_t dequant_bits_fp4(uint32_t x6, uint32_t x12, uint32_t c1x2, uint32_t c2x2) {
+  const uint32_t t = (x6 & 0x01C001C0u) | (x12 & 0x80008000u);
+  uint32_t u, v;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(u) : "r"(t), "r"(c1x2));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(u), "r"(c2x2));
+  return v;
+}
+// Eight e2m1 codes of one 32-bit word (pairs in bits [4j, 4j+4) and [16+4j, 20+4j)) -> eight bf16 in K order.
+__device__ __forceinline__ uint4 dequant_word_fp4(uint32_t w, uint32_t c1x2, uint32_t c2x2) {
+  return make_uint4(dequant_bits_fp4(w << 6, w << 12, c1x2, c2x2), dequant_bits_fp4(w << 2, w << 8, c1x2, c2x2),
+                    dequant_bits_fp4(w >> 2, w << 4, c1x2, c2x2), dequant_bits_fp4(w >> 6, w, c1x2, c2x2));
+}
+
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-template <int MODE, int MT>
+template <int MODE, int MT, int FMT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
   using C = Cfg<MT>;
@@ -324,14 +349,19 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
     if (T < total_tiles) {
       TileCoord c = decode_tile(s->off, s->prefix, C::kRows, T, cur_e);
       int64_t idx = sz_index(c, 0);
-      uint32_t s_next = __ldg(p.b_scales + idx), z_next = __ldg(p.b_zeros + idx);
+      uint32_t s_next = __ldg(p.b_scales + idx), z_next = FMT == kFmtInt4 ? __ldg(p.b_zeros + idx) : 0u;
       for (;;) {
         const int Tn = T + num_ctas;
         const bool has_next = Tn < total_tiles;
         TileCoord cn = c;
         for (int g = 0; g < KG; ++g) {
-          const uint32_t s2 = s_next | (s_next << 16);
-          const uint32_t zc2 = (0x4300u | z_next) * 0x00010001u;  // bf16x2 of 128 + z
+          uint32_t s2, zc2;  // integer: s and 128 + z as bf16x2; e2m1: the two per-group factors
+          if constexpr (FMT == kFmtInt4) {
+            s2 = s_next | (s_next << 16);
+            zc2 = (0x4300u | z_next) * 0x00010001u;
+          } else {
+            fp4_group_consts(s_next, zc2, s2);
+          }
           if (g + 1 < KG) {
             idx = sz_index(c, g + 1);
           } else if (has_next) {
@@ -339,7 +369,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
             idx = sz_index(cn, 0);
           }
           s_next = __ldg(p.b_scales + idx);
-          z_next = __ldg(p.b_zeros + idx);
+          if constexpr (FMT == kFmtInt4) z_next = __ldg(p.b_zeros + idx);
           const uint32_t step = step0 + 2 * g + grp;
           const uint32_t qs = step % kQStages, q_phase = (step / kQStages) & 1u;
           const uint32_t ds = step % kDqStages, dq_phase = (step / kDqStages) & 1u;
@@ -355,7 +385,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           const uint32_t words[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
           for (int i = 0; i < 8; ++i)  // 16-byte chunk i of the row lands at chunk i ^ (row % 8): SWIZZLE_128B
-            *reinterpret_cast<uint4*>(row_dst + ((i ^ (n & 7)) << 4)) = dequant_word(words[i], zc2, s2);
+            *reinterpret_cast<uint4*>(row_dst + ((i ^ (n & 7)) << 4)) =
+                FMT == kFmtInt4 ? dequant_word(words[i], zc2, s2) : dequant_word_fp4(words[i], zc2, s2);
           fence_proxy_async_smem();  // generic-proxy stores -> visible to the tensor core's async proxy
           __syncwarp();
           if (lane == 0) mbar_arrive(&s->dq_full[ds]);
@@ -488,12 +519,12 @@ CUresult make_tmap_a(EncodeTiledFn encode, CUtensorMap* m, const void* base, uin
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int MODE, int MT>
+template <int MODE, int MT, int FMT>
 cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
   static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
   bool& attr_set = attr_set_dev[L.device & 63];
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE, MT, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem_bytes<MT>()));
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -503,14 +534,20 @@ cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& 
   const int64_t m_tiles_max = a.rows_total / Cfg<MT>::kRows + a.E;
   const int grid = static_cast<int>(std::min<int64_t>(L.sm_count, m_tiles_max * p.n_tiles));
   ++*L.launches;
-  return launch_pdl(gemm_w4a16_kernel<MODE, MT>, static_cast<unsigned>(grid), kThreads, smem_bytes<MT>(), L.stream, ta, p);
+  return launch_pdl(gemm_w4a16_kernel<MODE, MT, FMT>, static_cast<unsigned>(grid), kThreads, smem_bytes<MT>(), L.stream,
+                    ta, p);
+}
+
+template <int MODE, int FMT>
+cudaError_t launch_fmt(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
+  // groups of at most 128 rows on average (decode-sized calls): 128-row tiles
+  if (a.rows_total <= a.E * BM) return launch_mode<MODE, 1, FMT>(L, ta, p, a);
+  return launch_mode<MODE, 2, FMT>(L, ta, p, a);
 }
 
 template <int MODE>
 cudaError_t launch_mt(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
-  // groups of at most 128 rows on average (decode-sized calls): 128-row tiles
-  if (a.rows_total <= a.E * BM) return launch_mode<MODE, 1>(L, ta, p, a);
-  return launch_mode<MODE, 2>(L, ta, p, a);
+  return a.fmt == kFmtE2m1 ? launch_fmt<MODE, kFmtE2m1>(L, ta, p, a) : launch_fmt<MODE, kFmtInt4>(L, ta, p, a);
 }
 
 }  // namespace

@@ -173,6 +173,39 @@ __device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float inv, 
   return word;
 }
 
+// ---- FP4 (e2m1) weights (Sec. 2.2, floating-point quantization): s = amax / 6, W_q = [W / s]_FP4 ----
+// Same groups, code order and storage as the integer format; s = bf16(max(amax, 2^-40) / 6).
+// The magnitude code of |w| / s rounded to the nearest of 0, .5, 1, 1.5, 2, 3, 4, 6 (ties to the even
+// code, saturating) is the number of rounding boundaries it passes: .25 .75 1.25 1.75 2.5 3.5 5, where a
+// value exactly on a boundary goes to the neighbour with mantissa bit 0 (so the boundaries are
+// exclusive, inclusive, exclusive, ...).  |w| / s against a boundary b compares like |w| against b s,
+// and b s is exact in fp32 (3 x 8 significant bits), as is the comparison of the IEEE quotient:
+// two distinct numbers of at most 8 and 11 bits differ by more than the quotient's rounding error.
+struct Fp4Bounds { float t[7]; };
+__device__ __forceinline__ Fp4Bounds fp4_bounds(float s) {
+  Fp4Bounds b;
+  const float k[7] = {0.25f, 0.75f, 1.25f, 1.75f, 2.5f, 3.5f, 5.0f};
+#pragma unroll
+  for (int i = 0; i < 7; ++i) b.t[i] = __fmul_rn(k[i], s);
+  return b;
+}
+__device__ __forceinline__ uint32_t fp4_code(uint32_t bits_hi, const Fp4Bounds& b) {  // bf16 bits in [16, 32)
+  const float a = __uint_as_float(bits_hi & 0x7FFF0000u);
+  const uint32_t mag = (a > b.t[0]) + (a >= b.t[1]) + (a > b.t[2]) + (a >= b.t[3]) + (a > b.t[4]) + (a >= b.t[5]) +
+                       (a > b.t[6]);
+  return ((bits_hi >> 28) & 8u) | mag;
+}
+__device__ __forceinline__ uint32_t fp4_word(const uint4& v, const Fp4Bounds& b) {
+  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+  uint32_t word = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    word |= fp4_code(in[j] << 16, b) << (4 * j);
+    word |= fp4_code(in[j] & 0xFFFF0000u, b) << (4 * j + 16);
+  }
+  return word;
+}
+
 __device__ __forceinline__ void minmax_u4(const uint4& v, float& lo, float& hi) {
   const uint32_t in[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -183,6 +216,7 @@ __device__ __forceinline__ void minmax_u4(const uint4& v, float& lo, float& hi) 
   }
 }
 
+template <int FMT>  // 0: unsigned 4-bit integer with zero point, 1: e2m1 (no zero point: `zeros` unused)
 __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t* __restrict__ w, int64_t rows,
                                                                  int64_t N, int64_t K,
                                                                  uint8_t* __restrict__ packed,
@@ -216,13 +250,23 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
     lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
     hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
   }
-  const float range = fmaxf(__fsub_rn(hi, lo), kAmaxFloor);
-  const uint32_t s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
-  const float s = bf16_bits_to_f32(s_bits);
-  const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
-  const float inv = __fdiv_rn(1.0f, s);
-  const float zm = zf + 8388608.0f;
-  const uint2 out = make_uint2(w4_word(v0, s, inv, zm), w4_word(v1, s, inv, zm));
+  uint32_t s_bits;
+  float zf = 0.0f;
+  uint2 out;
+  if constexpr (FMT == 0) {
+    const float range = fmaxf(__fsub_rn(hi, lo), kAmaxFloor);
+    s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
+    const float s = bf16_bits_to_f32(s_bits);
+    zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
+    const float inv = __fdiv_rn(1.0f, s);
+    const float zm = zf + 8388608.0f;
+    out = make_uint2(w4_word(v0, s, inv, zm), w4_word(v1, s, inv, zm));
+  } else {
+    const float amax = fmaxf(fmaxf(-lo, hi), kAmaxFloor);  // lo <= 0 <= hi
+    s_bits = f32_to_bf16_bits(__fdiv_rn(amax, 6.0f));
+    const Fp4Bounds b = fp4_bounds(bf16_bits_to_f32(s_bits));
+    out = make_uint2(fp4_word(v0, b), fp4_word(v1, b));
+  }
   if (!live) return;
   const uint32_t e32 = row32 / static_cast<uint32_t>(N);
   const int64_t e = e32, n = row32 - e32 * static_cast<uint32_t>(N);
@@ -237,10 +281,10 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
   if (sub == 0) {
     const int64_t idx = (e * kb + g) * N + n;
     scales[idx] = static_cast<uint16_t>(s_bits);
-    zeros[idx] = static_cast<uint8_t>(zf);
+    if (FMT == 0) zeros[idx] = static_cast<uint8_t>(zf);
     if (pub_packed) {
       pub_scales[idx] = static_cast<uint16_t>(s_bits);
-      pub_zeros[idx] = static_cast<uint8_t>(zf);
+      if (FMT == 0) pub_zeros[idx] = static_cast<uint8_t>(zf);
     }
   }
 }
@@ -289,15 +333,16 @@ cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, i
                     dst_rows, fanout, M * fanout, pair_w, sorted_w);
 }
 
-cudaError_t launch_quantize_weight_w4(const Launch& L, const uint16_t* w, int64_t E, int64_t N, int64_t K,
+cudaError_t launch_quantize_weight_w4(const Launch& L, int fmt, const uint16_t* w, int64_t E, int64_t N, int64_t K,
                                       uint8_t* packed, uint16_t* scales, uint8_t* zeros, uint8_t* pub_packed,
                                       uint16_t* pub_scales, uint8_t* pub_zeros) {
   const int64_t groups = E * N * (K / kBlock);
   if (groups == 0) return cudaSuccess;
   const int64_t blocks = (groups * 8 + 255) / 256;
   ++*L.launches;
-  return launch_pdl(quantize_weight_w4_kernel, static_cast<unsigned>(blocks), 256, 0, L.stream, w, E * N, N, K, packed,
-                    scales, zeros, pub_packed, pub_scales, pub_zeros);
+  return launch_pdl(fmt == kFmtE2m1 ? quantize_weight_w4_kernel<1> : quantize_weight_w4_kernel<0>,
+                    static_cast<unsigned>(blocks), 256, 0, L.stream, w, E * N, N, K, packed, scales, zeros, pub_packed,
+                    pub_scales, pub_zeros);
 }
 
 cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,

@@ -60,6 +60,23 @@ def w_hat_of(q):
     return oracle.dequant_w4(*host_weights(q))
 
 
+class Int4:
+    """The calls of the integer format, so that the checks below also serve the e2m1 format."""
+    @staticmethod
+    def quantize(ctx, w):
+        return ctx.quantize_weight_w4(w)
+
+    @staticmethod
+    def linear(ctx, x, q, **kw):
+        return ctx.linear_fwd_w4a16(x, *q, **kw)
+
+    @staticmethod
+    def moe(ctx, x, ids, wts, q13, q2, **kw):
+        return ctx.moe_fwd_w4a16(x, ids, wts, q13, q2, **kw)
+
+    w_hat = staticmethod(w_hat_of)
+
+
 # ------------------------------------------------------------------------------ quantizer
 @pytest.mark.parametrize("e,n,k", [(1, 128, 128), (3, 256, 384), (2, 1536, 2048), (4, 640, 256)])
 def test_quantizer_bit_exact(ctx, e, n, k):
@@ -120,17 +137,17 @@ def test_quantizer_publish_writes_two_equal_copies(ctx):
 
 
 # ------------------------------------------------------------------------------ dense GEMM
-def check_linear(ctx, seed, m, n, k):
+def check_linear(ctx, seed, m, n, k, fmt=Int4):
     """fp32: |gpu - oracle| <= 1e-3 * ||x_row|| * ||w^_col|| (the oracle sums exactly; the tensor
     core adds K exact products in fp32).  bf16: the rounding of the GPU's own fp32, bit for bit,
     and within 1 ulp of the oracle's except where cancellation makes an ulp smaller than the
     fp32 bound (rare)."""
     case = inputs.linear_case(seed, m, n, k)
-    q = ctx.quantize_weight_w4(bits_to_torch(case.w))
+    q = fmt.quantize(ctx, bits_to_torch(case.w))
     xt = bits_to_torch(case.x)
-    y, y32 = ctx.linear_fwd_w4a16(xt, *q, want_f32=True)
+    y, y32 = fmt.linear(ctx, xt, q, want_f32=True)
     assert ctx.poll() == 0
-    w_hat = w_hat_of(q)
+    w_hat = fmt.w_hat(q)
     o32, o16 = oracle.linear_bf16(case.x, w_hat)
     g32, g16 = y32.cpu().numpy(), torch_to_bits(y)
     nx = np.linalg.norm(inputs.bf16_bits_to_f32(case.x).astype(np.float64), axis=1)
@@ -179,19 +196,20 @@ def test_linear_rows_do_not_depend_on_the_batch(ctx):
 
 # ------------------------------------------------------------------------------ MoE layer
 class DeviceCase:
-    def __init__(self, ctx, case):
+    def __init__(self, ctx, case, fmt=Int4):
         self.case = case
+        self.fmt = fmt
         self.x = bits_to_torch(case.x)
         self.ids = to_dev(case.ids)
         self.wts = to_dev(case.weights)
-        self.w13 = ctx.quantize_weight_w4(bits_to_torch(case.w13))
-        self.w2 = ctx.quantize_weight_w4(bits_to_torch(case.w2))
+        self.w13 = fmt.quantize(ctx, bits_to_torch(case.w13))
+        self.w2 = fmt.quantize(ctx, bits_to_torch(case.w2))
 
     def run(self, ctx, debug=False, rows=None):
         x, ids, wts = self.x, self.ids, self.wts
         if rows is not None:
             x, ids, wts = x[rows].contiguous(), ids[rows].contiguous(), wts[rows].contiguous()
-        return ctx.moe_fwd_w4a16(x, ids, wts, self.w13, self.w2, debug=debug)
+        return self.fmt.moe(ctx, x, ids, wts, self.w13, self.w2, debug=debug)
 
 
 def _norm_tol(a_bits, w_hat_bits):
@@ -200,12 +218,12 @@ def _norm_tol(a_bits, w_hat_bits):
     return 1e-3 * na[:, None] * nw[None, :]
 
 
-def check_moe(ctx, case, end_to_end=True):
-    dc = DeviceCase(ctx, case)
+def check_moe(ctx, case, end_to_end=True, fmt=Int4):
+    dc = DeviceCase(ctx, case, fmt)
     out, d = dc.run(ctx, debug=True)
     assert ctx.poll() == 0
     c = case
-    w13h, w2h = w_hat_of(dc.w13), w_hat_of(dc.w2)
+    w13h, w2h = fmt.w_hat(dc.w13), fmt.w_hat(dc.w2)
 
     # 1. permutation: bit-exact
     off, srt, _ = oracle.permute(c.ids, c.E)
