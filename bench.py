@@ -430,16 +430,17 @@ def main():
         }
         del wr
 
-    # ---------------- W4A16 variant of the same layer (4-bit weights, bf16 activations)
-    if not args.no_w4a16:
-        q13 = ctx.quantize_weight_w4(w13)
-        q2 = ctx.quantize_weight_w4(w2)
+    # ---------------- 4-bit weight-only variants of the same layer (bf16 activations): integer codes with a
+    # zero point ("w4a16") and e2m1 floating point ("fp4a16"); same storage, same kernels
+    def bench_4bit(label, quantize, moe_fwd):
+        q13 = quantize(w13)
+        q2 = quantize(w2)
         ws4 = torch.empty(ctx.moe_w4a16_workspace_bytes(M_TRAIN, H, I, E, TOPK), dtype=torch.uint8, device=dev)
 
         def step4():
-            ctx.quantize_weight_w4(w13, out=q13)
-            ctx.quantize_weight_w4(w2, out=q2)
-            ctx.moe_fwd_w4a16(x, ids, wts, q13, q2, out=out, workspace=ws4)
+            quantize(w13, out=q13)
+            quantize(w2, out=q2)
+            moe_fwd(x, ids, wts, q13, q2, out=out, workspace=ws4)
 
         steps4 = max(args.steps // 2, 10)
         for _ in range(3):
@@ -461,7 +462,7 @@ def main():
         gu_tf = 2.0 * M_TRAIN * TOPK * H * 2 * I / (gu4 * 1e-3) / 1e12
         dn_tf = 2.0 * M_TRAIN * TOPK * I * H / (dn4 * 1e-3) / 1e12
         w4 = {
-            "workload": f"moe_ffn_train_M{M_TRAIN} with W4A16 weights (per-step 4-bit quantization + layer forward)",
+            "workload": f"moe_ffn_train_M{M_TRAIN} with {label} weights (per-step 4-bit quantization + layer forward)",
             "ms_per_step": ms4, "tokens_per_s": world * M_TRAIN / (ms4 * 1e-3),
             "stage_ms": {k: v[0] / steps4 for k, v in st4.items() if v[1]},
             "gate_up_tflops": gu_tf, "down_tflops": dn_tf,
@@ -477,7 +478,7 @@ def main():
 
         def dstep4(i):
             a, b = sets4[i & 1]
-            ctx.moe_fwd_w4a16(xd4, idd4, wtd4, a, b, out=outd4, workspace=ws4)
+            moe_fwd(xd4, idd4, wtd4, a, b, out=outd4, workspace=ws4)
 
         for i in range(10):
             dstep4(i)
@@ -495,14 +496,17 @@ def main():
         ctx.check_device_status()
         wbytes4 = sum(t.numel() * t.element_size() for t in (*q13, *q2)) + 2 * M_DECODE * H * 2
         w4["decode"] = {
-            "workload": "moe_ffn_decode_M256 with W4A16 weights (pre-quantized, two copies alternated)",
+            "workload": f"moe_ffn_decode_M256 with {label} weights (pre-quantized, two copies alternated)",
             "ms_per_step": d4_ms, "tokens_per_s": world * M_DECODE / (d4_ms * 1e-3),
             "algorithmic_bytes": wbytes4, "gbs": wbytes4 / (d4_ms * 1e-3) / 1e9,
             "frac_hbm_measured": wbytes4 / (d4_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
             "stage_ms": {k: v[0] / dsteps4 for k, v in dst4.items() if v[1]},
         }
-        result["w4a16"] = w4
-        del q13, q2, sets4, ws4
+        return w4
+
+    if not args.no_w4a16:
+        result["w4a16"] = bench_4bit("W4A16", ctx.quantize_weight_w4, ctx.moe_fwd_w4a16)
+        result["fp4a16"] = bench_4bit("FP4A16 (e2m1)", ctx.quantize_weight_fp4, ctx.moe_fwd_fp4a16)
 
     # ---------------- full-precision backward of the dense projection (QKV shape of the training configuration)
     if not args.no_backward:

@@ -142,83 +142,124 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint16_t* __res
 // out inside as [word quad 0..1][row 0..127][16 bytes] so that the 128 threads that expand it
 // read consecutive 16-byte pieces.  Scales (bf16 bits) and zero points are stored group-major,
 // [E][K/128][N], contiguous along the weight rows.
-// rint(w / s) + z clamped to 0..15 for one element, equal to the IEEE-division form bit for bit
-// but without a division per element.  w and s are bf16 values (8 significant bits each), so the
-// exact quotient is either exactly half-way between two integers or at least 2^-14 (relative) away
-// from such a point: the product with inv = fl(1 / s) (relative error ~2^-23) then rounds to the
-// same integer except at exact ties, which the exact residual r = w - q0 s identifies
-// (2 r = +-s) and resolves to the even neighbour.
-__device__ __forceinline__ uint32_t w4_code(float w, float s, float inv, float zm) {
-  const float kMagic = 12582912.0f;               // 1.5 * 2^23: adding it rounds to an integer
-  float q0 = __fsub_rn(__fmaf_rn(w, inv, kMagic), kMagic);
-  const float r = __fmaf_rn(-q0, s, w);           // exact: q0 s has at most 13 significant bits
-  if (fabsf(__fadd_rn(r, r)) == s) {              // tie between q0 and q0 + sign(r)
-    const float other = r > 0.0f ? q0 + 1.0f : q0 - 1.0f;
-    const float half = 0.5f * q0;
-    if (__fsub_rn(__fadd_rn(half, kMagic), kMagic) != half) q0 = other;  // q0 odd: the other one is even
-  }
-  // zm = z + 2^23: the code is clamped in that domain, where the integer sits in the low mantissa bits
-  const float v = fminf(fmaxf(__fadd_rn(q0, zm), 8388608.0f), 8388623.0f);
-  return __float_as_uint(v) & 15u;
-}
+__device__ __forceinline__ __nv_bfloat162 as_bf2(uint32_t u) { return *reinterpret_cast<__nv_bfloat162*>(&u); }
+__device__ __forceinline__ uint32_t bf2_bits(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
 
-__device__ __forceinline__ uint32_t w4_word(const uint4& v, float s, float inv, float zm) {
-  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
-  uint32_t word = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    word |= w4_code(bf16_bits_to_f32(in[j] & 0xFFFFu), s, inv, zm) << (4 * j);
-    word |= w4_code(__uint_as_float(in[j] & 0xFFFF0000u), s, inv, zm) << (4 * j + 16);
-  }
+__device__ __forceinline__ uint32_t fma_bf2(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t add_bf2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// Whether a boundary was passed is read from a sign bit, with integer instructions only.  d is the
+// bf16x2 difference value - boundary (never a subnormal: the operands have few bits).  Adding 0x0080 to
+// each half (one exponent step) makes +0 positive and keeps every other sign: sign clear <=> d >= 0, for
+// boundaries that belong to the upper code.  Subtracting it makes +0 negative and keeps every other sign
+// (a borrow out of the low half can only turn a high half that is +0 or positive-minimal around, and the
+// latter cannot occur): sign clear <=> d > 0, for boundaries that belong to the lower code.
+constexpr uint32_t kTieUp = 0x00800080u, kTieDown = 0xFF7FFF80u, kSigns = 0x80008000u;
+
+// q = clamp(rint(w / s) + z, 0, 15) for two adjacent elements at once, equal to the IEEE-division form
+// bit for bit but without a division: q is the number of boundaries (j - z - 1/2) s, j = 1..15, that w
+// passes, where a w exactly on a boundary goes to the even neighbour of rint.  w and s are bf16 (8
+// significant bits), the multiplier m = j - z - 1/2 has at most 6, so w - m s is exact before the one
+// rounding of a fused multiply-add, which keeps its sign and gives zero only for an exact tie, also in
+// bf16; and the IEEE quotient w / s compares with m as w does with m s, because distinct numbers of 8 and
+// 14 bits differ by far more than the quotient's rounding error.  A four-level binary search over j
+// (8, then +-4, +-2, +-1) therefore yields the four bits of q, one bf16x2 FMA per level.
+// Ties: the boundary below code j belongs to rint value j - 1 - z; it goes up when that is odd, i.e.
+// for even j when z is even and for odd j when z is odd.
+struct W4Group {
+  uint32_t neg_s;         // -s twice
+  uint32_t m8;            // 7.5 - z twice: the first boundary
+  uint32_t tie_hi, tie_lo;  // kTieUp / kTieDown for the first three levels (even j) / the last level (odd j)
+};
+__device__ __forceinline__ W4Group w4_group(uint32_t s_bits, float zf) {
+  W4Group g;
+  g.neg_s = (s_bits | 0x8000u) * 0x00010001u;
+  g.m8 = f32_to_bf16_bits(7.5f - zf) * 0x00010001u;   // a half-integer below 16: exact
+  const bool z_odd = (static_cast<int>(zf) & 1) != 0;
+  g.tie_hi = z_odd ? kTieDown : kTieUp;
+  g.tie_lo = z_odd ? kTieUp : kTieDown;
+  return g;
+}
+// codes of the pair (elements 2j, 2j+1 of a word's eight) OR-ed into `word` at bits [4j, 4j+4) and [16+4j, 20+4j)
+template <int J>
+__device__ __forceinline__ uint32_t w4_codes2(uint32_t word, uint32_t w2, const W4Group& g) {
+  uint32_t m = g.m8;
+  uint32_t t = fma_bf2(m, g.neg_s, w2) + g.tie_hi;                       // j = 8
+  word |= (~t >> (12 - 4 * J)) & (0x00080008u << (4 * J));
+  m = add_bf2(m, 0xC080C080u ^ (~t & kSigns));                           // +4 where passed, else -4
+  t = fma_bf2(m, g.neg_s, w2) + g.tie_hi;
+  word |= (~t >> (13 - 4 * J)) & (0x00040004u << (4 * J));
+  m = add_bf2(m, 0xC000C000u ^ (~t & kSigns));                           // +-2
+  t = fma_bf2(m, g.neg_s, w2) + g.tie_hi;
+  word |= (~t >> (14 - 4 * J)) & (0x00020002u << (4 * J));
+  m = add_bf2(m, 0xBF80BF80u ^ (~t & kSigns));                           // +-1
+  t = fma_bf2(m, g.neg_s, w2) + g.tie_lo;
+  word |= (~t >> (15 - 4 * J)) & (0x00010001u << (4 * J));
   return word;
+}
+__device__ __forceinline__ uint32_t w4_word(const uint4& v, const W4Group& g) {
+  return w4_codes2<3>(w4_codes2<2>(w4_codes2<1>(w4_codes2<0>(0u, v.x, g), v.y, g), v.z, g), v.w, g);
 }
 
 // ---- FP4 (e2m1) weights (Sec. 2.2, floating-point quantization): s = amax / 6, W_q = [W / s]_FP4 ----
 // Same groups, code order and storage as the integer format; s = bf16(max(amax, 2^-40) / 6).
 // The magnitude code of |w| / s rounded to the nearest of 0, .5, 1, 1.5, 2, 3, 4, 6 (ties to the even
-// code, saturating) is the number of rounding boundaries it passes: .25 .75 1.25 1.75 2.5 3.5 5, where a
+// code, saturating) is the number of rounding boundaries b = .25 .75 1.25 1.75 2.5 3.5 5 it passes, where a
 // value exactly on a boundary goes to the neighbour with mantissa bit 0 (so the boundaries are
-// exclusive, inclusive, exclusive, ...).  |w| / s against a boundary b compares like |w| against b s,
-// and b s is exact in fp32 (3 x 8 significant bits), as is the comparison of the IEEE quotient:
-// two distinct numbers of at most 8 and 11 bits differ by more than the quotient's rounding error.
-struct Fp4Bounds { float t[7]; };
-__device__ __forceinline__ Fp4Bounds fp4_bounds(float s) {
-  Fp4Bounds b;
-  const float k[7] = {0.25f, 0.75f, 1.25f, 1.75f, 2.5f, 3.5f, 5.0f};
-#pragma unroll
-  for (int i = 0; i < 7; ++i) b.t[i] = __fmul_rn(k[i], s);
-  return b;
-}
-__device__ __forceinline__ uint32_t fp4_code(uint32_t bits_hi, const Fp4Bounds& b) {  // bf16 bits in [16, 32)
-  const float a = __uint_as_float(bits_hi & 0x7FFF0000u);
-  const uint32_t mag = (a > b.t[0]) + (a >= b.t[1]) + (a > b.t[2]) + (a >= b.t[3]) + (a > b.t[4]) + (a >= b.t[5]) +
-                       (a > b.t[6]);
-  return ((bits_hi >> 28) & 8u) | mag;
-}
-__device__ __forceinline__ uint32_t fp4_word(const uint4& v, const Fp4Bounds& b) {
-  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
-  uint32_t word = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    word |= fp4_code(in[j] << 16, b) << (4 * j);
-    word |= fp4_code(in[j] & 0xFFFF0000u, b) << (4 * j + 16);
-  }
+// exclusive, inclusive, exclusive, ...).  As above, the sign of |w| - b s from one bf16x2 FMA decides
+// each comparison exactly.  Three levels give the three bits: b = 1.75 (>=); then 3.5 or .75 (>=); then 5,
+// 2.5, 1.25 or .25 (>).  With P1, P2 = +-1 for passed / not passed, the next boundaries are the exact
+// bf16 polynomials  b1 = 2.125 + 1.375 P1  and  b0 = (2.25 + 1.5 P1) + P2 (.875 + .375 P1),  kept negated.
+template <int J>
+__device__ __forceinline__ uint32_t fp4_codes2(uint32_t word, uint32_t w2, uint32_t s2) {
+  const uint32_t a2 = w2 & 0x7FFF7FFFu;
+  uint32_t t = fma_bf2(0xBFE0BFE0u /* -1.75 */, s2, a2) + kTieUp;
+  word |= (~t >> (13 - 4 * J)) & (0x00040004u << (4 * J));
+  const uint32_t p1 = 0x3F803F80u | (t & kSigns);                        // +1 where passed, else -1
+  const uint32_t nb1 = fma_bf2(p1, 0xBFB0BFB0u /* -1.375 */, 0xC008C008u /* -2.125 */);
+  t = fma_bf2(nb1, s2, a2) + kTieUp;
+  word |= (~t >> (14 - 4 * J)) & (0x00020002u << (4 * J));
+  const uint32_t p2 = 0x3F803F80u | (t & kSigns);
+  const uint32_t u = fma_bf2(p1, 0xBFC0BFC0u /* -1.5 */, 0xC010C010u /* -2.25 */);
+  const uint32_t v = fma_bf2(p1, 0xBEC0BEC0u /* -.375 */, 0xBF60BF60u /* -.875 */);
+  t = fma_bf2(fma_bf2(p2, v, u), s2, a2) + kTieDown;
+  word |= (~t >> (15 - 4 * J)) & (0x00010001u << (4 * J));
+  if (J == 3) word |= w2 & 0x80008000u;                                  // sign: bit 3 of the code
+  else word |= (w2 >> (12 - 4 * J)) & (0x00080008u << (4 * J));
   return word;
 }
+__device__ __forceinline__ uint32_t fp4_word(const uint4& v, uint32_t s2) {
+  return fp4_codes2<3>(fp4_codes2<2>(fp4_codes2<1>(fp4_codes2<0>(0u, v.x, s2), v.y, s2), v.z, s2), v.w, s2);
+}
+__device__ __forceinline__ __nv_bfloat162 absmax_u4(const uint4& v, __nv_bfloat162 m) {
+  m = __hmax2(m, as_bf2(v.x & 0x7FFF7FFFu));
+  m = __hmax2(m, as_bf2(v.y & 0x7FFF7FFFu));
+  m = __hmax2(m, as_bf2(v.z & 0x7FFF7FFFu));
+  return __hmax2(m, as_bf2(v.w & 0x7FFF7FFFu));
+}
 
-__device__ __forceinline__ void minmax_u4(const uint4& v, float& lo, float& hi) {
+__device__ __forceinline__ void minmax_u4(const uint4& v, __nv_bfloat162& lo, __nv_bfloat162& hi) {
   const uint32_t in[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const float a = bf16_bits_to_f32(in[j] & 0xFFFFu), b = __uint_as_float(in[j] & 0xFFFF0000u);
-    lo = fminf(lo, fminf(a, b));
-    hi = fmaxf(hi, fmaxf(a, b));
+    lo = __hmin2(lo, as_bf2(in[j]));
+    hi = __hmax2(hi, as_bf2(in[j]));
   }
 }
 
+// A block owns 32 consecutive weight rows (8 threads per row, 16 elements each) and walks a range of
+// their K-groups, so that the row and chunk arithmetic is done once and the next group's 32 bytes are
+// in flight while the current one is encoded.  Rows never straddle an expert (N % 128 == 0).
 template <int FMT>  // 0: unsigned 4-bit integer with zero point, 1: e2m1 (no zero point: `zeros` unused)
-__global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t* __restrict__ w, int64_t rows,
-                                                                 int64_t N, int64_t K,
+__global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t* __restrict__ w, int64_t N, int64_t K,
+                                                                 int groups_per_block,
                                                                  uint8_t* __restrict__ packed,
                                                                  uint16_t* __restrict__ scales,
                                                                  uint8_t* __restrict__ zeros,
@@ -227,64 +268,61 @@ __global__ void __launch_bounds__(256) quantize_weight_w4_kernel(const uint16_t*
                                                                  uint8_t* __restrict__ pub_zeros) {
   pdl_trigger();
   pdl_wait();
-  // 32-bit index arithmetic (the launcher guarantees fewer than 2^31 groups): 64-bit divisions
-  // would cost more instructions than the quantization itself
-  const uint32_t kb = static_cast<uint32_t>(K / kBlock);
-  const uint32_t gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 3;
-  const bool live = gid < static_cast<uint32_t>(rows) * kb;
-  const uint32_t gg = live ? gid : 0u;
-  const uint32_t row32 = gg / kb, g32 = gg - row32 * kb;
-  const int64_t row = row32, g = g32;
+  const int kb = static_cast<int>(K / kBlock);
+  const int g_begin = blockIdx.y * groups_per_block, g_end = min(kb, g_begin + groups_per_block);
+  const uint32_t row = blockIdx.x * 32u + (threadIdx.x >> 3);   // over all experts
   const int sub = threadIdx.x & 7;
-  const uint4* src = reinterpret_cast<const uint4*>(w + row * K + g * kBlock + sub * 16);
-  uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
-  if (live) {
-    v0 = __ldg(src);
-    v1 = __ldg(src + 1);
-  }
-  float lo = 0.0f, hi = 0.0f;
-  minmax_u4(v0, lo, hi);
-  minmax_u4(v1, lo, hi);
+  const uint32_t e = row / static_cast<uint32_t>(N), n = row - e * static_cast<uint32_t>(N);
+  const uint4* src = reinterpret_cast<const uint4*>(w + static_cast<int64_t>(row) * K + sub * 16) + g_begin * 16;
+  // byte offset of this thread's two words in the chunk of K-step 2g + sub/4: words 2(sub%4), 2(sub%4)+1
+  const int64_t chunk0 = (static_cast<int64_t>(e) * (N / kBlock) + (n >> 7)) * (K / 64) + (sub >> 2);
+  int64_t at = (chunk0 + 2 * g_begin) * 4096 + ((sub & 3) >> 1) * 2048 + (n & (kBlock - 1)) * 16 + (sub & 1) * 8;
+  int64_t idx = (static_cast<int64_t>(e) * kb + g_begin) * N + n;
+  if (g_begin >= g_end) return;
+  uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
+  for (int g = g_begin; g < g_end; ++g, src += 16, at += 8192, idx += N) {
+    const uint4 c0 = v0, c1 = v1;
+    if (g + 1 < g_end) {
+      v0 = __ldg(src + 16);
+      v1 = __ldg(src + 17);
+    }
+    uint32_t s_bits;
+    float zf = 0.0f;
+    uint2 out;
+    if constexpr (FMT == 0) {
+      __nv_bfloat162 lo2 = as_bf2(0u), hi2 = as_bf2(0u);  // zero stays representable: lo <= 0 <= hi
+      minmax_u4(c0, lo2, hi2);
+      minmax_u4(c1, lo2, hi2);
 #pragma unroll
-  for (int o = 4; o > 0; o >>= 1) {
-    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
-    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
-  }
-  uint32_t s_bits;
-  float zf = 0.0f;
-  uint2 out;
-  if constexpr (FMT == 0) {
-    const float range = fmaxf(__fsub_rn(hi, lo), kAmaxFloor);
-    s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
-    const float s = bf16_bits_to_f32(s_bits);
-    zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
-    const float inv = __fdiv_rn(1.0f, s);
-    const float zm = zf + 8388608.0f;
-    out = make_uint2(w4_word(v0, s, inv, zm), w4_word(v1, s, inv, zm));
-  } else {
-    const float amax = fmaxf(fmaxf(-lo, hi), kAmaxFloor);  // lo <= 0 <= hi
-    s_bits = f32_to_bf16_bits(__fdiv_rn(amax, 6.0f));
-    const Fp4Bounds b = fp4_bounds(bf16_bits_to_f32(s_bits));
-    out = make_uint2(fp4_word(v0, b), fp4_word(v1, b));
-  }
-  if (!live) return;
-  const uint32_t e32 = row32 / static_cast<uint32_t>(N);
-  const int64_t e = e32, n = row32 - e32 * static_cast<uint32_t>(N);
-  {
-    const int64_t ks = g * 2 + (sub >> 2);  // K-step of 64 elements
-    const int64_t chunk = (e * (N / kBlock) + (n >> 7)) * (K / 64) + ks;
-    const int quad = (sub & 3) >> 1, piece = sub & 1;  // words 2(sub%4), 2(sub%4)+1 of the K-step's eight
-    const int64_t at = chunk * 4096 + quad * 2048 + (n & (kBlock - 1)) * 16 + piece * 8;
+      for (int o = 4; o > 0; o >>= 1) {
+        lo2 = __hmin2(lo2, as_bf2(__shfl_xor_sync(0xFFFFFFFFu, bf2_bits(lo2), o)));
+        hi2 = __hmax2(hi2, as_bf2(__shfl_xor_sync(0xFFFFFFFFu, bf2_bits(hi2), o)));
+      }
+      const float lo = fminf(__low2float(lo2), __high2float(lo2)), hi = fmaxf(__low2float(hi2), __high2float(hi2));
+      const float range = fmaxf(__fsub_rn(hi, lo), kAmaxFloor);
+      s_bits = f32_to_bf16_bits(__fdiv_rn(range, 15.0f));
+      const float s = bf16_bits_to_f32(s_bits);
+      zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.0f), 15.0f);
+      const W4Group grp = w4_group(s_bits, zf);
+      out = make_uint2(w4_word(c0, grp), w4_word(c1, grp));
+    } else {
+      __nv_bfloat162 m2 = absmax_u4(c1, absmax_u4(c0, as_bf2(0u)));
+#pragma unroll
+      for (int o = 4; o > 0; o >>= 1) m2 = __hmax2(m2, as_bf2(__shfl_xor_sync(0xFFFFFFFFu, bf2_bits(m2), o)));
+      const float amax = fmaxf(fmaxf(__low2float(m2), __high2float(m2)), kAmaxFloor);
+      s_bits = f32_to_bf16_bits(__fdiv_rn(amax, 6.0f));
+      const uint32_t s2 = s_bits * 0x00010001u;
+      out = make_uint2(fp4_word(c0, s2), fp4_word(c1, s2));
+    }
     *reinterpret_cast<uint2*>(packed + at) = out;
     if (pub_packed) *reinterpret_cast<uint2*>(pub_packed + at) = out;  // the rollout engine's copy (Sec. 3.1 item 3)
-  }
-  if (sub == 0) {
-    const int64_t idx = (e * kb + g) * N + n;
-    scales[idx] = static_cast<uint16_t>(s_bits);
-    if (FMT == 0) zeros[idx] = static_cast<uint8_t>(zf);
-    if (pub_packed) {
-      pub_scales[idx] = static_cast<uint16_t>(s_bits);
-      if (FMT == 0) pub_zeros[idx] = static_cast<uint8_t>(zf);
+    if (sub == 0) {
+      scales[idx] = static_cast<uint16_t>(s_bits);
+      if (FMT == 0) zeros[idx] = static_cast<uint8_t>(zf);
+      if (pub_packed) {
+        pub_scales[idx] = static_cast<uint16_t>(s_bits);
+        if (FMT == 0) pub_zeros[idx] = static_cast<uint8_t>(zf);
+      }
     }
   }
 }
@@ -336,13 +374,16 @@ cudaError_t launch_quantize_act(const Launch& L, const uint16_t* x, int64_t M, i
 cudaError_t launch_quantize_weight_w4(const Launch& L, int fmt, const uint16_t* w, int64_t E, int64_t N, int64_t K,
                                       uint8_t* packed, uint16_t* scales, uint8_t* zeros, uint8_t* pub_packed,
                                       uint16_t* pub_scales, uint8_t* pub_zeros) {
-  const int64_t groups = E * N * (K / kBlock);
-  if (groups == 0) return cudaSuccess;
-  const int64_t blocks = (groups * 8 + 255) / 256;
+  const int64_t row_blocks = E * N / 32, kb = K / kBlock;
+  if (row_blocks == 0 || kb == 0) return cudaSuccess;
+  // split the K-groups of a row block over several CTAs until the grid fills the device a few times over
+  const int64_t want = static_cast<int64_t>(L.sm_count) * 32;
+  const int64_t split = std::min<int64_t>(kb, std::max<int64_t>(1, (want + row_blocks - 1) / row_blocks));
+  const int per = static_cast<int>((kb + split - 1) / split);
+  const dim3 grid(static_cast<unsigned>(row_blocks), static_cast<unsigned>((kb + per - 1) / per));
   ++*L.launches;
-  return launch_pdl(fmt == kFmtE2m1 ? quantize_weight_w4_kernel<1> : quantize_weight_w4_kernel<0>,
-                    static_cast<unsigned>(blocks), 256, 0, L.stream, w, E * N, N, K, packed, scales, zeros, pub_packed,
-                    pub_scales, pub_zeros);
+  return launch_pdl(fmt == kFmtE2m1 ? quantize_weight_w4_kernel<1> : quantize_weight_w4_kernel<0>, grid, 256, 0,
+                    L.stream, w, N, K, per, packed, scales, zeros, pub_packed, pub_scales, pub_zeros);
 }
 
 cudaError_t launch_scatter_rows(const Launch& L, const uint16_t* x, int64_t M, int64_t H, uint16_t* out,
