@@ -172,6 +172,57 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
                  void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Expert-parallel form of qarl_moe_fwd: the layer cut into the three stages between which rows
+ * travel when the experts are split across GPUs (contiguous ranges of expert ids per GPU).
+ *   token's GPU : qarl_moe_dispatch      rows quantized once, laid out sorted by expert id
+ *   (exchange 1 : each GPU receives the rows of its experts, per source in expert order)
+ *   expert's GPU: qarl_moe_experts_fwd   gate_up, SwiGLU, re-quantization, down, * pair weight
+ *   (exchange 2 : the bf16 contributions travel back to where their rows came from)
+ *   token's GPU : qarl_moe_combine_sorted  the k-sum in ascending expert id
+ * The stages run the kernels of qarl_moe_fwd on the same per-row data, so by the row invariance
+ * (App. C) the output is bitwise that of qarl_moe_fwd with all experts on one GPU, for any
+ * number of GPUs and any split of the tokens.  The exchanges are the caller's (the Python
+ * package does them with all-to-all collectives); with one GPU the three calls in a row are the
+ * whole layer.  All pointers are device pointers; nothing is allocated.
+ * ------------------------------------------------------------------------------------- */
+
+/* in : x_bf16 [M, H], topk_ids [M, k] (global expert ids in [0, E)), topk_weights [M, k] fp32.
+ * out: codes_sorted u8 [M*k, H] and scales_sorted fp32 [M*k, H/128]: the quantized row of pair
+ *      p's token at position pos_of_pair[p]; weights_sorted fp32 [M*k]: the pair's top-k weight
+ *      at the same position; offsets i32 [E+1]: positions [offsets[e], offsets[e+1]) belong to
+ *      expert e (stable order of flat pair id inside); pos_of_pair i32 [M*k].
+ * workspace: qarl_moe_dispatch_workspace_bytes(M, E, k) bytes, 256-byte aligned.
+ * Limits: H % 128 == 0, 1 <= k <= 32, 1 <= E <= 1024, M*k < 2^31.  M == 0: offsets zeroed. */
+size_t qarl_moe_dispatch_workspace_bytes(int64_t M, int64_t E, int64_t k);
+int qarl_moe_dispatch(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
+                      const float* topk_weights, int64_t M, int64_t H, int64_t E, int64_t k,
+                      uint8_t* codes_sorted, float* scales_sorted, float* weights_sorted,
+                      int32_t* offsets, int32_t* pos_of_pair, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* in : R rows (codes u8 [R, H], scales fp32 [R, H/128], row_weights fp32 [R]) grouped by local
+ *      expert: rows [offsets[j], offsets[j+1]) use expert j of the E_local experts whose weights
+ *      are given (w13 [E_local, 2I, H], w2 [E_local, H, I], codes + block scales as
+ *      qarl_quantize_weight writes them); offsets i32 [E_local+1] on the device, offsets[E_local] == R.
+ * out: contrib bf16 [R, H]: row r = bf16(row_weights[r] * (h_r . W2_e)), in the order of the input.
+ * workspace: qarl_moe_experts_workspace_bytes(R, I) bytes, 256-byte aligned.
+ * Limits: H % 128 == 0, I % 128 == 0, 1 <= E_local <= 1024, R < 2^31. */
+size_t qarl_moe_experts_workspace_bytes(int64_t R, int64_t I);
+int qarl_moe_experts_fwd(qarl_ctx* ctx, const uint8_t* codes, const float* scales,
+                         const float* row_weights, const int32_t* offsets, int64_t R, int64_t H,
+                         int64_t I, int64_t E_local, const uint8_t* w13_codes,
+                         const float* w13_scales, const uint8_t* w2_codes, const float* w2_scales,
+                         void* contrib_bf16, void* workspace, size_t workspace_bytes, void* stream);
+
+/* out[t] = bf16(sum over the token's k pairs, in ascending expert id, of
+ * float(contrib_sorted[pos_of_pair[t*k + j]])), starting from 0.0f: the last step of
+ * qarl_moe_fwd on contributions held in dispatch order.  contrib_sorted bf16 [M*k, H];
+ * topk_ids and pos_of_pair as given to / written by qarl_moe_dispatch.  H % 8 == 0. */
+int qarl_moe_combine_sorted(qarl_ctx* ctx, const void* contrib_sorted_bf16, const int32_t* topk_ids,
+                            const int32_t* pos_of_pair, int64_t M, int64_t H, int64_t E, int64_t k,
+                            void* out_bf16, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * W4A16: 4-bit integer weight-only quantization with bf16 activations (Sec. 2.2, integer
  * quantization: W_q = clamp(round(W/s) + z, q_min, q_max), W^ = s (W_q - z); Sec. 3.1 item 1
  * names W4A16 as the format of the larger MoE models).  Choices the paper leaves open, fixed

@@ -33,6 +33,8 @@ EXPORTS = [
     "qarl_quantize_weight_w4", "qarl_linear_fwd_w4a16", "qarl_moe_w4a16_workspace_bytes",
     "qarl_moe_fwd_w4a16", "qarl_linear_bwd", "qarl_quantize_weight_publish",
     "qarl_tbpo_workspace_bytes", "qarl_tbpo_loss", "qarl_router_fwd", "qarl_grouped_linear_bwd", "qarl_moe_bwd_workspace_bytes", "qarl_moe_bwd",
+    "qarl_moe_dispatch_workspace_bytes", "qarl_moe_dispatch", "qarl_moe_experts_workspace_bytes",
+    "qarl_moe_experts_fwd", "qarl_moe_combine_sorted",
     "qarl_quantize_weight_w4_publish", "qarl_quantize_weight_fp4", "qarl_linear_fwd_fp4a16", "qarl_moe_fwd_fp4a16",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
@@ -126,6 +128,16 @@ def load() -> C.CDLL:
     L.qarl_moe_bwd_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
     L.qarl_moe_bwd.restype = C.c_int
     L.qarl_moe_bwd.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, p, p, p, p, p, p, p, sz, p]
+    L.qarl_moe_dispatch_workspace_bytes.restype = sz
+    L.qarl_moe_dispatch_workspace_bytes.argtypes = [i64, i64, i64]
+    L.qarl_moe_dispatch.restype = C.c_int
+    L.qarl_moe_dispatch.argtypes = [p, p, p, p, i64, i64, i64, i64, p, p, p, p, p, p, sz, p]
+    L.qarl_moe_experts_workspace_bytes.restype = sz
+    L.qarl_moe_experts_workspace_bytes.argtypes = [i64, i64]
+    L.qarl_moe_experts_fwd.restype = C.c_int
+    L.qarl_moe_experts_fwd.argtypes = [p, p, p, p, p, i64, i64, i64, i64, p, p, p, p, p, p, sz, p]
+    L.qarl_moe_combine_sorted.restype = C.c_int
+    L.qarl_moe_combine_sorted.argtypes = [p, p, p, p, i64, i64, i64, i64, p, p]
     L.qarl_quantize_weight_fp4.restype = C.c_int
     L.qarl_quantize_weight_fp4.argtypes = [p, p, i64, i64, i64, p, p, p, p, p]
     L.qarl_linear_fwd_fp4a16.restype = C.c_int
@@ -329,6 +341,52 @@ class Context:
                                           _ptr(y), _ptr(ws), ws.numel(),
                                           C.byref(dbg) if dbg is not None else None, _stream()))
         return (y, d) if debug else y
+
+    # ------------------------------------------------------------------ expert-parallel stages
+    def moe_dispatch(self, x, topk_ids, topk_weights, E: int):
+        """Quantize the tokens once and lay their (token, expert) rows out sorted by expert id ->
+        dict(codes [P, H] u8, scales [P, H/128] f32, weights [P] f32, offsets [E+1] i32, pos_of_pair [P] i32)."""
+        assert x.dtype == torch.bfloat16 and x.is_contiguous()
+        assert topk_ids.dtype == torch.int32 and topk_weights.dtype == torch.float32
+        M, H = x.shape
+        k = topk_ids.shape[1]
+        P, dev = M * k, x.device
+        d = dict(codes=torch.empty((P, H), dtype=torch.uint8, device=dev),
+                 scales=torch.empty((P, H // 128), dtype=torch.float32, device=dev),
+                 weights=torch.empty(P, dtype=torch.float32, device=dev),
+                 offsets=torch.empty(E + 1, dtype=torch.int32, device=dev),
+                 pos_of_pair=torch.empty(P, dtype=torch.int32, device=dev))
+        ws = self.workspace(int(self.lib.qarl_moe_dispatch_workspace_bytes(M, E, k)))
+        self._check(self.lib.qarl_moe_dispatch(self.h, _ptr(x), _ptr(topk_ids), _ptr(topk_weights), M, H, E, k,
+                                               _ptr(d["codes"]), _ptr(d["scales"]), _ptr(d["weights"]),
+                                               _ptr(d["offsets"]), _ptr(d["pos_of_pair"]), _ptr(ws), ws.numel(),
+                                               _stream()))
+        return d
+
+    def moe_experts_fwd(self, codes, scales, row_weights, offsets, w13_codes, w13_scales, w2_codes, w2_scales,
+                        out=None):
+        """gate_up, SwiGLU, down and the pair weight for rows grouped by local expert -> contrib bf16 [R, H]."""
+        R, H = codes.shape
+        E_local, I2, _ = w13_codes.shape
+        I = I2 // 2
+        assert offsets.dtype == torch.int32 and offsets.numel() == E_local + 1
+        assert codes.is_contiguous() and scales.is_contiguous() and row_weights.is_contiguous()
+        contrib = out if out is not None else torch.empty((R, H), dtype=torch.bfloat16, device=codes.device)
+        assert contrib.is_contiguous() and contrib.dtype == torch.bfloat16
+        ws = self.workspace(int(self.lib.qarl_moe_experts_workspace_bytes(R, I)))
+        self._check(self.lib.qarl_moe_experts_fwd(self.h, _ptr(codes), _ptr(scales), _ptr(row_weights), _ptr(offsets),
+                                                  R, H, I, E_local, _ptr(w13_codes), _ptr(w13_scales), _ptr(w2_codes),
+                                                  _ptr(w2_scales), _ptr(contrib), _ptr(ws), ws.numel(), _stream()))
+        return contrib
+
+    def moe_combine_sorted(self, contrib_sorted, topk_ids, pos_of_pair, E: int):
+        """The k-sum in ascending expert id over contributions held in dispatch order -> out bf16 [M, H]."""
+        M, k = topk_ids.shape
+        H = contrib_sorted.shape[1]
+        out = torch.empty((M, H), dtype=torch.bfloat16, device=contrib_sorted.device)
+        self._check(self.lib.qarl_moe_combine_sorted(self.h, _ptr(contrib_sorted), _ptr(topk_ids), _ptr(pos_of_pair),
+                                                     M, H, E, k, _ptr(out), _stream()))
+        return out
 
     # ------------------------------------------------------------------ W4A16
     def quantize_weight_w4(self, w: torch.Tensor, out=None):

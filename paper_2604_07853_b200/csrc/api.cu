@@ -15,17 +15,6 @@ namespace {
 
 using namespace qarl;
 
-int run_gemm(qarl_ctx* ctx, const Launch& L, const GemmArgs& a) {
-  CUresult cu = CUDA_SUCCESS;
-  cudaError_t e = launch_gemm(L, ctx->encode, a, &cu);
-  if (cu != CUDA_SUCCESS) {
-    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
-    return QARL_ERR_CUDA;
-  }
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "gemm launch");
-  return QARL_OK;
-}
-
 // Workspace carve-up of qarl_moe_fwd; every slice starts on a 256-byte boundary.
 struct MoePlan {
   size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, a_codes, a_scales, h_codes, h_scales, contrib, total;

@@ -31,4 +31,16 @@ inline void mark(qarl_ctx* ctx, cudaStream_t st, int stage) {
   ctx->mark_stage[ctx->marks_used++] = stage;
 }
 
+// The block-scaled FP8 GEMM with its error reporting.
+inline int run_gemm(qarl_ctx* ctx, const Launch& L, const GemmArgs& a) {
+  CUresult cu = CUDA_SUCCESS;
+  cudaError_t e = launch_gemm(L, ctx->encode, a, &cu);
+  if (cu != CUDA_SUCCESS) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+    return QARL_ERR_CUDA;
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "gemm launch");
+  return QARL_OK;
+}
+
 }  // namespace qarl

@@ -102,8 +102,9 @@ int64_t permute_num_chunks(int64_t P);
 cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
                            const PermuteBuffers& b);
 
+// pos_of_pair == nullptr: contrib is indexed by flat pair id; else by pos_of_pair[pair] (sorted order)
 cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
-                           int64_t H, int64_t E, uint16_t* out);
+                           int64_t H, int64_t E, uint16_t* out, const int32_t* pos_of_pair = nullptr);
 
 cudaError_t launch_wait_selftest(const Launch& L, unsigned long long limit_ns);
 cudaError_t launch_rmsnorm(const Launch& L, const uint16_t* x, int64_t M, int64_t H, float eps, uint16_t* out);

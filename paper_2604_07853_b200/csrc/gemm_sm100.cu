@@ -369,7 +369,9 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       int my_pair = 0;  // down: destination (flat pair id) of the lane-th row this warp handles
       if (MODE == kModeDown) {
         const int row = c.m0 + ew + kEpiWarps * lane;
-        if (row < c.m_end) my_pair = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
+        // no pair map: the contribution stays at its sorted position (expert-parallel use)
+        if (row < c.m_end)
+          my_pair = p.sorted_pair ? min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1) : row;  // in bounds even after bad ids
       }
       {
         TRACE_T0();
