@@ -195,6 +195,10 @@ def main():
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-w4a16", action="store_true")
+    ap.add_argument("--no-ep", action="store_true", help="skip the expert-parallel form of the layer")
+    ap.add_argument("--ep", action="store_true",
+                    help="with --gpus N > 1: split the experts across the ranks (two NCCL all-to-alls per layer) "
+                         "in the expert_parallel section instead of running it as one rank per GPU")
     ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--no-tbpo", action="store_true")
     ap.add_argument("--no-router", action="store_true")
@@ -429,6 +433,43 @@ def main():
             "frac_hbm_measured": rbytes / (r_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
         }
         del wr
+
+    # ---------------- expert-parallel form of the layer: dispatch / experts / combine as separate calls, the
+    # rows exchanged between them (nothing to exchange with one rank; --ep splits the experts over the ranks)
+    if not args.no_ep:
+        from paper_2604_07853_b200.expert_parallel import CudaStages, ExpertParallelMoE, expert_range, run_local
+        ep_world = world if (args.ep and world > 1) else 1
+        ep_rank = rank if ep_world > 1 else 0
+        lo, hi = expert_range(ep_rank, ep_world, E)
+        ep = ExpertParallelMoE(CudaStages(ctx, (w13c[lo:hi], w13s[lo:hi]), (w2c[lo:hi], w2s[lo:hi]), E),
+                               ep_rank, ep_world, E)
+
+        def ep_fwd():
+            return ep.forward(x, ids, wts) if ep_world > 1 else run_local([ep], [(x, ids, wts)])[0]
+
+        same = None
+        if ep_world == 1:
+            ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, workspace=ws)
+            same = bool(torch.equal(ep_fwd(), out))
+        esteps = max(args.steps // 4, 10)
+        for _ in range(3):
+            ep_fwd()
+        barrier()
+        ev0.record()
+        for _ in range(esteps):
+            ep_fwd()
+        ev1.record()
+        barrier()
+        ep_ms = max_over_ranks(ev0.elapsed_time(ev1)) / esteps
+        ctx.check_device_status()
+        result["expert_parallel"] = {
+            "workload": f"moe_ffn_train_M{M_TRAIN} layer forward as dispatch / experts / combine stages, "
+                        f"{ep_world} expert-parallel rank(s)"
+                        + (" with NCCL all-to-all exchanges" if ep_world > 1 else " (no exchange; one host sync per layer for the row counts)"),
+            "ms_per_layer": ep_ms, "tokens_per_s": world * M_TRAIN / (ep_ms * 1e-3),
+            "bytewise_equal_to_fused_layer": same,
+        }
+        del ep
 
     # ---------------- 4-bit weight-only variants of the same layer (bf16 activations): integer codes with a
     # zero point ("w4a16") and e2m1 floating point ("fp4a16"); same storage, same kernels

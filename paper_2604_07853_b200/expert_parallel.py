@@ -145,7 +145,7 @@ def run_local(ranks: list[ExpertParallelMoE], inputs: list[tuple]) -> list[torch
     contribs = []
     for r, (ep, st) in enumerate(zip(ranks, sts)):
         st.counts_in = torch.stack([sts[s].counts_out[r] for s in range(world)])
-        got = [torch.cat([sts[s].send[i][bounds[s][r]] for s in range(world)]) for i in range(3)]
+        got = [_cat([sts[s].send[i][bounds[s][r]] for s in range(world)]) for i in range(3)]
         contribs.append(ep.middle(st, *got))
     outs = []
     for r, (ep, st) in enumerate(zip(ranks, sts)):
@@ -153,5 +153,9 @@ def run_local(ranks: list[ExpertParallelMoE], inputs: list[tuple]) -> list[torch
         for g in range(world):                    # what rank g computed for the rows that came from rank r
             edges = [0] + torch.cumsum(sts[g].counts_in.sum(1), 0).tolist()
             pieces.append(contribs[g][edges[r]:edges[r + 1]])
-        outs.append(ep.finish(st, torch.cat(pieces)))
+        outs.append(ep.finish(st, _cat(pieces)))
     return outs
+
+
+def _cat(pieces: list[torch.Tensor]) -> torch.Tensor:
+    return pieces[0] if len(pieces) == 1 else torch.cat(pieces)

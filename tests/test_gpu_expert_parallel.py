@@ -98,6 +98,29 @@ def test_decode_layer_shape_on_four_ranks(ctx):
     run_ranks(ctx, case, 4, even_split(case.x.shape[0], 4))
 
 
+def test_forward_over_a_one_rank_nccl_group(ctx):
+    """The per-process driver with its real collectives (all_to_all_single on device tensors); one rank is
+    all this machine has, so the exchanges are self-sends, but counts, splits and buffers take the NCCL path."""
+    import socket
+    import torch.distributed as dist
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        case = inputs.moe_case(42, 300, h=256, i=128, e=8, k=2, zipf_s=1.1)
+        x, ids, wts, w13, w2 = device_case(ctx, case)
+        ref = ctx.moe_fwd(x, ids, wts, *w13, *w2).clone()
+        ep = ExpertParallelMoE(CudaStages(ctx, w13, w2, case.E), 0, 1, case.E)
+        out = ep.forward(x, ids, wts)
+        assert ctx.poll() == 0
+        assert torch.equal(out, ref)
+    finally:
+        dist.destroy_process_group()
+
+
 def test_stage_argument_checks(ctx):
     dev = torch.device("cuda", 0)
     x = torch.zeros((4, 192), dtype=torch.bfloat16, device=dev)        # H not a multiple of 128
