@@ -595,11 +595,17 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             acc_hi[j] = __fmul2_rn(w2, acc_hi[j]);
           }
         }
+#ifdef QARL_TRACE
+        trace_acc[9] += clock64() - _tend0;
+#endif
         {
           TRACE_T0();
           if (!wait_or_abort(&s->out_empty, (tile_iter & 1u) ^ 1u, s, p)) break;  // previous tile drained
           TRACE_ADD(4);
         }
+#ifdef QARL_TRACE
+        const long long _tst0 = clock64();
+#endif
         if (warp_live) {
           uint4* d_lo = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + hs * (kSliceCols * 2));
           uint4* d_hi = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + BNH * 2 + hs * (kSliceCols * 2));
@@ -615,6 +621,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         if (lane == 0) mbar_arrive(&s->out_full);
 #ifdef QARL_TRACE
         trace_acc[8] += clock64() - _tend0;
+        trace_acc[10] += clock64() - _tst0;
 #endif
         if (!has_next) break;
         T = Tn;
