@@ -321,13 +321,13 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   d.offsets = pb.offsets;
   d.out_bf16 = contrib;
   d.out_f32 = dbg ? dbg->down_f32 : nullptr;
-  d.sorted_pair = pb.sorted_pair;
+  d.sorted_pair = nullptr;  // contributions stay in sorted order (dense row blocks); the k-sum finds them by position
   d.pair_weights = sorted_w;
   rc = run_gemm(ctx, L, d);
   if (rc != QARL_OK) return rc;
   mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);
 
-  if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out))) != cudaSuccess)
+  if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out), pb.pos_of_pair)) != cudaSuccess)
     return cuda_fail(ctx, e, "combine");
   mark(ctx, L.stream, QARL_STAGE_COMBINE);
 

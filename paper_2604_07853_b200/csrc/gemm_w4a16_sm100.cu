@@ -417,7 +417,8 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
       int64_t out_row = row;
       if (MODE == kModeDown && valid) {
         w = __ldg(p.pair_weights + row);
-        out_row = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
+        // no pair map: the contribution stays at its sorted position
+        if (p.sorted_pair) out_row = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
       }
       if (mt == 0) {
         if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) { ok = false; break; }
