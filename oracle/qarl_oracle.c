@@ -430,7 +430,8 @@ int oracle_moe(const uint16_t *x, const int32_t *ids, const float *wts,
  * the paper's headline results use (Sec. 3.1 item 1: W4A16 for larger MoE models).
  *   Quant:   W_q = clamp( round(W / s) + z, q_min, q_max ),   Dequant:  W^ = s (W_q - z)
  * Readings where the paper is silent: unsigned 4-bit codes (q_min = 0, q_max = 15); one
- * (s, z) per group of 128 consecutive K elements of one weight row; asymmetric min/max
+ * (s, z) per group of 128 consecutive K elements of one weight row (the group size is not in the
+ * paper: "parity unpinned" on this point, for this format and the FP4 one below); asymmetric min/max
  * calibration with zero kept representable: lo = min(0, min W), hi = max(0, max W),
  * s = bf16( fl(max(hi - lo, 2^-40) / 15) ) -- the group scale is kept in the model's 16-bit type,
  * as W4A16 checkpoints store it, and is returned here as the fp32 of that bf16 value --
