@@ -12,6 +12,9 @@
  * contributions are added (oracle_linear_q's kb-ascending chain, oracle_combine's
  * ascending-expert chain) is "parity unpinned" by the paper -- App. C only requires that
  * some fixed order be used.  The order chosen here is stated beside each function.
+ * Likewise "parity unpinned" by the paper, each stated beside its function: the group size of
+ * the two 4-bit weight formats (128 along K), and the router's top-k softmax rule (the paper
+ * names a router but gives no formula); what follows from those choices is pinned as above.
  *
  * Build: gcc -O2 -fopenmp -ffp-contract=off -fno-fast-math -shared -fPIC (see oracle/build.py).
  * OpenMP is used over independent rows / experts only, never inside a reduction whose
