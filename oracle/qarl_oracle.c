@@ -736,7 +736,8 @@ void oracle_tbpo(const float *lp_cur, const float *lp_old_learner, const float *
  * operands (exact sum, rounded once to fp32); the k largest logits of a token, ties to the lower
  * expert id, in descending order; weights = softmax over the k selected fp32 logits (exp of
  * logit - max in double, normalised, rounded to fp32).  The router stays in bf16: it is not
- * quantized.
+ * quantized.  The rule itself is "parity unpinned" (nothing in the paper fixes it); the tests pin what
+ * the rule implies (sorted selection, ties, weights summing to one, the softmax closed form).
  * ===================================================================================== */
 void oracle_router_topk(const float *logits, int64_t M, int64_t E, int64_t k, int32_t *ids, float *wts) {
 #pragma omp parallel for schedule(static)
