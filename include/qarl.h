@@ -25,7 +25,10 @@
  *     outside [0, E), an expert repeated within one token, a bounded wait that expired) set
  *     the context's device status word; the outputs of that call are unspecified and the
  *     error is reported by qarl_poll_device_status.
- *   - A context belongs to one device and may be used from one host thread at a time.
+ *   - A context belongs to one device and may be used from one host thread at a time.  Several
+ *     contexts (on the same or on different devices) may be used from several host threads at
+ *     once: the little process-wide state the library keeps (per-device launch attributes, the
+ *     address of the static scratch array) is written atomically and idempotently.
  *   - There is no CPU fallback: without an sm_100 device qarl_create fails.
  */
 #ifndef QARL_H_

@@ -28,6 +28,25 @@ int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H
  * qarl_poll_device_status reports (and clears) the error.  Nothing traps, faults or hangs. */
 int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream);
 
+/* The two calls below exist so that a test can watch the FP8 GEMM's own pipeline give up on a wait
+ * (the library never needs them).  Both only store a value in the context (host side, not
+ * synchronized with calls running on other threads); it applies to the GEMM kernels launched
+ * through `ctx` afterwards.
+ *
+ * qarl_harness_set_wait_limit_ns: the bound, in nanoseconds, of every barrier wait inside those
+ * kernels (0 restores the default of 2 s; other values are clamped to [1 us, 2 s]).
+ *
+ * qarl_harness_stop_producer_after: the TMA producer of every CTA stops arming shared-memory
+ * stages after `stages` of them (a negative value restores normal operation).  It waits for its
+ * copies in flight and leaves its loop; nothing else is told.  The MMA role then waits on a stage
+ * that nothing fills: its bounded wait runs out, it records QARL_ERR_DEVICE_TIMEOUT and raises the
+ * CTA's abort flag; every other role leaves its loop at its next wait; the MMA role waits
+ * (bounded) for the MMAs it had issued; TMEM is freed and the kernel returns.  Outputs of such a
+ * call are unspecified; the context stays usable and qarl_poll_device_status reports the error.
+ * Nothing traps, faults or spins without a bound. */
+int qarl_harness_set_wait_limit_ns(qarl_ctx* ctx, uint64_t limit_ns);
+int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,7 +38,8 @@ EXPORTS = [
     "qarl_quantize_weight_w4_publish", "qarl_quantize_weight_fp4", "qarl_linear_fwd_fp4a16", "qarl_moe_fwd_fp4a16",
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
-HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest"]
+HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest", "qarl_harness_set_wait_limit_ns",
+                   "qarl_harness_stop_producer_after"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise"]
 
@@ -154,6 +155,10 @@ def load() -> C.CDLL:
     L.qarl_harness_rmsnorm.argtypes = [p, p, i64, i64, C.c_float, p, p]
     L.qarl_harness_wait_selftest.restype = C.c_int
     L.qarl_harness_wait_selftest.argtypes = [p, C.c_uint64, p]
+    L.qarl_harness_set_wait_limit_ns.restype = C.c_int
+    L.qarl_harness_set_wait_limit_ns.argtypes = [p, C.c_uint64]
+    L.qarl_harness_stop_producer_after.restype = C.c_int
+    L.qarl_harness_stop_producer_after.argtypes = [p, i64]
     _lib = L
     return L
 
@@ -232,6 +237,14 @@ class Context:
     def harness_wait_selftest(self, limit_ns: int = 1_000_000):
         """Launch the bounded-wait self test (a wait nothing satisfies); poll() then returns -7."""
         self._check(self.lib.qarl_harness_wait_selftest(self.h, limit_ns, _stream()))
+
+    def harness_set_wait_limit_ns(self, limit_ns: int):
+        """Bound of every barrier wait in the GEMM kernels launched from now on (0: default)."""
+        self._check(self.lib.qarl_harness_set_wait_limit_ns(self.h, limit_ns))
+
+    def harness_stop_producer_after(self, stages: int):
+        """FP8 GEMM TMA producers stop arming stages after `stages` (negative: normal operation)."""
+        self._check(self.lib.qarl_harness_stop_producer_after(self.h, stages))
 
     def harness_rmsnorm(self, x: torch.Tensor, eps: float = 1e-6, out=None):
         """Row-invariant RMSNorm (weight 1) used by the alignment-stack test; not part of the API."""

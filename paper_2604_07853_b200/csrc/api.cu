@@ -361,6 +361,19 @@ int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, flo
   return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "rmsnorm");
 }
 
+int qarl_harness_set_wait_limit_ns(qarl_ctx* ctx, uint64_t limit_ns) {
+  if (!ctx) return QARL_ERR_INVALID_ARG;
+  if (limit_ns != 0) limit_ns = limit_ns < 1000 ? 1000 : (limit_ns > 2000000000ull ? 2000000000ull : limit_ns);
+  ctx->wait_limit_ns = limit_ns;
+  return QARL_OK;
+}
+
+int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages) {
+  if (!ctx) return QARL_ERR_INVALID_ARG;
+  ctx->stop_after_stages = stages < 0 ? -1 : static_cast<int>(stages > 0x7FFFFFFF ? 0x7FFFFFFF : stages);
+  return QARL_OK;
+}
+
 int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream) {
   if (!ctx) return QARL_ERR_INVALID_ARG;
   if (limit_ns < 1000) limit_ns = 1000;

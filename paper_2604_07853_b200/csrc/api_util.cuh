@@ -21,6 +21,8 @@ inline Launch make_launch(qarl_ctx* ctx, void* stream) {
   L.sm_count = ctx->sm_count;
   L.d_status = ctx->d_status;
   L.launches = &ctx->launches;
+  L.wait_limit_ns = ctx->wait_limit_ns;
+  L.stop_after_stages = ctx->stop_after_stages;
   return L;
 }
 

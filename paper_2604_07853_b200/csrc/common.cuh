@@ -61,6 +61,8 @@ struct Launch {
   int sm_count;
   int* d_status;
   int64_t* launches;  // host counter
+  unsigned long long wait_limit_ns = 0;  // bound of every device-side barrier wait (0: the default, 2 s)
+  int stop_after_stages = -1;            // test harness only: FP8 GEMM producers stop after this many stages
 };
 
 // Launch with the programmatic-stream-serialization attribute (see pdl_wait above).
@@ -233,6 +235,8 @@ struct qarl_ctx {
   int sm_count;
   int* d_status;
   int64_t launches;
+  unsigned long long wait_limit_ns = 0;  // 0: default; set only by the test harness
+  int stop_after_stages = -1;            // -1: off; set only by the test harness
   qarl::EncodeTiledFn encode;
   char err[256];
   // stage timing: marks[i] closes stage mark_stage[i] (-1: an opening mark)

@@ -30,6 +30,7 @@
 // order of accumulation: a result does not depend on the grid or on the other rows.
 // Every wait is bounded (status word + CTA-wide abort flag), as in the other GEMMs.
 #include <algorithm>
+#include <atomic>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -84,6 +85,7 @@ struct __align__(8) SmemTail {
   uint64_t empty[kMaxStages];
   uint64_t tmem_full[kMaxAccBufs];
   uint64_t tmem_empty[kMaxAccBufs];
+  uint64_t teardown;
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
@@ -107,6 +109,13 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sm
       return false;
     }
   }
+}
+
+// The same for a whole warp: every lane polls, then the lanes vote, so all 32 take the same
+// branch and the warp-wide operations that follow never see a split warp (lanes polling on
+// their own could disagree when a barrier completes right at the limit).
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const Bf16Params& p) {
+  return __all_sync(0xFFFFFFFFu, wait_or_abort(bar, parity, s, p) ? 1 : 0) != 0;
 }
 
 __device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
@@ -136,6 +145,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       mbar_init(&s->tmem_full[i], 1);
       mbar_init(&s->tmem_empty[i], kEpiWarps);
     }
+    mbar_init(&s->teardown, 1);
     s->abort_flag = 0;
     fence_mbar_init();
   }
@@ -258,10 +268,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
       const Tile t = tile_of(T, cur_e);
       if (t.KS == 0) continue;  // an expert without rows: the epilogue writes zeros, no accumulator is used
-      if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
+      if (!warp_wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) { ok = false; break; }
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * MT) * BN;
       for (int ks = 0; ks < t.KS; ++ks) {
-        if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
+        if (!warp_wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
         uint8_t* a_tile = smem + static_cast<size_t>(stage) * kStageBytes;
         if (GROUP == kGroupedContraction && ks == t.KS - 1 && t.last_valid < BK) {
           // rows last_valid .. 63 of both 64-column blocks of A belong to the next expert: make them zero
@@ -298,6 +308,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       }
       if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
     }
+    // Nothing of this CTA's tensor work may be in flight when its TMEM and shared memory go
+    // away: after an abort some MMAs may still be executing, so wait (bounded) for them.
+    if (!ok && lane == 0) {
+      umma_commit(&s->teardown);
+      mbar_wait_bounded(&s->teardown, 0, 20000000ull);
+    }
   } else if (warp < kEpiWarps) {
     const int r = warp * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
@@ -309,7 +325,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int j0 = t.j0;
       const bool have_acc = t.KS > 0;
       if (have_acc) {
-        if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
+        if (!warp_wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) break;
         tc_fence_after_sync();
       }
 #pragma unroll 1
@@ -403,13 +419,15 @@ CUresult make_tmap_mn3d(EncodeTiledFn encode, CUtensorMap* m, const void* base, 
 template <bool A_MN, bool B_MN, int GROUP, int MT>
 cudaError_t launch_variant(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const Bf16Params& p,
                            int64_t tiles) {
-  static bool attr_set_dev[64] = {};
-  bool& attr_set = attr_set_dev[L.device & 63];
-  if (!attr_set) {
+  // sticky per function and device; atomic: contexts on several host threads may launch at once (both
+  // would set the same value)
+  static std::atomic<bool> attr_set_dev[64];
+  std::atomic<bool>& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set.load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<A_MN, B_MN, GROUP, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem_bytes<MT>()));
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set.store(true, std::memory_order_release);
   }
   // full rounds only: with W = ceil(tiles / SMs) rounds, ceil(tiles / W) CTAs finish in W rounds
   // (for grouped rows `tiles` is an upper bound: the surplus CTAs find no tile and retire)

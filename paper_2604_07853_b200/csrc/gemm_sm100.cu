@@ -32,6 +32,7 @@
 // QARL_ERR_DEVICE_TIMEOUT, raises a CTA-wide abort flag that all other waits poll, and the
 // CTA drains and frees its TMEM, so a broken pipeline returns an error instead of hanging.
 #include <algorithm>
+#include <atomic>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -45,14 +46,8 @@ constexpr int BM = 128;           // rows per tile (UMMA M)
 constexpr int BNH = 128;          // columns per half tile
 constexpr int BN = 2 * BNH;       // UMMA N
 constexpr int BK = 128;           // one K-block = one 128-byte swizzle span of e4m3
-#ifndef QARL_FP8_STAGES
-#define QARL_FP8_STAGES 3
-#endif
-constexpr int kStages = QARL_FP8_STAGES;
-#ifndef QARL_FP8_ACCBUFS
-#define QARL_FP8_ACCBUFS 2
-#endif
-constexpr int kAccBufs = QARL_FP8_ACCBUFS;       // TMEM accumulators of 256 columns
+constexpr int kStages = 3;        // shared-memory ring of 48 KB stages
+constexpr int kAccBufs = 2;       // TMEM accumulators of 256 columns
 constexpr int kPromoWarps = 8;    // warps 0-7
 constexpr int kEpiWarps = 4;      // warps 8-11
 constexpr int kTmaWarp = 12;
@@ -91,7 +86,7 @@ struct GemmParams {
   const float* pair_weights;  // down: combine weight of each sorted position
   int* status;
   unsigned long long wait_limit_ns;
-  unsigned long long* trace;  // QARL_TRACE builds only: per-CTA wait-cycle counters [grid][8]
+  int stop_after_stages;   // test harness only (< 0: off): the TMA producer stops arming stages after this many
 };
 
 struct __align__(8) SmemTail {
@@ -101,6 +96,7 @@ struct __align__(8) SmemTail {
   uint64_t tmem_empty[kAccBufs];
   uint64_t out_full;
   uint64_t out_empty;
+  uint64_t teardown;
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
@@ -129,6 +125,8 @@ __device__ __forceinline__ TileCoord decode_tile(const SmemTail* s, int T, int& 
   return c;
 }
 
+// Bounded wait of one thread.  False: the limit ran out here (the error is recorded and the
+// CTA-wide abort flag raised) or another thread raised the flag; the caller leaves its loop.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const GemmParams& p) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
@@ -145,15 +143,13 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sm
   }
 }
 
-// Wait-time tracing (development aid, compiled out unless QARL_TRACE is defined): cycles each
-// role spends blocked on each barrier, summed per CTA.
-#ifdef QARL_TRACE
-#define TRACE_T0() const long long _t0 = clock64()
-#define TRACE_ADD(slot) trace_acc[slot] += clock64() - _t0
-#else
-#define TRACE_T0()
-#define TRACE_ADD(slot)
-#endif
+// The same for a whole warp: every lane polls (one polling lane with 31 parked at a shuffle
+// measured 2x slower on the short-K down projection), then the lanes vote, so all 32 take the
+// same branch and the warp-wide shuffles and barriers that follow never see a split warp
+// (lanes polling on their own could disagree when a barrier completes right at the limit).
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const GemmParams& p) {
+  return __all_sync(0xFFFFFFFFu, wait_or_abort(bar, parity, s, p) ? 1 : 0) != 0;
+}
 
 // silu(g) * u in fp32 with the fast exp and reciprocal (relative error ~1e-6, far below the
 // half-ulp of the bf16 the result is rounded to).
@@ -184,10 +180,6 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   uint8_t* out_tile = smem + static_cast<size_t>(kStages) * kStageBytes;
   SmemTail* s = reinterpret_cast<SmemTail*>(out_tile + kOutBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef QARL_TRACE
-  long long trace_acc[12] = {0};
-  const long long trace_start = clock64();
-#endif
 
   // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
   pdl_trigger();
@@ -202,6 +194,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     }
     mbar_init(&s->out_full, kPromoWarps);
     mbar_init(&s->out_empty, kEpiWarps);
+    mbar_init(&s->teardown, 1);
     s->abort_flag = 0;
     fence_mbar_init();
   }
@@ -238,15 +231,28 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     }
   }
   pdl_wait();  // everything above read no data of the predecessor; from here on its results are needed
-  for (int e = threadIdx.x; e <= p.E; e += kThreads)
-    s->off[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.rows_total);
+  // Group boundaries, forced into [0, rows_total]: whatever the caller's array holds, no tile
+  // and no store mask derived from it can reach outside the tensors.
+  for (int e = threadIdx.x; e <= p.E; e += kThreads) {
+    const int raw = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.rows_total);
+    const int v = min(max(raw, 0), p.rows_total);
+    if (v != raw) set_status(p.status, QARL_ERR_INVALID_ARG);
+    s->off[e] = v;
+  }
   __syncthreads();
-  if (warp == 0) {  // exclusive scan of tiles per expert
+  if (warp == 0) {
+    // exclusive scan of tiles per expert
     int carry = 0;
     for (int base = 0; base < p.E; base += 32) {
       const int e = base + lane;
       int v = 0;
-      if (e < p.E) v = ((s->off[e + 1] - s->off[e] + BM - 1) / BM) * p.n_tiles;
+      if (e < p.E) {
+        // a group that ends before it starts (offsets out of order) is reported and gets no tile;
+        // with every boundary inside [0, rows_total] the other groups stay inside the tensors
+        const int rows = s->off[e + 1] - s->off[e];
+        if (rows < 0) set_status(p.status, QARL_ERR_INVALID_ARG);
+        v = ((max(rows, 0) + BM - 1) / BM) * p.n_tiles;
+      }
       int inc = v;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -286,6 +292,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         int stage = 0;
         uint32_t phase = 0;
         uint32_t armed = 0, armed_parity = 0;  // per-stage: has a load in flight / its parity
+        int armed_total = 0;
         int cur_e = 0;
         bool ok = true;
         // weight rows of a tile's two halves
@@ -303,11 +310,9 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           int row_lo, row_hi;
           b_rows(c, row_lo, row_hi);
           for (int kb = 0; kb < KB; ++kb) {
-            {
-              TRACE_T0();
-              if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
-              TRACE_ADD(0);
-            }
+            if (p.stop_after_stages >= 0 && armed_total >= p.stop_after_stages) { ok = false; break; }
+            ++armed_total;
+            if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
             uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
             uint8_t* b_dst = a_dst + kABytes;
             mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
@@ -333,16 +338,8 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         bool ok = true;
         for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
           for (int kb = 0; kb < KB; ++kb) {
-            {
-              TRACE_T0();
-              if (!wait_or_abort(&s->tmem_empty[ks], acc_phase ^ 1, s, p)) { ok = false; break; }
-              TRACE_ADD(2);
-            }
-            {
-              TRACE_T0();
-              if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
-              TRACE_ADD(1);
-            }
+            if (!wait_or_abort(&s->tmem_empty[ks], acc_phase ^ 1, s, p)) { ok = false; break; }
+            if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
             const uint64_t a_desc = umma_desc_k_sw128(a_addr);
@@ -356,6 +353,13 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             if (++stage == kStages) { stage = 0; phase ^= 1; }
             if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
           }
+        }
+        // Nothing of this CTA's tensor work may be in flight when its TMEM and shared memory
+        // go away: after a normal run every MMA has been consumed already; after an abort
+        // some may still be executing, so wait (bounded) for all of them.
+        if (!ok) {
+          umma_commit(&s->teardown);
+          mbar_wait_bounded(&s->teardown, 0, 20000000ull);
         }
       }
     }
@@ -373,11 +377,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         if (row < c.m_end)
           my_pair = p.sorted_pair ? min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1) : row;  // in bounds even after bad ids
       }
-      {
-        TRACE_T0();
-        if (!wait_or_abort(&s->out_full, tile_iter & 1u, s, p)) break;
-        TRACE_ADD(6);
-      }
+      if (!warp_wait_or_abort(&s->out_full, tile_iter & 1u, s, p)) break;
       if (MODE == kModeGateUp) {
         // 8 lanes per row, 4 rows per pass.  Lane `sub` owns h columns [8 sub, 8 sub + 8) and
         // [64 + 8 sub, 64 + 8 sub + 8) of the row's 128-wide quantization group, so that a
@@ -527,11 +527,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             swl_next = __ldg(sw_lo_ptr);
             swh_next = __ldg(sw_lo_ptr + sw_hi_off);
           }
-          {
-            TRACE_T0();
-            if (!wait_or_abort(&s->tmem_full[ks], acc_phase, s, p)) { ok = false; break; }
-            TRACE_ADD(3);
-          }
+          if (!warp_wait_or_abort(&s->tmem_full[ks], acc_phase, s, p)) { ok = false; break; }
           tc_fence_after_sync();
           if (!warp_live) {
             tc_fence_before_sync();
@@ -571,9 +567,6 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
         }
         if (!ok) break;
-#ifdef QARL_TRACE
-        const long long _tend0 = clock64();
-#endif
 
         // ---- hand the tile to the epilogue warps as bf16 -----------------------------------
         if ((MODE == kModeLinear || MODE == kModeDown) && p.out_f32 && valid) {  // debug fp32 dump
@@ -595,17 +588,7 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             acc_hi[j] = __fmul2_rn(w2, acc_hi[j]);
           }
         }
-#ifdef QARL_TRACE
-        trace_acc[9] += clock64() - _tend0;
-#endif
-        {
-          TRACE_T0();
-          if (!wait_or_abort(&s->out_empty, (tile_iter & 1u) ^ 1u, s, p)) break;  // previous tile drained
-          TRACE_ADD(4);
-        }
-#ifdef QARL_TRACE
-        const long long _tst0 = clock64();
-#endif
+        if (!warp_wait_or_abort(&s->out_empty, (tile_iter & 1u) ^ 1u, s, p)) break;  // previous tile drained
         if (warp_live) {
           uint4* d_lo = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + hs * (kSliceCols * 2));
           uint4* d_hi = reinterpret_cast<uint4*>(out_tile + r * kOutPitch + BNH * 2 + hs * (kSliceCols * 2));
@@ -619,10 +602,6 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&s->out_full);
-#ifdef QARL_TRACE
-        trace_acc[8] += clock64() - _tend0;
-        trace_acc[10] += clock64() - _tst0;
-#endif
         if (!has_next) break;
         T = Tn;
         c = cn;
@@ -631,15 +610,6 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     }
   }
 
-#ifdef QARL_TRACE
-  if (p.trace && lane == 0 && (warp == kTmaWarp || warp == kMmaWarp || warp == 0 || warp == kPromoWarps)) {
-    unsigned long long* t = p.trace + static_cast<size_t>(blockIdx.x) * 16;
-    if (warp == kTmaWarp) t[0] = trace_acc[0];
-    if (warp == kMmaWarp) { t[1] = trace_acc[1]; t[2] = trace_acc[2]; }
-    if (warp == 0) { t[3] = trace_acc[3]; t[4] = trace_acc[4]; t[5] = clock64() - trace_start; t[8] = trace_acc[8]; t[9] = trace_acc[9]; t[10] = trace_acc[10]; }
-    if (warp == kPromoWarps) { t[6] = trace_acc[6]; t[7] = clock64() - trace_start; }
-  }
-#endif
   // ---- teardown ---------------------------------------------------------------------------
   tc_fence_before_sync();
   __syncthreads();
@@ -651,11 +621,6 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
 
 }  // namespace
 
-#ifdef QARL_TRACE
-static unsigned long long* g_trace = nullptr;
-static unsigned g_trace_launch = 0;
-extern "C" void qarl_trace_set(unsigned long long* dev_ptr) { g_trace = dev_ptr; }
-#endif
 
 namespace {
 
@@ -673,13 +638,15 @@ CUresult make_tmap(EncodeTiledFn encode, CUtensorMap* m, const void* base, uint6
 template <int MODE>
 cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p,
                         int grid) {
-  static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
-  bool& attr_set = attr_set_dev[L.device & 63];
-  if (!attr_set) {
+  // sticky per function and device; atomic: contexts on several host threads may launch at once (both
+  // would set the same value)
+  static std::atomic<bool> attr_set_dev[64];
+  std::atomic<bool>& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set.load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_blockscaled_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kSmemBytes));
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set.store(true, std::memory_order_release);
   }
   ++*L.launches;
   return launch_pdl(gemm_blockscaled_kernel<MODE>, static_cast<unsigned>(grid), kThreads, kSmemBytes, L.stream, ta, tb, p);
@@ -716,16 +683,14 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
   p.sorted_pair = a.sorted_pair;
   p.pair_weights = a.pair_weights;
   p.status = L.d_status;
-  p.wait_limit_ns = 2000000000ull;
+  p.wait_limit_ns = L.wait_limit_ns ? L.wait_limit_ns : 2000000000ull;
+  p.stop_after_stages = L.stop_after_stages;
   // decode-sized call (at most one row tile per expert): see the early prefetch in the kernel
   if (a.rows_total <= a.E * BM) {
     const int64_t tile_bytes = static_cast<int64_t>(p.kblocks) * kBBytes;
     const int64_t budget = 80ll << 20;  // stay well inside the 126 MB L2
     p.early_prefetch = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(3, budget / (tile_bytes * L.sm_count))));
   }
-#ifdef QARL_TRACE
-  p.trace = g_trace ? g_trace + static_cast<size_t>(g_trace_launch++ & 1) * 148 * 16 : nullptr;
-#endif
   // upper bound on the tile count (group sizes live on the device): each expert adds at most
   // one partial row tile
   const int64_t m_tiles_max = a.rows_total / BM + a.E;

@@ -33,6 +33,7 @@
 // Every wait on an mbarrier is bounded; on expiry the thread records QARL_ERR_DEVICE_TIMEOUT,
 // raises a CTA-wide abort flag that all other waits poll, and the CTA drains and frees its TMEM.
 #include <algorithm>
+#include <atomic>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -111,6 +112,7 @@ struct __align__(8) SmemTail {
   uint64_t dq_empty[kMaxDqStages];
   uint64_t tmem_full[kMaxAccBufs];
   uint64_t tmem_empty[kMaxAccBufs];
+  uint64_t teardown;
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
@@ -135,6 +137,13 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sm
       return false;
     }
   }
+}
+
+// The same for a whole warp: every lane polls, then the lanes vote, so all 32 take the same
+// branch and the warp-wide operations that follow never see a split warp (lanes polling on
+// their own could disagree when a barrier completes right at the limit).
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, SmemTail* s, const W4Params& p) {
+  return __all_sync(0xFFFFFFFFu, wait_or_abort(bar, parity, s, p) ? 1 : 0) != 0;
 }
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
@@ -219,6 +228,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
       mbar_init(&s->tmem_full[i], 1);
       mbar_init(&s->tmem_empty[i], kEpiWarps);
     }
+    mbar_init(&s->teardown, 1);
     s->abort_flag = 0;
     fence_mbar_init();
   }
@@ -304,7 +314,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
       uint32_t ld_phase = 0, dq_phase = 0, acc_phase = 0;
       bool ok = true;
       for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
-        if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) break;
+        if (!wait_or_abort(&s->tmem_empty[acc], acc_phase ^ 1, s, p)) { ok = false; break; }
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * MT) * BN;
         for (int ks = 0; ks < KS; ++ks) {
           if (!wait_or_abort(&s->a_full[ls], ld_phase, s, p)) { ok = false; break; }
@@ -325,6 +335,12 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           if (++ds == kDqStages) { ds = 0; dq_phase ^= 1; }
         }
         if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1; }
+      }
+      // Nothing of this CTA's tensor work may be in flight when its TMEM and shared memory go
+      // away: after an abort some MMAs may still be executing, so wait (bounded) for them.
+      if (!ok) {
+        umma_commit(&s->teardown);
+        mbar_wait_bounded(&s->teardown, 0, 20000000ull);
       }
     }
   } else if (warp >= kEpiWarps && warp < kEpiWarps + kDqWarps) {
@@ -373,14 +389,14 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
           const uint32_t step = step0 + 2 * g + grp;
           const uint32_t qs = step % kQStages, q_phase = (step / kQStages) & 1u;
           const uint32_t ds = step % kDqStages, dq_phase = (step / kDqStages) & 1u;
-          if (!wait_or_abort(&s->q_full[qs], q_phase, s, p)) { ok = false; break; }
+          if (!warp_wait_or_abort(&s->q_full[qs], q_phase, s, p)) { ok = false; break; }
           // a chunk is [word quad 0..1][row][16 bytes]: consecutive threads read consecutive pieces
           const uint4* q_src = reinterpret_cast<const uint4*>(q_base + static_cast<size_t>(qs) * kQBytes +
                                                               half * kQHalfBytes + nr * 16);
           const uint4 q0 = q_src[0], q1 = q_src[kQHalfBytes / 32];
           __syncwarp();
           if (lane == 0) mbar_arrive(&s->q_empty[qs]);  // the codes are in registers
-          if (!wait_or_abort(&s->dq_empty[ds], dq_phase ^ 1, s, p)) { ok = false; break; }
+          if (!warp_wait_or_abort(&s->dq_empty[ds], dq_phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* row_dst = dq_base + static_cast<size_t>(ds) * kDqBytes + n * 128;
           const uint32_t words[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
@@ -421,7 +437,7 @@ gemm_w4a16_kernel(const __grid_constant__ CUtensorMap tm_a, const W4Params p) {
         if (p.sorted_pair) out_row = min(max(__ldg(p.sorted_pair + row), 0), p.rows_total - 1);  // in bounds even after bad ids
       }
       if (mt == 0) {
-        if (!wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) { ok = false; break; }
+        if (!warp_wait_or_abort(&s->tmem_full[acc], acc_phase, s, p)) { ok = false; break; }
         tc_fence_after_sync();
       }
       const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>((acc * MT + mt) * BN);
@@ -522,13 +538,15 @@ CUresult make_tmap_a(EncodeTiledFn encode, CUtensorMap* m, const void* base, uin
 
 template <int MODE, int MT, int FMT>
 cudaError_t launch_mode(const Launch& L, const CUtensorMap& ta, const W4Params& p, const GemmW4Args& a) {
-  static bool attr_set_dev[64] = {};  // the attribute is sticky per function and device
-  bool& attr_set = attr_set_dev[L.device & 63];
-  if (!attr_set) {
+  // sticky per function and device; atomic: contexts on several host threads may launch at once (both
+  // would set the same value)
+  static std::atomic<bool> attr_set_dev[64];
+  std::atomic<bool>& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set.load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_w4a16_kernel<MODE, MT, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem_bytes<MT>()));
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set.store(true, std::memory_order_release);
   }
   // upper bound on the tile count (group sizes live on the device): each expert adds at most
   // one partial row tile

@@ -4,6 +4,8 @@
 // carries until the process exits.
 #include <stdio.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -20,7 +22,9 @@ constexpr size_t kScratchBytes = kCodesBytes + kScalesBytes;
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_addr[kMaxDevices] = {};
+// per device, written once; atomic because contexts on several host threads may make their first call at
+// the same time (both resolve the same address)
+std::atomic<unsigned char*> g_scratch_addr[kMaxDevices];
 
 }  // namespace
 
@@ -44,7 +48,7 @@ extern "C" int qarl_linear_fwd_static(qarl_ctx* ctx, const void* x, int64_t M, i
 
   // Set-up on the first call for this device: resolve the array's device address while the
   // context's device is current.  (No allocation happens here or anywhere below.)
-  if (g_scratch_addr[ctx->device] == nullptr) {
+  if (g_scratch_addr[ctx->device].load(std::memory_order_acquire) == nullptr) {
     int cur = -1;
     cudaError_t e = cudaGetDevice(&cur);
     if (e != cudaSuccess || cur != ctx->device) {
@@ -58,9 +62,9 @@ extern "C" int qarl_linear_fwd_static(qarl_ctx* ctx, const void* x, int64_t M, i
       snprintf(ctx->err, sizeof(ctx->err), "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
       return QARL_ERR_CUDA;
     }
-    g_scratch_addr[ctx->device] = p;
+    g_scratch_addr[ctx->device].store(p, std::memory_order_release);
   }
-  unsigned char* base = g_scratch_addr[ctx->device];
+  unsigned char* base = g_scratch_addr[ctx->device].load(std::memory_order_acquire);
   uint8_t* xc = base;
   float* xs = reinterpret_cast<float*>(base + kCodesBytes);
 

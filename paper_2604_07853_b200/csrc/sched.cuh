@@ -28,9 +28,12 @@ __device__ __forceinline__ TileCoord decode_tile(const int32_t* off, const int32
 
 // Fills off[0..E] from the device offsets (or one dense group) and prefix[0..E] with the
 // exclusive scan of tiles per expert.  Called by every thread of the CTA; contains barriers.
+// Boundaries are forced into [0, rows_total] and a group that ends before it starts gets no
+// tile, so whatever the offsets array holds, no tile reaches outside the tensors.
 __device__ __forceinline__ void build_tile_list(int32_t* off, int32_t* prefix, const int32_t* offsets, int rows_total,
                                                 int E, int rows_per_tile, int n_tiles) {
-  for (int e = threadIdx.x; e <= E; e += blockDim.x) off[e] = offsets ? offsets[e] : (e == 0 ? 0 : rows_total);
+  for (int e = threadIdx.x; e <= E; e += blockDim.x)
+    off[e] = offsets ? min(max(offsets[e], 0), rows_total) : (e == 0 ? 0 : rows_total);
   __syncthreads();
   if (threadIdx.x < 32) {
     const int lane = threadIdx.x;
@@ -38,7 +41,7 @@ __device__ __forceinline__ void build_tile_list(int32_t* off, int32_t* prefix, c
     for (int base = 0; base < E; base += 32) {
       const int e = base + lane;
       int v = 0;
-      if (e < E) v = ((off[e + 1] - off[e] + rows_per_tile - 1) / rows_per_tile) * n_tiles;
+      if (e < E) v = ((max(off[e + 1] - off[e], 0) + rows_per_tile - 1) / rows_per_tile) * n_tiles;
       int inc = v;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {

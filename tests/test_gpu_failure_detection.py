@@ -32,3 +32,43 @@ def test_expired_wait_is_reported_and_context_survives():
         ctx.check_device_status()
     assert ei.value.status == -7
     ctx.close()
+
+
+@pytest.mark.parametrize("stop_after", [0, 1, 5])
+def test_gemm_pipeline_wait_expires_and_context_survives(stop_after):
+    """The FP8 GEMM's own abort protocol: the TMA producer stops arming stages (a host-set test
+    switch), so the MMA role waits on a stage that nothing fills; its bounded wait (1 ms here)
+    runs out, the CTA aborts, drains and frees its TMEM, the kernel returns, the status word says
+    QARL_ERR_DEVICE_TIMEOUT, and the next call with the normal settings gives the reference bytes."""
+    build.build()
+    ctx = binding.Context(0)
+    case = inputs.linear_case(5, 300, 384, 1024)           # 3 row tiles x 2 column tiles x 8 K-blocks
+    wc, ws = ctx.quantize_weight(bits_to_torch(case.w))
+    x = bits_to_torch(case.x)
+    ref = ctx.linear_fwd(x, wc, ws).clone()
+    assert ctx.poll() == 0
+    ctx.harness_set_wait_limit_ns(1_000_000)
+    ctx.harness_stop_producer_after(stop_after)
+    t0 = time.perf_counter()
+    ctx.linear_fwd(x, wc, ws)
+    assert ctx.poll() == -7
+    assert time.perf_counter() - t0 < 1.0
+    ctx.harness_stop_producer_after(-1)
+    ctx.harness_set_wait_limit_ns(0)
+    assert ctx.poll() == 0
+    for _ in range(2):
+        assert torch.equal(ctx.linear_fwd(x, wc, ws), ref) and ctx.poll() == 0
+    # the same through the grouped (MoE) kernels
+    c = inputs.moe_case(2, 96, h=512, i=256, e=8, k=2)
+    w13c, w13s = ctx.quantize_weight(bits_to_torch(c.w13))
+    w2c, w2s = ctx.quantize_weight(bits_to_torch(c.w2))
+    args = (bits_to_torch(c.x), torch.from_numpy(c.ids).cuda(), torch.from_numpy(c.weights).cuda(), w13c, w13s, w2c, w2s)
+    ref_moe = ctx.moe_fwd(*args).clone()
+    ctx.harness_set_wait_limit_ns(1_000_000)
+    ctx.harness_stop_producer_after(min(stop_after, 2))     # a gate_up tile of this shape has 4 stages
+    ctx.moe_fwd(*args)
+    assert ctx.poll() == -7
+    ctx.harness_stop_producer_after(-1)
+    ctx.harness_set_wait_limit_ns(0)
+    assert torch.equal(ctx.moe_fwd(*args), ref_moe) and ctx.poll() == 0
+    ctx.close()

@@ -3,8 +3,8 @@ qarl_linear_fwd.  It exists for callers that cannot obtain device memory at call
 server whose memory pool already owns the whole GPU, a plugin under someone else's allocator):
 its scratch is a fixed array inside the library, shared by every call on the device and never
 cleared.  Two calls in a row, the second on a smaller and different input, check that nothing
-stale from the first call leaks into the second.  Collected last so that a run stopping at the
-first failure has already run everything else; it passes alone in a fresh process as well."""
+stale from the first call leaks into the second.  The test needs no state from any other test
+(it creates its own context) and leaves none behind."""
 import numpy as np
 import pytest
 import torch
