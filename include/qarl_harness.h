@@ -47,6 +47,22 @@ int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream);
 int qarl_harness_set_wait_limit_ns(qarl_ctx* ctx, uint64_t limit_ns);
 int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages);
 
+/* Roofline denominators measured with the library's own instructions (used by the benchmark; the
+ * paper has no counterpart).  Both only launch a kernel on `stream`; the caller times it with
+ * CUDA events.
+ *
+ * qarl_harness_fp8_mma_peak: every SM issues `kblocks_per_sm` back-to-back K-blocks of four
+ * tcgen05.mma kind::f8f6f4 instructions (128 x 256 x 32, e4m3 operands resident in shared memory,
+ * fp32 accumulators in TMEM) -- the instruction shape and operand path of the FP8 GEMM without its
+ * loads, promotion and epilogue.  *flop_out (host pointer, may be NULL) receives the floating-point
+ * operations the launch performs (2 * 128 * 256 * 128 per K-block per SM).
+ *
+ * qarl_harness_read_stream: reads `bytes` bytes (a multiple of 16, 16-byte aligned device pointer)
+ * once with 16-byte loads, eight in flight per thread, and stores nothing (sink4: 4 writable device
+ * bytes that are practically never written). */
+int qarl_harness_fp8_mma_peak(qarl_ctx* ctx, int64_t kblocks_per_sm, double* flop_out, void* stream);
+int qarl_harness_read_stream(qarl_ctx* ctx, const void* buf, size_t bytes, void* sink4, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

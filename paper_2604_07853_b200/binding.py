@@ -39,7 +39,7 @@ EXPORTS = [
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest", "qarl_harness_set_wait_limit_ns",
-                   "qarl_harness_stop_producer_after"]
+                   "qarl_harness_stop_producer_after", "qarl_harness_fp8_mma_peak", "qarl_harness_read_stream"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise"]
 
@@ -159,6 +159,10 @@ def load() -> C.CDLL:
     L.qarl_harness_set_wait_limit_ns.argtypes = [p, C.c_uint64]
     L.qarl_harness_stop_producer_after.restype = C.c_int
     L.qarl_harness_stop_producer_after.argtypes = [p, i64]
+    L.qarl_harness_fp8_mma_peak.restype = C.c_int
+    L.qarl_harness_fp8_mma_peak.argtypes = [p, i64, C.POINTER(C.c_double), p]
+    L.qarl_harness_read_stream.restype = C.c_int
+    L.qarl_harness_read_stream.argtypes = [p, p, sz, p, p]
     _lib = L
     return L
 
@@ -245,6 +249,17 @@ class Context:
     def harness_stop_producer_after(self, stages: int):
         """FP8 GEMM TMA producers stop arming stages after `stages` (negative: normal operation)."""
         self._check(self.lib.qarl_harness_stop_producer_after(self.h, stages))
+
+    def harness_fp8_mma_peak(self, kblocks_per_sm: int) -> float:
+        """Launch the dense FP8 MMA peak kernel; returns the floating-point operations it performs."""
+        fl = C.c_double(0.0)
+        self._check(self.lib.qarl_harness_fp8_mma_peak(self.h, kblocks_per_sm, C.byref(fl), _stream()))
+        return fl.value
+
+    def harness_read_stream(self, buf: torch.Tensor, sink: torch.Tensor):
+        """Launch the read-only streaming kernel over `buf` (bytes a multiple of 16)."""
+        self._check(self.lib.qarl_harness_read_stream(self.h, _ptr(buf), buf.numel() * buf.element_size(),
+                                                      _ptr(sink), _stream()))
 
     def harness_rmsnorm(self, x: torch.Tensor, eps: float = 1e-6, out=None):
         """Row-invariant RMSNorm (weight 1) used by the alignment-stack test; not part of the API."""

@@ -374,6 +374,20 @@ int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages) {
   return QARL_OK;
 }
 
+int qarl_harness_fp8_mma_peak(qarl_ctx* ctx, int64_t kblocks_per_sm, double* flop_out, void* stream) {
+  if (!ctx || kblocks_per_sm < 1 || kblocks_per_sm > 100000000ll) return QARL_ERR_INVALID_ARG;
+  if (flop_out) *flop_out = 2.0 * 128 * 256 * 128 * static_cast<double>(kblocks_per_sm) * ctx->sm_count;
+  cudaError_t e = launch_fp8_mma_peak(make_launch(ctx, stream), static_cast<int>(kblocks_per_sm));
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "fp8_mma_peak");
+}
+
+int qarl_harness_read_stream(qarl_ctx* ctx, const void* buf, size_t bytes, void* sink4, void* stream) {
+  if (!ctx || !buf || !sink4) return QARL_ERR_INVALID_ARG;
+  if (!aligned16(buf) || (reinterpret_cast<uintptr_t>(sink4) & 3u)) return QARL_ERR_MISALIGNED;
+  cudaError_t e = launch_read_stream(make_launch(ctx, stream), buf, bytes, static_cast<uint32_t*>(sink4));
+  return e == cudaSuccess ? QARL_OK : cuda_fail(ctx, e, "read_stream");
+}
+
 int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream) {
   if (!ctx) return QARL_ERR_INVALID_ARG;
   if (limit_ns < 1000) limit_ns = 1000;

@@ -109,6 +109,8 @@ cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32
                            int64_t H, int64_t E, uint16_t* out, const int32_t* pos_of_pair = nullptr);
 
 cudaError_t launch_wait_selftest(const Launch& L, unsigned long long limit_ns);
+cudaError_t launch_fp8_mma_peak(const Launch& L, int kblocks);
+cudaError_t launch_read_stream(const Launch& L, const void* buf, size_t bytes, uint32_t* sink);
 cudaError_t launch_rmsnorm(const Launch& L, const uint16_t* x, int64_t M, int64_t H, float eps, uint16_t* out);
 
 enum GemmMode { kModeLinear = 0, kModeGateUp = 1, kModeDown = 2 };

@@ -1,5 +1,7 @@
 // Test-harness glue (not part of the quantized-forward API): a row-invariant RMSNorm used
 // between layers by the alignment-stack test.
+#include <atomic>
+
 #include "common.cuh"
 #include "../../include/qarl_harness.h"
 #include "ptx_sm100.cuh"
@@ -52,7 +54,108 @@ __global__ void wait_selftest_kernel(unsigned long long limit_ns, int* status) {
   }
 }
 
+// ---- roofline denominators measured with the library's own instructions --------------------
+// Dense FP8 tensor-core peak: one CTA per SM, one thread issuing back-to-back K-blocks of four
+// tcgen05.mma kind::f8f6f4 (128 x 256 x 32, e4m3 x e4m3 -> fp32) on operands that already sit in
+// shared memory (two 48 KB operand sets, 128-byte swizzle layout, pseudo-random finite codes) into
+// two TMEM accumulators used in turn.  No TMA, no promotion, no epilogue: what the tensor pipe and
+// its shared-memory operand fetch sustain with the instruction shape the GEMM uses.
+__global__ void __launch_bounds__(128, 1) fp8_mma_peak_kernel(int kblocks, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t done[2];
+  __shared__ uint32_t taddr;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&done[0], 1);
+    ptx::mbar_init(&done[1], 1);
+    ptx::fence_mbar_init();
+  }
+  // finite e4m3 codes (exponent field never all ones together with mantissa 7): a cheap hash
+  uint32_t* w = reinterpret_cast<uint32_t*>(smem);
+  for (int i = threadIdx.x; i < 2 * 48 * 1024 / 4; i += blockDim.x) {
+    uint32_t h = (static_cast<uint32_t>(i) + 977u * blockIdx.x) * 2654435761u;
+    h ^= h >> 15;
+    w[i] = h & 0xBFBFBFBFu;  // clears exponent bit 6 of every byte: |value| < 2, no NaN code
+  }
+  if (warp == 0) {
+    ptx::tmem_alloc(&taddr, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::fence_proxy_async_smem();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  if (warp == 1 && lane == 0) {
+    constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, 256);
+    uint32_t ph[2] = {0, 0};
+    bool ok = true;
+    for (int i = 0; i < kblocks && ok; ++i) {
+      const int b = i & 1;
+      if (i >= 2) {  // the accumulator's previous K-block has completed
+        ok = ptx::mbar_wait_bounded(&done[b], ph[b], 2000000000ull);
+        ph[b] ^= 1;
+      }
+      const uint32_t a_addr = ptx::smem_u32(smem + b * 48 * 1024);
+      const uint64_t ad = ptx::umma_desc_k_sw128(a_addr), bd = ptx::umma_desc_k_sw128(a_addr + 16384);
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) ptx::umma_f8(taddr + b * 256, ad + 2 * k4, bd + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
+      ptx::umma_commit(&done[b]);
+    }
+    for (int b = 0; b < 2 && ok; ++b)
+      if (kblocks > b) ok = ptx::mbar_wait_bounded(&done[b], ph[b], 2000000000ull);
+    if (!ok) set_status(status, QARL_ERR_DEVICE_TIMEOUT);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(taddr, 512);
+  }
+}
+
+// Read-only streaming peak: every thread keeps eight independent 16-byte loads in flight over a
+// grid-strided sweep of the buffer and folds them into one word that is never stored.
+__global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restrict__ p, size_t n, uint32_t* sink) {
+  uint32_t acc = 0;
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  for (; i + 7 * stride < n; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __ldg(p + i + j * stride);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc ^= v[j].x ^ v[j].y ^ v[j].z ^ v[j].w;
+  }
+  for (; i < n; i += stride) {
+    const uint4 v = __ldg(p + i);
+    acc ^= v.x ^ v.y ^ v.z ^ v.w;
+  }
+  if (acc == 0x9E3779B9u) *sink = acc;  // practically never: keeps the loads alive
+}
+
 }  // namespace
+
+cudaError_t launch_fp8_mma_peak(const Launch& L, int kblocks) {
+  static std::atomic<bool> attr_set_dev[64];
+  constexpr int kSmem = 1024 + 2 * 48 * 1024;
+  std::atomic<bool>& attr_set = attr_set_dev[L.device & 63];
+  if (!attr_set.load(std::memory_order_acquire)) {
+    cudaError_t e = cudaFuncSetAttribute(fp8_mma_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    attr_set.store(true, std::memory_order_release);
+  }
+  fp8_mma_peak_kernel<<<L.sm_count, 128, kSmem, L.stream>>>(kblocks, L.d_status);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_read_stream(const Launch& L, const void* buf, size_t bytes, uint32_t* sink) {
+  if (bytes < 16) return cudaSuccess;
+  read_stream_kernel<<<L.sm_count * 4, 512, 0, L.stream>>>(static_cast<const uint4*>(buf), bytes / 16, sink);
+  ++*L.launches;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_wait_selftest(const Launch& L, unsigned long long limit_ns) {
   wait_selftest_kernel<<<1, 32, 0, L.stream>>>(limit_ns, L.d_status);
