@@ -47,6 +47,13 @@ int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream);
 int qarl_harness_set_wait_limit_ns(qarl_ctx* ctx, uint64_t limit_ns);
 int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages);
 
+/* The grouped FP8 GEMM has two kernels that produce the same bytes: the wide-tile one (128 token rows
+ * x 256 weight rows per tile) and the swapped-operand one for decode-sized groups (128 weight rows x
+ * at most 32 token rows).  The library picks by size; this call forces one (1 = wide, 2 = decode where
+ * it applies: grouped calls with K <= 8192) or restores the automatic choice (0), so that a test can
+ * run one input through both and compare.  Host side only, stored in the context. */
+int qarl_harness_set_gemm_path(qarl_ctx* ctx, int path);
+
 /* Roofline denominators measured with the library's own instructions (used by the benchmark; the
  * paper has no counterpart).  Both only launch a kernel on `stream`; the caller times it with
  * CUDA events.

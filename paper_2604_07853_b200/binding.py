@@ -39,7 +39,8 @@ EXPORTS = [
 ]
 STATIC_LINEAR_MAX_ELEMS = 4 * 1024 * 1024
 HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest", "qarl_harness_set_wait_limit_ns",
-                   "qarl_harness_stop_producer_after", "qarl_harness_fp8_mma_peak", "qarl_harness_read_stream"]
+                   "qarl_harness_stop_producer_after", "qarl_harness_fp8_mma_peak", "qarl_harness_read_stream",
+                   "qarl_harness_set_gemm_path"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
           "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise"]
 
@@ -159,6 +160,8 @@ def load() -> C.CDLL:
     L.qarl_harness_set_wait_limit_ns.argtypes = [p, C.c_uint64]
     L.qarl_harness_stop_producer_after.restype = C.c_int
     L.qarl_harness_stop_producer_after.argtypes = [p, i64]
+    L.qarl_harness_set_gemm_path.restype = C.c_int
+    L.qarl_harness_set_gemm_path.argtypes = [p, C.c_int]
     L.qarl_harness_fp8_mma_peak.restype = C.c_int
     L.qarl_harness_fp8_mma_peak.argtypes = [p, i64, C.POINTER(C.c_double), p]
     L.qarl_harness_read_stream.restype = C.c_int
@@ -249,6 +252,10 @@ class Context:
     def harness_stop_producer_after(self, stages: int):
         """FP8 GEMM TMA producers stop arming stages after `stages` (negative: normal operation)."""
         self._check(self.lib.qarl_harness_stop_producer_after(self.h, stages))
+
+    def harness_set_gemm_path(self, path: int):
+        """0: automatic choice of the grouped FP8 GEMM kernel, 1: wide tiles, 2: decode (swapped operands)."""
+        self._check(self.lib.qarl_harness_set_gemm_path(self.h, path))
 
     def harness_fp8_mma_peak(self, kblocks_per_sm: int) -> float:
         """Launch the dense FP8 MMA peak kernel; returns the floating-point operations it performs."""

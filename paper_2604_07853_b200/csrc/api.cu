@@ -368,6 +368,12 @@ int qarl_harness_set_wait_limit_ns(qarl_ctx* ctx, uint64_t limit_ns) {
   return QARL_OK;
 }
 
+int qarl_harness_set_gemm_path(qarl_ctx* ctx, int path) {
+  if (!ctx || path < 0 || path > 2) return QARL_ERR_INVALID_ARG;
+  ctx->gemm_path = path;
+  return QARL_OK;
+}
+
 int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages) {
   if (!ctx) return QARL_ERR_INVALID_ARG;
   ctx->stop_after_stages = stages < 0 ? -1 : static_cast<int>(stages > 0x7FFFFFFF ? 0x7FFFFFFF : stages);

@@ -23,6 +23,7 @@ inline Launch make_launch(qarl_ctx* ctx, void* stream) {
   L.launches = &ctx->launches;
   L.wait_limit_ns = ctx->wait_limit_ns;
   L.stop_after_stages = ctx->stop_after_stages;
+  L.gemm_path = ctx->gemm_path;
   return L;
 }
 

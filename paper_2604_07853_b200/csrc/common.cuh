@@ -63,6 +63,7 @@ struct Launch {
   int64_t* launches;  // host counter
   unsigned long long wait_limit_ns = 0;  // bound of every device-side barrier wait (0: the default, 2 s)
   int stop_after_stages = -1;            // test harness only: FP8 GEMM producers stop after this many stages
+  int gemm_path = 0;                     // test harness only: 0 = automatic, 1 = wide-tile kernel, 2 = decode kernel
 };
 
 // Launch with the programmatic-stream-serialization attribute (see pdl_wait above).
@@ -144,6 +145,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 // Returns cudaSuccess, or an error; *cu_err receives a driver error from tensor-map encoding.
 cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
+// The swapped-operand kernel for decode-sized row groups (same bytes out; see gemm_decode_sm100.cu);
+// launch_gemm picks it when gemm_decode_applies (L.gemm_path forces one or the other in tests).
+bool gemm_decode_applies(const GemmArgs& a);
+cudaError_t launch_gemm_decode(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
 
 // ---- W4A16 (4-bit group-quantized weights, bf16 activations) --------------------------------
 // 4-bit weight formats (Sec. 2.2): unsigned integer codes with a zero point, or e2m1 floating point
@@ -239,6 +244,7 @@ struct qarl_ctx {
   int64_t launches;
   unsigned long long wait_limit_ns = 0;  // 0: default; set only by the test harness
   int stop_after_stages = -1;            // -1: off; set only by the test harness
+  int gemm_path = 0;                     // 0: automatic; set only by the test harness
   qarl::EncodeTiledFn encode;
   char err[256];
   // stage timing: marks[i] closes stage mark_stage[i] (-1: an opening mark)

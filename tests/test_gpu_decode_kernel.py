@@ -1,0 +1,65 @@
+"""The grouped FP8 GEMM has a wide-tile kernel and a swapped-operand kernel for decode-sized groups.
+Both must give the same bytes for every row (the fixed K-reduction order of App. C holds across
+kernels, not only across batch sizes): one input goes through both, forced by the harness switch,
+and every stage the layer exposes is compared bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_07853_b200 import binding, build, inputs
+from util import bits_to_torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    build.build()
+    c = binding.Context(0)
+    yield c
+    c.harness_set_gemm_path(0)
+    c.close()
+
+
+def _layer(ctx, c, path, debug=True):
+    ctx.harness_set_gemm_path(path)
+    w13c, w13s = ctx.quantize_weight(bits_to_torch(c.w13))
+    w2c, w2s = ctx.quantize_weight(bits_to_torch(c.w2))
+    r = ctx.moe_fwd(bits_to_torch(c.x), torch.from_numpy(c.ids).cuda(), torch.from_numpy(c.weights).cuda(),
+                    w13c, w13s, w2c, w2s, debug=debug)
+    assert ctx.poll() == 0
+    ctx.harness_set_gemm_path(0)
+    return r
+
+
+@pytest.mark.parametrize("m,h,i,e,k", [(256, 2048, 768, 128, 8), (64, 512, 256, 8, 2), (1, 512, 256, 8, 2),
+                                       (300, 384, 128, 4, 2), (8, 2048, 768, 128, 8), (33, 256, 384, 2, 1)])
+def test_decode_kernel_equals_wide_kernel_stage_by_stage(ctx, m, h, i, e, k):
+    c = inputs.moe_case(21, m, h=h, i=i, e=e, k=k)
+    out_w, d_w = _layer(ctx, c, 1)
+    out_d, d_d = _layer(ctx, c, 2)
+    P = m * k
+    for key in ("expert_offsets", "sorted_pair", "gate_up", "h", "h_codes", "h_scales", "down_f32"):
+        a, b = d_w[key], d_d[key]
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), key
+    assert torch.equal(out_w, out_d)
+    # and without the debug dumps
+    assert torch.equal(_layer(ctx, c, 1, debug=False), _layer(ctx, c, 2, debug=False))
+    assert P > 0
+
+
+def test_automatic_choice_matches_both(ctx):
+    """Decode shape: the automatic path (the decode kernel at this size) against the forced wide one."""
+    c = inputs.moe_case(3, 256)
+    auto = _layer(ctx, c, 0, debug=False)
+    wide = _layer(ctx, c, 1, debug=False)
+    assert torch.equal(auto, wide)
+
+
+def test_skewed_groups_through_the_decode_kernel(ctx):
+    """Groups far larger than one 32-row chunk (and empty ones) through the decode kernel."""
+    c = inputs.moe_case(5, 700, h=512, i=256, e=8, k=2, zipf_s=1.1)
+    out_w, d_w = _layer(ctx, c, 1)
+    out_d, d_d = _layer(ctx, c, 2)
+    assert torch.equal(d_w["h_codes"], d_d["h_codes"]) and torch.equal(d_w["down_f32"].view(torch.int32), d_d["down_f32"].view(torch.int32))
+    assert torch.equal(out_w, out_d)
