@@ -58,14 +58,19 @@ def test_moe_training_shape_sampled(ctx):
     sizes = np.diff(off)
     assert sizes.sum() == M * k and sizes.max() > 10 * np.median(sizes)      # skewed, as intended
 
-    # sampled sorted positions: first/last rows of the smallest, median and largest groups plus random ones
+    # sampled sorted positions: the first and the last row of EVERY expert group (where a tile's mask
+    # decides), the middle of the smallest, median and largest groups, and random ones: > 512 rows
     rng = np.random.default_rng(0)
     order = np.argsort(sizes)
     picks = []
+    for e in range(E):
+        if sizes[e] > 0:
+            picks += [off[e], off[e + 1] - 1]
     for e in (order[np.nonzero(sizes[order])[0][0]], order[E // 2], order[-1]):
-        picks += [off[e], off[e + 1] - 1, (off[e] + off[e + 1]) // 2]
-    picks += list(rng.integers(0, M * k, size=40))
+        picks.append((off[e] + off[e + 1]) // 2)
+    picks += list(rng.integers(0, M * k, size=300))
     picks = np.array(sorted(set(int(q) for q in picks)))
+    assert picks.size >= 512
     tok = srt[picks] // k
     exp = ids_h.reshape(-1)[srt[picks]]
     xs_bits = torch_to_bits(x[torch.from_numpy(tok).cuda()])
@@ -76,8 +81,16 @@ def test_moe_training_shape_sampled(ctx):
     hs = d["h_scales"][torch.from_numpy(picks).cuda()].cpu().numpy()
     dn = d["down_f32"][torch.from_numpy(picks).cuda()].cpu().numpy()
     far = 0
+    wcache = {}
+
+    def weights_of(e):
+        if e not in wcache:
+            wcache.clear()                      # picks are sorted by position, hence by expert: keep one
+            wcache[e] = (w13c[e].cpu().numpy(), w13s[e].cpu().numpy(), w2c[e].cpu().numpy(), w2s[e].cpu().numpy())
+        return wcache[e]
+
     for i, e in enumerate(exp):
-        a13, s13 = w13c[e].cpu().numpy(), w13s[e].cpu().numpy()
+        a13, s13, a2, s2 = weights_of(int(e))
         o32, o16 = oracle.linear_q(xc[i:i + 1], xs[i:i + 1], a13, s13)
         dist = bf16_ulp_dist(gu[i:i + 1], o16)
         bad = dist > 1
@@ -89,7 +102,6 @@ def test_moe_training_shape_sampled(ctx):
         assert bf16_ulp_dist(hh[i:i + 1], oracle.swiglu(gu[i:i + 1])).max() <= 1
         oc, os_ = oracle.quantize_act(hh[i:i + 1])
         assert np.array_equal(hc[i:i + 1], oc) and np.array_equal(hs[i:i + 1], os_)
-        a2, s2 = w2c[e].cpu().numpy(), w2s[e].cpu().numpy()
         o32, _ = oracle.linear_q(hc[i:i + 1], hs[i:i + 1], a2, s2)
         tol = _tol(dec, hc[i:i + 1], hs[i:i + 1], a2, s2)
         assert (np.abs(dn[i:i + 1].astype(np.float64) - o32) <= tol).all()
@@ -98,7 +110,7 @@ def test_moe_training_shape_sampled(ctx):
     # combine: sampled tokens, bit-exact given the GPU's fp32 rows
     pos = np.empty(M * k, dtype=np.int64)
     pos[srt] = np.arange(M * k)
-    for t in rng.integers(0, M, size=24):
+    for t in rng.integers(0, M, size=256):
         rows = torch.from_numpy(pos[t * k:(t + 1) * k]).cuda()
         y = d["down_f32"][rows].cpu().numpy()
         ref = oracle.combine(y, ids_h[t:t + 1], wts_h[t:t + 1])

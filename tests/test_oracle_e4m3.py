@@ -121,3 +121,21 @@ def test_bf16_rne_vs_torch():
     v = v[np.isfinite(v)]
     ref = torch.from_numpy(v).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(oracle.bf16_rne(v), ref)
+
+
+def test_encode_every_fp32_bit_pattern_vs_torch_cast():
+    """All 2^32 fp32 bit patterns (the finite ones: NaN and infinity are outside the contract) through
+    the oracle's encoder and through torch's float8_e4m3fn cast after an explicit clamp to +-448
+    (the cast rounds to nearest even; the clamp is the saturation the reading adds)."""
+    n = 1 << 26
+    checked = 0
+    for base in range(0, 1 << 32, n):
+        v = np.arange(base, base + n, dtype=np.uint64).astype(np.uint32).view(np.float32)
+        fin = np.isfinite(v)
+        if not fin.all():
+            v = v[fin]
+        got = oracle.e4m3_encode(v)
+        ref = torch.from_numpy(v).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+        assert np.array_equal(got, ref), hex(base)
+        checked += v.size
+    assert checked == (1 << 32) - (1 << 24)              # everything but the two exponent-255 ranges (2 x 2^23)
