@@ -274,17 +274,24 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   pb.pos_of_pair = reinterpret_cast<int32_t*>(ws + pl.pos_of_pair);
   // Bad ids are skipped by the permutation and leave their entries of these arrays stale; every
   // consumer clamps the indices it reads from them, so no clearing pass is needed.
-  mark(ctx, L.stream, -1);
-  if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
-  mark(ctx, L.stream, QARL_STAGE_PERMUTE);
-
   uint8_t* a_codes = ws + pl.a_codes;
   float* a_scales = reinterpret_cast<float*>(ws + pl.a_scales);
   float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
-  if ((e = launch_quantize_act(L, static_cast<const uint16_t*>(x), M, H, H, a_codes, a_scales, pb.pos_of_pair,
-                               static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
-    return cuda_fail(ctx, e, "quantize_act");
-  mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
+  mark(ctx, L.stream, -1);
+  if (moe_prep_small_applies(M, k, E)) {
+    // decode-sized: grouping + quantization + scatter in one launch (timed as the quantize_act stage)
+    if ((e = launch_moe_prep_small(L, ids, M, k, E, pb, static_cast<const uint16_t*>(x), H, wts, a_codes, a_scales,
+                                   sorted_w)) != cudaSuccess)
+      return cuda_fail(ctx, e, "moe_prep");
+    mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
+  } else {
+    if ((e = launch_permute(L, ids, M, k, E, pb)) != cudaSuccess) return cuda_fail(ctx, e, "permute");
+    mark(ctx, L.stream, QARL_STAGE_PERMUTE);
+    if ((e = launch_quantize_act(L, static_cast<const uint16_t*>(x), M, H, H, a_codes, a_scales, pb.pos_of_pair,
+                                 static_cast<int>(k), wts, sorted_w)) != cudaSuccess)
+      return cuda_fail(ctx, e, "quantize_act");
+    mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
+  }
 
   uint8_t* h_codes = ws + pl.h_codes;
   float* h_scales = reinterpret_cast<float*>(ws + pl.h_scales);

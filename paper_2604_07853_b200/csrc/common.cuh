@@ -105,6 +105,12 @@ int64_t permute_num_chunks(int64_t P);
 cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
                            const PermuteBuffers& b);
 
+// Decode-sized layers (M * k <= 2048): the grouping and the scattering activation quantization in one launch.
+bool moe_prep_small_applies(int64_t M, int64_t k, int64_t E);
+cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
+                                  const PermuteBuffers& b, const uint16_t* x, int64_t K, const float* pair_w,
+                                  uint8_t* codes, float* scales, float* sorted_w);
+
 // pos_of_pair == nullptr: contrib is indexed by flat pair id; else by pos_of_pair[pair] (sorted order)
 cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
                            int64_t H, int64_t E, uint16_t* out, const int32_t* pos_of_pair = nullptr);

@@ -8,6 +8,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "quant_device.cuh"
 
 namespace qarl {
 namespace {
@@ -186,6 +187,127 @@ __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int3
   }
 }
 
+// ---- decode-sized layers (P <= 2048): grouping + activation quantization in ONE launch --------
+// Every CTA repeats the whole (tiny, deterministic) grouping in its shared memory -- the ids are 8 KB
+// and sit in L2 -- and then quantizes its own share of the activation groups, writing each token's
+// codes, scales and combine weight to the token's k expert-sorted rows.  CTA 0 also publishes offsets,
+// sorted_pair and pos_of_pair.  One launch and one dependency instead of two of each; the loads of
+// the activations are issued before the grouping so that their latency hides behind it.
+__global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
+    const int32_t* __restrict__ ids, int64_t P, int E, int fanout, const uint16_t* __restrict__ x, int64_t M, int64_t K,
+    const float* __restrict__ pair_w, int32_t* __restrict__ offsets, int32_t* __restrict__ sorted_pair,
+    int32_t* __restrict__ pos_of_pair, uint8_t* __restrict__ codes, float* __restrict__ scales,
+    float* __restrict__ sorted_w, int* status) {
+  extern __shared__ int32_t sm[];
+  pdl_trigger();
+  pdl_wait();
+  int32_t* whist = sm;                 // [kWarps][E]
+  int32_t* total = sm + kWarps * E;    // [E]
+  int32_t* scratch = total + E;        // [33]
+  int32_t* spos = scratch + 33;        // [kChunk] sorted position of every pair (-1: bad id)
+  const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+  const bool publish = blockIdx.x == 0;
+
+  // this thread's share of the quantization: 16 elements of one 1x128 group
+  const int64_t kb = K / kBlock;
+  const int64_t gid = (static_cast<int64_t>(blockIdx.x) * blockDim.x + tid) >> 3;
+  const bool live = gid < M * kb;
+  const int64_t g = live ? gid : 0;
+  const int64_t row = g / kb, b = g % kb;
+  const int sub = tid & 7;
+  uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+  if (live) {
+    const uint4* src = reinterpret_cast<const uint4*>(x + row * K + b * kBlock + sub * 16);
+    v0 = __ldg(src);
+    v1 = __ldg(src + 1);
+  }
+
+  // ---- the grouping (as permute_single_cta_kernel), positions kept in shared memory
+  constexpr int kRounds = kPairsPerWarp / 32;
+  const int64_t p0 = static_cast<int64_t>(wid) * kPairsPerWarp + lane;
+  int my[kRounds];
+  bool bad = false;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int64_t p = p0 + r * 32;
+    int e = -1;
+    if (p < P) {
+      e = __ldg(ids + p);
+      if (e < 0 || e >= E) { bad = true; e = -1; }
+    }
+    my[r] = e;
+  }
+  if (bad && publish) set_status(status, QARL_ERR_BAD_EXPERT_ID);
+  for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
+  for (int i = tid; i < kChunk; i += kThreads) spos[i] = -1;
+  __syncthreads();
+  int32_t* hist_w = whist + wid * E;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int e = my[r];
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += kThreads) {
+    int s = 0;
+    for (int w = 0; w < kWarps; ++w) s += whist[w * E + e];
+    total[e] = s;
+  }
+  __syncthreads();
+  const int all = block_exclusive_scan(total, E, scratch);
+  for (int e = tid; e < E; e += kThreads) {
+    int run = total[e];
+    if (publish) offsets[e] = run;
+    for (int w = 0; w < kWarps; ++w) {
+      const int c = whist[w * E + e];
+      whist[w * E + e] = run;
+      run += c;
+    }
+  }
+  if (publish && tid == 0) offsets[E] = all;
+  __syncthreads();
+  const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int e = my[r];
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    int pos = -1;
+    if (e >= 0) pos = hist_w[e] + __popc(peers & lt);
+    __syncwarp();
+    if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
+    __syncwarp();
+    if (e >= 0) {
+      const int64_t p = p0 + r * 32;
+      spos[p] = pos;
+      if (publish) {
+        sorted_pair[pos] = static_cast<int32_t>(p);
+        pos_of_pair[p] = pos;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- quantize this thread's group and scatter it to the token's sorted rows
+  uint32_t m = fold_halves(absmax_u4(absmax_u4(0, v0), v1));
+#pragma unroll
+  for (int o = 4; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  float inv;
+  const float s = block_scale(bf16_bits_to_f32(m), &inv);
+  uint4 out;
+  encode8(v0, inv, out.x, out.y);
+  encode8(v1, inv, out.z, out.w);
+  if (!live) return;
+  for (int j = 0; j < fanout; ++j) {
+    const int d = spos[row * fanout + j];
+    if (d < 0) continue;  // a pair with a bad expert id has no sorted row
+    *reinterpret_cast<uint4*>(codes + static_cast<int64_t>(d) * K + b * kBlock + sub * 16) = out;
+    if (sub == 0) scales[static_cast<int64_t>(d) * kb + b] = s;
+    if (sub == 0 && b == 0 && sorted_w != nullptr) sorted_w[d] = pair_w[row * fanout + j];
+  }
+}
+
 // ---- large problems: per-chunk histogram, one-CTA scan, per-chunk scatter ----------------
 __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ ids, int64_t P, int E,
                                                                 int32_t* __restrict__ chunk_hist, int* status) {
@@ -283,6 +405,26 @@ __global__ void __launch_bounds__(kThreads) permute_scatter_kernel(const int32_t
 }  // namespace
 
 int64_t permute_num_chunks(int64_t P) { return (P + kChunk - 1) / kChunk; }
+
+bool moe_prep_small_applies(int64_t M, int64_t k, int64_t E) { return M * k <= kChunk && E <= 1024; }
+
+cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
+                                  const PermuteBuffers& b, const uint16_t* x, int64_t K, const float* pair_w,
+                                  uint8_t* codes, float* scales, float* sorted_w) {
+  const int e = static_cast<int>(E);
+  const size_t smem = (static_cast<size_t>(kWarps) * e + e + 33 + kChunk) * sizeof(int32_t);
+  if (smem > 48 * 1024) {
+    cudaError_t err = cudaFuncSetAttribute(moe_prep_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+  }
+  const int64_t groups = M * (K / kBlock);
+  const int64_t blocks = std::max<int64_t>(1, (groups * 8 + kThreads - 1) / kThreads);
+  ++*L.launches;
+  return launch_pdl(moe_prep_small_kernel, static_cast<unsigned>(blocks), kThreads, smem, L.stream, ids, M * k, e,
+                    static_cast<int>(k), x, M, K, pair_w, b.offsets, b.sorted_pair, b.pos_of_pair, codes, scales, sorted_w,
+                    L.d_status);
+}
 
 cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
                            const PermuteBuffers& b) {
