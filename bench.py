@@ -870,8 +870,6 @@ def main():
         ctx.check_device_status()
         wbytes = w13c.numel() + w2c.numel() + (w13s.numel() + w2s.numel()) * 4 + 2 * M_DECODE * H * 2
         kern_ms = sum(v[0] for v in dst.values()) / dsteps
-        gu_d = dst["gate_up_gemm"][0] / max(dst["gate_up_gemm"][1], 1)
-        dn_d = dst["down_gemm"][0] / max(dst["down_gemm"][1], 1)
         result["decode"] = {
             "workload": "moe_ffn_decode_M256 (weights pre-quantized, two weight copies alternated: 1.2 GB > L2)",
             "ms_per_step": d_ms, "tokens_per_s": world * M_DECODE / (d_ms * 1e-3),
@@ -879,8 +877,6 @@ def main():
             "frac_hbm_measured": wbytes / (d_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
             "frac_hbm_nominal_8000": wbytes / (d_ms * 1e-3) / 1e9 / 8000.0,
             "stage_ms": {k: v[0] / dsteps for k, v in dst.items() if v[1]},
-            "gate_up_gbs": (w13c.numel() + w13s.numel() * 4) / (gu_d * 1e-3) / 1e9,
-            "down_gbs": (w2c.numel() + w2s.numel() * 4) / (dn_d * 1e-3) / 1e9,
             "sum_of_kernel_ms": kern_ms,
         }
 

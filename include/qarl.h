@@ -443,7 +443,8 @@ enum {
   QARL_STAGE_TBPO = 9,
   QARL_STAGE_ROUTER = 10,
   QARL_STAGE_BWD_ELEMENTWISE = 11,
-  QARL_NUM_STAGES = 12
+  QARL_STAGE_MOE_DECODE_LAYER = 12, /* decode-sized qarl_moe_fwd: gate_up + down + combine in one launch */
+  QARL_NUM_STAGES = 13
 };
 int qarl_profile_begin(qarl_ctx* ctx, int max_marks);
 int qarl_profile_end(qarl_ctx* ctx, double* stage_ms, int64_t* stage_launches);

@@ -49,9 +49,11 @@ int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages);
 
 /* The grouped FP8 GEMM has two kernels that produce the same bytes: the wide-tile one (128 token rows
  * x 256 weight rows per tile) and the swapped-operand one for decode-sized groups (128 weight rows x
- * at most 32 token rows).  The library picks by size; this call forces one (1 = wide, 2 = decode where
- * it applies: grouped calls with K <= 8192) or restores the automatic choice (0), so that a test can
- * run one input through both and compare.  Host side only, stored in the context. */
+ * at most 32 token rows); a decode-sized qarl_moe_fwd runs the latter once for the whole layer (gate_up
+ * tiles, down tiles and the k-sum in one launch).  The library picks by size; this call forces one
+ * (1 = wide, 2 = decode where it applies -- grouped calls with K <= 8192 --, one launch per projection
+ * and a separate combine) or restores the automatic choice (0), so that a test can run one input
+ * through each and compare.  Host side only, stored in the context. */
 int qarl_harness_set_gemm_path(qarl_ctx* ctx, int path);
 
 /* Roofline denominators measured with the library's own instructions (used by the benchmark; the

@@ -42,7 +42,7 @@ HARNESS_EXPORTS = ["qarl_harness_rmsnorm", "qarl_harness_wait_selftest", "qarl_h
                    "qarl_harness_stop_producer_after", "qarl_harness_fp8_mma_peak", "qarl_harness_read_stream",
                    "qarl_harness_set_gemm_path"]
 STAGES = ["quantize_weight", "quantize_act", "linear_gemm", "permute", "gate_up_gemm", "down_gemm",
-          "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise"]
+          "combine", "bwd_dx", "bwd_dw", "tbpo", "router", "bwd_elementwise", "moe_decode_layer"]
 
 
 class QarlError(RuntimeError):

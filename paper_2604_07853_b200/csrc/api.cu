@@ -17,7 +17,7 @@ using namespace qarl;
 
 // Workspace carve-up of qarl_moe_fwd; every slice starts on a 256-byte boundary.
 struct MoePlan {
-  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, a_codes, a_scales, h_codes, h_scales, contrib, total;
+  size_t chunk_hist, offsets, sorted_pair, pos_of_pair, sorted_w, a_codes, a_scales, h_codes, h_scales, contrib, sync, total;
 };
 MoePlan plan_moe(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   const size_t P = static_cast<size_t>(M * k);
@@ -38,6 +38,7 @@ MoePlan plan_moe(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   p.h_codes = take(P * I);
   p.h_scales = take(P * (I / kBlock) * sizeof(float));
   p.contrib = take(P * H * sizeof(uint16_t));
+  p.sync = take((E + 2) * sizeof(int32_t));  // counters of the one-launch decode layer
   p.total = o;
   return p;
 }
@@ -277,11 +278,13 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   uint8_t* a_codes = ws + pl.a_codes;
   float* a_scales = reinterpret_cast<float*>(ws + pl.a_scales);
   float* sorted_w = reinterpret_cast<float*>(ws + pl.sorted_w);
+  int32_t* layer_sync = reinterpret_cast<int32_t*>(ws + pl.sync);
+  const bool prep_small = moe_prep_small_applies(M, k, E);
   mark(ctx, L.stream, -1);
-  if (moe_prep_small_applies(M, k, E)) {
+  if (prep_small) {
     // decode-sized: grouping + quantization + scatter in one launch (timed as the quantize_act stage)
     if ((e = launch_moe_prep_small(L, ids, M, k, E, pb, static_cast<const uint16_t*>(x), H, wts, a_codes, a_scales,
-                                   sorted_w)) != cudaSuccess)
+                                   sorted_w, layer_sync, static_cast<int>(E + 2))) != cudaSuccess)
       return cuda_fail(ctx, e, "moe_prep");
     mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
   } else {
@@ -310,10 +313,6 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   g.h_codes = h_codes;
   g.h_scales = h_scales;
   g.h_bf16 = dbg ? static_cast<uint16_t*>(dbg->h_bf16) : nullptr;
-  int rc = run_gemm(ctx, L, g);
-  if (rc != QARL_OK) return rc;
-  mark(ctx, L.stream, QARL_STAGE_GATE_UP_GEMM);
-
   uint16_t* contrib = reinterpret_cast<uint16_t*>(ws + pl.contrib);
   GemmArgs d{};
   d.mode = kModeDown;
@@ -330,13 +329,31 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   d.out_f32 = dbg ? dbg->down_f32 : nullptr;
   d.sorted_pair = nullptr;  // contributions stay in sorted order (dense row blocks); the k-sum finds them by position
   d.pair_weights = sorted_w;
-  rc = run_gemm(ctx, L, d);
-  if (rc != QARL_OK) return rc;
-  mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);
 
-  if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out), pb.pos_of_pair)) != cudaSuccess)
-    return cuda_fail(ctx, e, "combine");
-  mark(ctx, L.stream, QARL_STAGE_COMBINE);
+  int rc;
+  if (prep_small && L.gemm_path == 0 && moe_decode_layer_applies(g, d)) {
+    // decode-sized: both projections and the k-sum in one launch (its counters were cleared by the
+    // grouping kernel)
+    CUresult cu = CUDA_SUCCESS;
+    e = launch_moe_decode_layer(L, ctx->encode, g, d, ids, pb.pos_of_pair, M, k, static_cast<uint16_t*>(out),
+                                layer_sync, &cu);
+    if (cu != CUDA_SUCCESS) {
+      snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+      return QARL_ERR_CUDA;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "moe decode layer launch");
+    mark(ctx, L.stream, QARL_STAGE_MOE_DECODE_LAYER);
+  } else {
+    rc = run_gemm(ctx, L, g);
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_GATE_UP_GEMM);
+    rc = run_gemm(ctx, L, d);
+    if (rc != QARL_OK) return rc;
+    mark(ctx, L.stream, QARL_STAGE_DOWN_GEMM);
+    if ((e = launch_combine(L, contrib, ids, M, k, H, E, static_cast<uint16_t*>(out), pb.pos_of_pair)) != cudaSuccess)
+      return cuda_fail(ctx, e, "combine");
+    mark(ctx, L.stream, QARL_STAGE_COMBINE);
+  }
 
   if (dbg) {
     if (dbg->expert_offsets &&

@@ -63,7 +63,7 @@ struct Launch {
   int64_t* launches;  // host counter
   unsigned long long wait_limit_ns = 0;  // bound of every device-side barrier wait (0: the default, 2 s)
   int stop_after_stages = -1;            // test harness only: FP8 GEMM producers stop after this many stages
-  int gemm_path = 0;                     // test harness only: 0 = automatic, 1 = wide-tile kernel, 2 = decode kernel
+  int gemm_path = 0;                     // test harness only: 0 = automatic, 1 = wide-tile kernel, 2 = decode kernel (one launch per projection)
 };
 
 // Launch with the programmatic-stream-serialization attribute (see pdl_wait above).
@@ -107,9 +107,11 @@ cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64
 
 // Decode-sized layers (M * k <= 2048): the grouping and the scattering activation quantization in one launch.
 bool moe_prep_small_applies(int64_t M, int64_t k, int64_t E);
+// `zero` / `zero_count`: int32 words the kernel clears (the counters of the one-launch layer that follows).
 cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
                                   const PermuteBuffers& b, const uint16_t* x, int64_t K, const float* pair_w,
-                                  uint8_t* codes, float* scales, float* sorted_w);
+                                  uint8_t* codes, float* scales, float* sorted_w, int32_t* zero = nullptr,
+                                  int zero_count = 0);
 
 // pos_of_pair == nullptr: contrib is indexed by flat pair id; else by pos_of_pair[pair] (sorted order)
 cudaError_t launch_combine(const Launch& L, const uint16_t* contrib, const int32_t* ids, int64_t M, int64_t k,
@@ -155,6 +157,14 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
 // launch_gemm picks it when gemm_decode_applies (L.gemm_path forces one or the other in tests).
 bool gemm_decode_applies(const GemmArgs& a);
 cudaError_t launch_gemm_decode(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err);
+// The decode-sized MoE layer after its grouping / quantization as ONE launch of that kernel: gate_up tiles,
+// down tiles (each waiting on a per-expert counter for the h rows it reads) and the k-sum of the
+// contributions.  `g` and `d` are the two projections as launch_gemm takes them (same groups);
+// `sync` is [2 + E] int32 that must be zero when the kernel starts.  Same bytes as the separate launches.
+bool moe_decode_layer_applies(const GemmArgs& g, const GemmArgs& d);
+cudaError_t launch_moe_decode_layer(const Launch& L, EncodeTiledFn encode, const GemmArgs& g, const GemmArgs& d,
+                                    const int32_t* ids, const int32_t* pos_of_pair, int64_t M, int64_t k, uint16_t* y,
+                                    int* sync, CUresult* cu_err);
 
 // ---- W4A16 (4-bit group-quantized weights, bf16 activations) --------------------------------
 // 4-bit weight formats (Sec. 2.2): unsigned integer codes with a zero point, or e2m1 floating point

@@ -18,6 +18,21 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kPairsPerWarp = 256;
 constexpr int kChunk = kWarps * kPairsPerWarp;  // 2048 pairs per CTA
 
+// Lanes of the warp whose id equals this lane's id (what match.any gives), from one ballot per id
+// bit: ten ballots cover every id below 1024 and -1 (a bad id, all ones in the low bits too: it is
+// told apart by the eleventh ballot).  match.any itself measured about a microsecond per call here,
+// which made the grouping the slowest kernel of a decode step.
+__device__ __forceinline__ uint32_t match_id(int e) {
+  uint32_t peers = 0xFFFFFFFFu;
+#pragma unroll
+  for (int b = 0; b < 11; ++b) {
+    const uint32_t bit = (static_cast<uint32_t>(e) >> (b == 10 ? 31 : b)) & 1u;
+    const uint32_t v = __ballot_sync(0xFFFFFFFFu, bit);
+    peers &= bit ? v : ~v;
+  }
+  return peers;
+}
+
 // Per-warp histogram of the warp's contiguous 256-pair slice into hist_w[0..E).  Lanes with
 // equal ids are found with match_any; the lowest such lane adds the group's size, so no
 // atomics are needed (one warp owns hist_w).
@@ -34,7 +49,7 @@ __device__ __forceinline__ void warp_histogram(const int32_t* __restrict__ ids, 
         e = -1;
       }
     }
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
     __syncwarp();
   }
@@ -54,7 +69,7 @@ __device__ __forceinline__ void warp_scatter(const int32_t* __restrict__ ids, in
       e = ids[p];
       if (e < 0 || e >= E) e = -1;
     }
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     int pos = -1;
     if (e >= 0) pos = cursor_w[e] + __popc(peers & lt);
     __syncwarp();
@@ -146,7 +161,7 @@ __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int3
 #pragma unroll
   for (int r = 0; r < kRounds; ++r) {
     const int e = my[r];
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
     __syncwarp();
   }
@@ -173,7 +188,7 @@ __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int3
 #pragma unroll
   for (int r = 0; r < kRounds; ++r) {
     const int e = my[r];
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     int pos = -1;
     if (e >= 0) pos = hist_w[e] + __popc(peers & lt);
     __syncwarp();
@@ -197,10 +212,12 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
     const int32_t* __restrict__ ids, int64_t P, int E, int fanout, const uint16_t* __restrict__ x, int64_t M, int64_t K,
     const float* __restrict__ pair_w, int32_t* __restrict__ offsets, int32_t* __restrict__ sorted_pair,
     int32_t* __restrict__ pos_of_pair, uint8_t* __restrict__ codes, float* __restrict__ scales,
-    float* __restrict__ sorted_w, int* status) {
+    float* __restrict__ sorted_w, int32_t* __restrict__ zero, int zero_count, int* status) {
   extern __shared__ int32_t sm[];
   pdl_trigger();
   pdl_wait();
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < zero_count; i += kThreads) zero[i] = 0;
   int32_t* whist = sm;                 // [kWarps][E]
   int32_t* total = sm + kWarps * E;    // [E]
   int32_t* scratch = total + E;        // [33]
@@ -245,7 +262,7 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
 #pragma unroll
   for (int r = 0; r < kRounds; ++r) {
     const int e = my[r];
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     if (e >= 0 && (__ffs(peers) - 1) == lane) hist_w[e] += __popc(peers);
     __syncwarp();
   }
@@ -272,7 +289,7 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
 #pragma unroll
   for (int r = 0; r < kRounds; ++r) {
     const int e = my[r];
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, e);
+    const uint32_t peers = match_id(e);
     int pos = -1;
     if (e >= 0) pos = hist_w[e] + __popc(peers & lt);
     __syncwarp();
@@ -410,7 +427,7 @@ bool moe_prep_small_applies(int64_t M, int64_t k, int64_t E) { return M * k <= k
 
 cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,
                                   const PermuteBuffers& b, const uint16_t* x, int64_t K, const float* pair_w,
-                                  uint8_t* codes, float* scales, float* sorted_w) {
+                                  uint8_t* codes, float* scales, float* sorted_w, int32_t* zero, int zero_count) {
   const int e = static_cast<int>(E);
   const size_t smem = (static_cast<size_t>(kWarps) * e + e + 33 + kChunk) * sizeof(int32_t);
   if (smem > 48 * 1024) {
@@ -423,7 +440,7 @@ cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M
   ++*L.launches;
   return launch_pdl(moe_prep_small_kernel, static_cast<unsigned>(blocks), kThreads, smem, L.stream, ids, M * k, e,
                     static_cast<int>(k), x, M, K, pair_w, b.offsets, b.sorted_pair, b.pos_of_pair, codes, scales, sorted_w,
-                    L.d_status);
+                    zero, zero_count, L.d_status);
 }
 
 cudaError_t launch_permute(const Launch& L, const int32_t* ids, int64_t M, int64_t k, int64_t E,

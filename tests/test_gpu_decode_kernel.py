@@ -1,7 +1,9 @@
-"""The grouped FP8 GEMM has a wide-tile kernel and a swapped-operand kernel for decode-sized groups.
-Both must give the same bytes for every row (the fixed K-reduction order of App. C holds across
-kernels, not only across batch sizes): one input goes through both, forced by the harness switch,
-and every stage the layer exposes is compared bit for bit."""
+"""The grouped FP8 GEMM has a wide-tile kernel and a swapped-operand kernel for decode-sized groups,
+and a decode-sized layer runs both projections and the k-sum as one launch of the latter.
+All must give the same bytes for every row (the fixed K-reduction order of App. C holds across
+kernels, not only across batch sizes): one input goes through each, forced by the harness switch
+(0 = automatic: the one-launch layer where it applies), and every stage the layer exposes is
+compared bit for bit."""
 import numpy as np
 import pytest
 import torch
@@ -37,14 +39,17 @@ def _layer(ctx, c, path, debug=True):
 def test_decode_kernel_equals_wide_kernel_stage_by_stage(ctx, m, h, i, e, k):
     c = inputs.moe_case(21, m, h=h, i=i, e=e, k=k)
     out_w, d_w = _layer(ctx, c, 1)
-    out_d, d_d = _layer(ctx, c, 2)
     P = m * k
-    for key in ("expert_offsets", "sorted_pair", "gate_up", "h", "h_codes", "h_scales", "down_f32"):
-        a, b = d_w[key], d_d[key]
-        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), key
-    assert torch.equal(out_w, out_d)
+    for path in (2, 0):
+        out_d, d_d = _layer(ctx, c, path)
+        for key in ("expert_offsets", "sorted_pair", "gate_up", "h", "h_codes", "h_scales", "down_f32"):
+            a, b = d_w[key], d_d[key]
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), (path, key)
+        assert torch.equal(out_w, out_d), path
     # and without the debug dumps
-    assert torch.equal(_layer(ctx, c, 1, debug=False), _layer(ctx, c, 2, debug=False))
+    wide = _layer(ctx, c, 1, debug=False)
+    assert torch.equal(wide, _layer(ctx, c, 2, debug=False))
+    assert torch.equal(wide, _layer(ctx, c, 0, debug=False))
     assert P > 0
 
 
@@ -63,3 +68,19 @@ def test_skewed_groups_through_the_decode_kernel(ctx):
     out_d, d_d = _layer(ctx, c, 2)
     assert torch.equal(d_w["h_codes"], d_d["h_codes"]) and torch.equal(d_w["down_f32"].view(torch.int32), d_d["down_f32"].view(torch.int32))
     assert torch.equal(out_w, out_d)
+
+
+@pytest.mark.parametrize("m,e,k,zipf", [(40, 64, 8, 0.0), (8, 128, 8, 0.0), (100, 16, 4, 1.1), (256, 128, 8, 1.1),
+                                         (3, 128, 8, 0.0), (200, 40, 5, 1.5)])
+def test_one_launch_layer_repeated_and_skewed(ctx, m, e, k, zipf):
+    """The one-launch layer on shapes with many empty experts, experts of several 32-row chunks and
+    fewer experts than the distance between an expert's two projections in its tile list; three
+    calls in a row (its counters are cleared by the grouping kernel of each call)."""
+    c = inputs.moe_case(77, m, h=512, i=256, e=e, k=k, zipf_s=zipf) if zipf else inputs.moe_case(77, m, h=512, i=256, e=e, k=k)
+    ref, d_ref = _layer(ctx, c, 2)
+    for _ in range(3):
+        out, d = _layer(ctx, c, 0)
+        assert torch.equal(d_ref["h_codes"], d["h_codes"]) and torch.equal(d_ref["h_scales"], d["h_scales"])
+        assert torch.equal(d_ref["down_f32"].view(torch.int32), d["down_f32"].view(torch.int32))
+        assert torch.equal(ref, out)
+        assert torch.equal(ref, _layer(ctx, c, 0, debug=False))
