@@ -29,9 +29,9 @@
 // list holds the gate_up tiles and the down tiles of every expert, the down tiles of expert e
 // kDepSlots experts after its gate_up tiles, so the weight stream never stops between the two
 // projections; a down tile starts once a per-expert counter says the h rows it reads are written
-// (release by the writers, acquire + proxy fence by the readers, every spin bounded); when a
-// CTA has finished its tiles it joins a grid-wide counter and the CTAs then sum every token's k
-// contributions in ascending expert id (the combine), reading them from L2.  Tile arithmetic,
+// (release by the writers, acquire + proxy fence by the readers, every spin bounded); a CTA that
+// has finished its tiles sums its share of the tokens -- a token's k contributions in ascending
+// expert id (the combine), read from L2 -- each as soon as the down tiles of its experts are done.  Tile arithmetic,
 // promotion chain and epilogues are the ones of the separate launches: the bytes are the same.
 #include <algorithm>
 #include <atomic>
@@ -70,7 +70,6 @@ constexpr uint32_t kOutBytes = NT * kOutRowBytes;
 constexpr int kModeLayer = 3;     // gate_up tiles + down tiles + combine in one launch (this file only)
 constexpr int kDepSlots = 32;     // the down tiles of expert e are listed with the gate_up tiles of expert e + kDepSlots
 constexpr int kMaxTopK = 32;
-constexpr int kOrderSlots = 16;   // combine: tokens of a CTA whose summation order is worked out ahead of the grid-wide wait
 constexpr int kSchedSlots = 4;    // layer: tile numbers the producer has drawn and the other roles have not yet read
 
 // Operands of one projection: token-side scales [rows_total, KB], weight scales [E, N/128, KB].
@@ -102,8 +101,8 @@ struct DecodeParams {
   const int32_t* pos_of_pair;  // [M * k]
   uint16_t* y;                 // [M, H]
   int M, k;
-  int* sync;                   // [0]: CTAs that finished their tiles; [1 + e]: finished gate_up tiles of expert e;
-                               // [1 + E]: tiles handed out so far (all zero on entry)
+  int* sync;                   // [0]: tiles handed out so far; [1 + e]: finished gate_up tiles of expert e;
+                               // [1 + E + e]: finished down tiles of expert e (all zero on entry)
   int* status;
   unsigned long long wait_limit_ns;
   int stop_after_stages;
@@ -132,7 +131,7 @@ struct __align__(8) SmemTail {
   int abort_flag;
   int ready_flag;
   int peek_T;
-  int32_t order[kOrderSlots][kMaxTopK];  // combine: contribution row of the rank-th smallest expert id of a token
+  int32_t order[1][kMaxTopK];  // combine: contribution row of the rank-th smallest expert id of a token
   int32_t off[kMaxExperts + 1];
   int32_t prefix[kMaxExperts + kDepSlots + 1];
 };
@@ -409,7 +408,7 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             return t < total_tiles ? t : -1;
           } else {
             if (!wait_or_abort(&s->sched_empty[sslot], sphase ^ 1, s, p)) { ok = false; return -1; }
-            int t = atomicAdd(p.sync + 1 + p.E, 1);
+            int t = atomicAdd(p.sync, 1);
             if (t >= total_tiles) t = -1;
             *reinterpret_cast<volatile int*>(&s->sched_T[sslot]) = t;
             mbar_arrive(&s->sched_full[sslot]);  // release: the number is visible to whoever sees the phase flip
@@ -754,56 +753,52 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&s->out_empty);  // the staging tile may be overwritten
-      if (kLayer && c.mode == kModeGateUp) {
-        // Other CTAs read these h codes by TMA and the scales by plain loads once the expert's counter
-        // says so: every writer orders its stores (both proxies), then one thread bumps the counter.
+      if (kLayer) {
+        // Other CTAs read what this tile wrote once the expert's counter says so -- the h codes by TMA
+        // and their scales by plain loads (gate_up), the contribution rows in the k-sum (down): every
+        // writer orders its stores (both proxies), then one thread bumps the counter.
         __threadfence();
-        fence_proxy_async_global();
+        if (c.mode == kModeGateUp) fence_proxy_async_global();
         named_bar_sync(4, kEpiThreads);
-        if (et == 0) red_release_gpu_add(p.sync + 1 + c.e, 1);
+        if (et == 0) red_release_gpu_add(p.sync + (c.mode == kModeGateUp ? 1 : 1 + p.E) + c.e, 1);
       }
     }
 
     if (kLayer) {
-      // ---- the combine: every CTA has to be done with its tiles first --------------------------
-      __threadfence();
-      ok = named_bar_all(4, kEpiThreads, ok);
-      if (et == 0) red_release_gpu_add(p.sync, 1);  // also after an abort: the other CTAs need not wait for the limit
+      // ---- the combine --------------------------------------------------------------------------
       // out[t] = bf16( sum of the token's k bf16 contributions in ascending expert id, from 0.0f ).
-      // CTA b sums tokens b, b + grid, ...  The order of a token's rows depends on inputs of the launch
-      // only: warp 0 works it out for the first tokens while the other CTAs are still finishing.
+      // CTA b sums tokens b, b + grid, ... as soon as the down tiles of the token's k experts are all
+      // finished (their counters), so a CTA that runs out of tiles early sums while others still stream.
+      ok = named_bar_all(4, kEpiThreads, ok);
       const int k = p.k, H = p.pj[1].N;
       const int64_t P = static_cast<int64_t>(p.M) * k;
-      auto rank_rows = [&](int64_t t, int32_t* dst) {  // whole warp; lane l < k holds the token's l-th pair
-        const int mine = lane < k ? p.ids[t * k + lane] : 0x7FFFFFFF;
-        const int64_t pos = lane < k ? p.pos_of_pair[t * k + lane] : 0;
-        int rank = 0;
-        bool repeated = false;
-        for (int jj = 0; jj < k; ++jj) {
-          const int other = __shfl_sync(0xFFFFFFFFu, mine, jj);
-          if (other < mine || (other == mine && jj < lane)) ++rank;
-          if (other == mine && jj != lane) repeated = true;
-        }
-        if (lane < k) {
-          if (repeated) set_status(p.status, QARL_ERR_BAD_EXPERT_ID);  // expert repeated in a token
-          dst[rank] = static_cast<int32_t>(min(max(pos, int64_t(0)), P - 1));
-        }
-      };
-      if (ew == 0) {
-        int i = 0;
-        for (int64_t t = blockIdx.x; t < p.M && i < kOrderSlots - 1; t += gridDim.x, ++i) rank_rows(t, s->order[i]);
-      }
-      if (ok) ok = counter_wait_or_abort(p.sync, static_cast<int>(gridDim.x), s, p);
-      ok = named_bar_all(4, kEpiThreads, ok);  // also publishes order[] to the four warps
+      const int* dcount = p.sync + 1 + p.E;
       if (ok) {
-        int i = 0;
-        for (int64_t t = blockIdx.x; t < p.M; t += gridDim.x, ++i) {
-          const int32_t* ord = s->order[min(i, kOrderSlots - 1)];
-          if (i >= kOrderSlots - 1) {  // beyond the slots filled ahead: the last slot, filled per token
-            named_bar_sync(4, kEpiThreads);
-            if (ew == 0) rank_rows(t, s->order[kOrderSlots - 1]);
-            named_bar_sync(4, kEpiThreads);
+        for (int64_t t = blockIdx.x; t < p.M; t += gridDim.x) {
+          // lane l < k of every warp holds the token's l-th pair: its rank among the token's expert ids
+          // gives the position of its row in the sum; the lane also waits for its expert's down tiles
+          const int mine = lane < k ? p.ids[t * k + lane] : 0x7FFFFFFF;
+          const int64_t pos = lane < k ? p.pos_of_pair[t * k + lane] : 0;
+          int rank = 0;
+          bool repeated = false;
+          for (int jj = 0; jj < k; ++jj) {
+            const int other = __shfl_sync(0xFFFFFFFFu, mine, jj);
+            if (other < mine || (other == mine && jj < lane)) ++rank;
+            if (other == mine && jj != lane) repeated = true;
           }
+          named_bar_sync(4, kEpiThreads);  // the previous token's readers of order[] are done
+          bool ready = true;
+          if (lane < k) {
+            if (ew == 0) {
+              if (repeated) set_status(p.status, QARL_ERR_BAD_EXPERT_ID);  // expert repeated in a token
+              s->order[0][rank] = static_cast<int32_t>(min(max(pos, int64_t(0)), P - 1));
+            }
+            if (mine >= 0 && mine < p.E)  // (a bad id has no row of its own: nothing to wait for)
+              ready = counter_wait_or_abort(dcount + mine, chunks_of(s->off, mine) * p.pj[1].n_pairs, s, p);
+          }
+          ok = named_bar_all(4, kEpiThreads, ready);  // every warp has acquired; order[] is published
+          if (!ok) break;
+          const int32_t* ord = s->order[0];
           for (int col = et * 8; col < H; col += kEpiThreads * 8) {
             float acc[8];
 #pragma unroll

@@ -208,7 +208,12 @@ __global__ void __launch_bounds__(kThreads) permute_single_cta_kernel(const int3
 // codes, scales and combine weight to the token's k expert-sorted rows.  CTA 0 also publishes offsets,
 // sorted_pair and pos_of_pair.  One launch and one dependency instead of two of each; the loads of
 // the activations are issued before the grouping so that their latency hides behind it.
-__global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
+// 16 warps of 128 pairs: four rounds per pass (the grouping is a chain of short dependent steps, so
+// more, shorter warps finish it sooner)
+constexpr int kPrepThreads = 512;
+constexpr int kPrepWarps = kPrepThreads / 32;
+constexpr int kPrepPairsPerWarp = kChunk / kPrepWarps;
+__global__ void __launch_bounds__(kPrepThreads) moe_prep_small_kernel(
     const int32_t* __restrict__ ids, int64_t P, int E, int fanout, const uint16_t* __restrict__ x, int64_t M, int64_t K,
     const float* __restrict__ pair_w, int32_t* __restrict__ offsets, int32_t* __restrict__ sorted_pair,
     int32_t* __restrict__ pos_of_pair, uint8_t* __restrict__ codes, float* __restrict__ scales,
@@ -217,9 +222,9 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
   pdl_trigger();
   pdl_wait();
   if (blockIdx.x == 0)
-    for (int i = threadIdx.x; i < zero_count; i += kThreads) zero[i] = 0;
-  int32_t* whist = sm;                 // [kWarps][E]
-  int32_t* total = sm + kWarps * E;    // [E]
+    for (int i = threadIdx.x; i < zero_count; i += kPrepThreads) zero[i] = 0;
+  int32_t* whist = sm;                 // [kPrepWarps][E]
+  int32_t* total = sm + kPrepWarps * E;    // [E]
   int32_t* scratch = total + E;        // [33]
   int32_t* spos = scratch + 33;        // [kChunk] sorted position of every pair (-1: bad id)
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
@@ -240,8 +245,8 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
   }
 
   // ---- the grouping (as permute_single_cta_kernel), positions kept in shared memory
-  constexpr int kRounds = kPairsPerWarp / 32;
-  const int64_t p0 = static_cast<int64_t>(wid) * kPairsPerWarp + lane;
+  constexpr int kRounds = kPrepPairsPerWarp / 32;
+  const int64_t p0 = static_cast<int64_t>(wid) * kPrepPairsPerWarp + lane;
   int my[kRounds];
   bool bad = false;
 #pragma unroll
@@ -255,8 +260,8 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
     my[r] = e;
   }
   if (bad && publish) set_status(status, QARL_ERR_BAD_EXPERT_ID);
-  for (int i = tid; i < kWarps * E; i += kThreads) whist[i] = 0;
-  for (int i = tid; i < kChunk; i += kThreads) spos[i] = -1;
+  for (int i = tid; i < kPrepWarps * E; i += kPrepThreads) whist[i] = 0;
+  for (int i = tid; i < kChunk; i += kPrepThreads) spos[i] = -1;
   __syncthreads();
   int32_t* hist_w = whist + wid * E;
 #pragma unroll
@@ -267,17 +272,17 @@ __global__ void __launch_bounds__(kThreads) moe_prep_small_kernel(
     __syncwarp();
   }
   __syncthreads();
-  for (int e = tid; e < E; e += kThreads) {
+  for (int e = tid; e < E; e += kPrepThreads) {
     int s = 0;
-    for (int w = 0; w < kWarps; ++w) s += whist[w * E + e];
+    for (int w = 0; w < kPrepWarps; ++w) s += whist[w * E + e];
     total[e] = s;
   }
   __syncthreads();
   const int all = block_exclusive_scan(total, E, scratch);
-  for (int e = tid; e < E; e += kThreads) {
+  for (int e = tid; e < E; e += kPrepThreads) {
     int run = total[e];
     if (publish) offsets[e] = run;
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < kPrepWarps; ++w) {
       const int c = whist[w * E + e];
       whist[w * E + e] = run;
       run += c;
@@ -429,16 +434,16 @@ cudaError_t launch_moe_prep_small(const Launch& L, const int32_t* ids, int64_t M
                                   const PermuteBuffers& b, const uint16_t* x, int64_t K, const float* pair_w,
                                   uint8_t* codes, float* scales, float* sorted_w, int32_t* zero, int zero_count) {
   const int e = static_cast<int>(E);
-  const size_t smem = (static_cast<size_t>(kWarps) * e + e + 33 + kChunk) * sizeof(int32_t);
+  const size_t smem = (static_cast<size_t>(kPrepWarps) * e + e + 33 + kChunk) * sizeof(int32_t);
   if (smem > 48 * 1024) {
     cudaError_t err = cudaFuncSetAttribute(moe_prep_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            static_cast<int>(smem));
     if (err != cudaSuccess) return err;
   }
   const int64_t groups = M * (K / kBlock);
-  const int64_t blocks = std::max<int64_t>(1, (groups * 8 + kThreads - 1) / kThreads);
+  const int64_t blocks = std::max<int64_t>(1, (groups * 8 + kPrepThreads - 1) / kPrepThreads);
   ++*L.launches;
-  return launch_pdl(moe_prep_small_kernel, static_cast<unsigned>(blocks), kThreads, smem, L.stream, ids, M * k, e,
+  return launch_pdl(moe_prep_small_kernel, static_cast<unsigned>(blocks), kPrepThreads, smem, L.stream, ids, M * k, e,
                     static_cast<int>(k), x, M, K, pair_w, b.offsets, b.sorted_pair, b.pos_of_pair, codes, scales, sorted_w,
                     zero, zero_count, L.d_status);
 }
