@@ -196,6 +196,10 @@ struct GemmW4Args {
   const float* pair_weights;
 };
 cudaError_t launch_gemm_w4a16(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err);
+// The swapped-operand kernel for decode-sized row groups (same bytes out; see gemm_w4a16_decode_sm100.cu);
+// launch_gemm_w4a16 picks it when gemm_w4a16_decode_applies (L.gemm_path forces one or the other in tests).
+bool gemm_w4a16_decode_applies(const GemmW4Args& a);
+cudaError_t launch_gemm_w4a16_decode(const Launch& L, EncodeTiledFn encode, const GemmW4Args& a, CUresult* cu_err);
 
 // ---- dense bf16 GEMM (full-precision backward): C[i,j] = sum_c A(i,c) B(j,c) ---------------------
 struct GemmBf16Args {
