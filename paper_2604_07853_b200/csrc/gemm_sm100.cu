@@ -51,7 +51,7 @@ constexpr int kAccBufs = 2;       // TMEM accumulators of 256 columns
 constexpr int kPromoWarps = 8;    // warps 0-7
 constexpr int kEpiWarps = 4;      // warps 8-11
 constexpr int kTmaWarp = 12;
-constexpr int kMmaWarp = 13;      // warps 14, 15 idle (setmaxnreg works on whole warpgroups)
+constexpr int kMmaWarp = 13;      // and 14: two issuers; warp 15 idle (setmaxnreg works on whole warpgroups)
 constexpr int kThreads = 16 * 32;
 // register re-allocation: 256 x 208 + 128 x 56 + 128 x 40 = 65536 = 512 x 128 (the launch allocation)
 constexpr int kPromoRegs = 208;
@@ -96,7 +96,7 @@ struct __align__(8) SmemTail {
   uint64_t tmem_empty[kAccBufs];
   uint64_t out_full;
   uint64_t out_empty;
-  uint64_t teardown;
+  uint64_t teardown[2];
   uint32_t tmem_addr;
   int abort_flag;
   int32_t off[kMaxExperts + 1];
@@ -194,7 +194,8 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     }
     mbar_init(&s->out_full, kPromoWarps);
     mbar_init(&s->out_empty, kEpiWarps);
-    mbar_init(&s->teardown, 1);
+    mbar_init(&s->teardown[0], 1);
+    mbar_init(&s->teardown[1], 1);
     s->abort_flag = 0;
     fence_mbar_init();
   }
@@ -329,37 +330,42 @@ gemm_blockscaled_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             if (armed & (1u << i)) mbar_wait_bounded(&s->full[i], (armed_parity >> i) & 1u, 20000000ull);
         }
       }
-    } else if (warp == kMmaWarp) {
-      // =============================== MMA issuer =======================================
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+      // =============================== MMA issuers ======================================
+      // Two threads, one per TMEM accumulator: K-block n of this CTA (counted across its tiles) is
+      // issued by thread n % 2 into accumulator n % 2.  Every K-block starts a fresh accumulator, so
+      // the two never write the same columns, and the fixed cost per K-block of one thread waiting,
+      // issuing and committing (about as long as the MMAs themselves take) is spread over two.
       if (lane == 0) {
         constexpr uint32_t idesc = umma_idesc_e4m3_f32(BM, BN);
-        int stage = 0, ks = 0;
-        uint32_t phase = 0, acc_phase = 0;
+        const int me = warp - kMmaWarp;
+        uint32_t n = 0;  // K-blocks of this CTA so far
         bool ok = true;
         for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
-          for (int kb = 0; kb < KB; ++kb) {
+          for (int kb = 0; kb < KB; ++kb, ++n) {
+            if (static_cast<int>(n & 1u) != me) continue;
+            const uint32_t stage = n % kStages, phase = (n / kStages) & 1u;
+            const uint32_t ks = n & 1u, acc_phase = (n >> 1) & 1u;
             if (!wait_or_abort(&s->tmem_empty[ks], acc_phase ^ 1, s, p)) { ok = false; break; }
             if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
             const uint64_t a_desc = umma_desc_k_sw128(a_addr);
             const uint64_t b_desc = umma_desc_k_sw128(a_addr + kABytes);
-            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ks) * BN;
+            const uint32_t d_tmem = tmem_base + ks * BN;
 #pragma unroll
             for (int k4 = 0; k4 < BK / 32; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
               umma_f8(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
             umma_commit(&s->empty[stage]);
             umma_commit(&s->tmem_full[ks]);
-            if (++stage == kStages) { stage = 0; phase ^= 1; }
-            if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
           }
         }
         // Nothing of this CTA's tensor work may be in flight when its TMEM and shared memory
         // go away: after a normal run every MMA has been consumed already; after an abort
         // some may still be executing, so wait (bounded) for all of them.
         if (!ok) {
-          umma_commit(&s->teardown);
-          mbar_wait_bounded(&s->teardown, 0, 20000000ull);
+          umma_commit(&s->teardown[me]);
+          mbar_wait_bounded(&s->teardown[me], 0, 20000000ull);
         }
       }
     }
