@@ -22,7 +22,7 @@
 // the multiplication by the pair's combine weight -- and transpose the tile through shared memory),
 // warps 4-7 epilogue (a warp per token row while the promotion warps run the next tile: gate_up =
 // SwiGLU, 1x128 amax / scale / e4m3 codes; down / linear = whole-row stores), warp 8 TMA producer,
-// warp 9 MMA issuer.
+// warps 9 and 10 MMA issuers (one per weight block of the pair).
 // Every barrier wait is bounded as in the wide kernel; an expired wait aborts the CTA cleanly.
 //
 // The whole decode-sized MoE layer also runs as ONE launch of this kernel (kModeLayer): the tile
@@ -52,8 +52,8 @@ constexpr int kStages = 5;         // 36 KB each: 180 KB of loads in flight per 
 constexpr int kAccBufs = 8;       // TMEM accumulators of 2 x NT columns
 constexpr int kPromoWarps = 4;     // warps 0-3 (warpgroup 0)
 constexpr int kEpiWarps = 4;       // warps 4-7 (warpgroup 1)
-constexpr int kTmaWarp = 8;        // warpgroup 2: warps 10, 11 idle (setmaxnreg works on whole warpgroups)
-constexpr int kMmaWarp = 9;
+constexpr int kTmaWarp = 8;        // warpgroup 2: warp 11 idle (setmaxnreg works on whole warpgroups)
+constexpr int kMmaWarp = 9;         // and 10: one issuer per weight block of the pair
 constexpr int kThreads = 12 * 32;
 // register re-allocation: 128 x (232 + 128 + 96) = 58368 <= 384 x 168 (the launch allocation)
 constexpr int kPromoRegs = 232;
@@ -123,7 +123,7 @@ struct __align__(8) SmemTail {
   uint64_t tmem_empty[kAccBufs];
   uint64_t out_full;
   uint64_t out_empty;
-  uint64_t teardown;
+  uint64_t teardown[2];
   uint64_t sched_full[kSchedSlots];
   uint64_t sched_empty[kSchedSlots];
   int sched_T[kSchedSlots];
@@ -325,16 +325,17 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&s->full[i], 1);
-      mbar_init(&s->empty[i], 1);
+      mbar_init(&s->empty[i], 2);      // the commits of the two MMA issuers
     }
     for (int i = 0; i < kAccBufs; ++i) {
-      mbar_init(&s->tmem_full[i], 1);
+      mbar_init(&s->tmem_full[i], 2);  // the two MMA issuers
       mbar_init(&s->tmem_empty[i], kPromoWarps);
     }
-    mbar_init(&s->teardown, 1);
+    mbar_init(&s->teardown[0], 1);
+    mbar_init(&s->teardown[1], 1);
     for (int i = 0; i < kSchedSlots; ++i) {
       mbar_init(&s->sched_full[i], 1);
-      mbar_init(&s->sched_empty[i], 1 + kPromoWarps + kEpiWarps);
+      mbar_init(&s->sched_empty[i], 2 + kPromoWarps + kEpiWarps);
     }
     mbar_init(&s->out_full, kPromoWarps);
     mbar_init(&s->out_empty, kEpiWarps);
@@ -448,9 +449,13 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (armed & (1u << i)) mbar_wait_bounded(&s->full[i], (armed_parity >> i) & 1u, 20000000ull);
         }
       }
-    } else if (warp == kMmaWarp) {
-      // =============================== MMA issuer =========================================
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+      // =============================== MMA issuers ========================================
+      // One thread per weight block of the pair: each feeds its own 32 columns of the accumulator, so the
+      // two never write the same TMEM columns, and the fixed cost per K-block of waiting, issuing and
+      // committing (which holds the shared-memory stage, i.e. bytes in flight from HBM) is halved.
       if (lane == 0) {
+        const int half = warp - kMmaWarp;
         constexpr uint32_t idesc = umma_idesc_e4m3_f32(BW, NT);
         int stage = 0, ks = 0, cur = 0, sslot = 0;
         uint32_t phase = 0, acc_phase = 0, sphase = 0;
@@ -475,15 +480,12 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (!wait_or_abort(&s->full[stage], phase, s, p)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(stage) * kStageBytes);
-            const uint64_t w_lo = umma_desc_k_sw128(a_addr), w_hi = umma_desc_k_sw128(a_addr + kABytes / 2);
+            const uint64_t w_desc = umma_desc_k_sw128(a_addr + half * (kABytes / 2));
             const uint64_t x_desc = umma_desc_k_sw128(a_addr + kABytes);
-            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ks) * (2 * NT);
+            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ks) * (2 * NT) + static_cast<uint32_t>(half) * NT;
 #pragma unroll
             for (int k4 = 0; k4 < BK / 32; ++k4)  // +32 bytes of K = +2 in the 16-byte address field
-              umma_f8(d_tmem, w_lo + 2 * k4, x_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
-#pragma unroll
-            for (int k4 = 0; k4 < BK / 32; ++k4)
-              umma_f8(d_tmem + NT, w_hi + 2 * k4, x_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
+              umma_f8(d_tmem, w_desc + 2 * k4, x_desc + 2 * k4, idesc, k4 > 0 ? 1u : 0u);
             umma_commit(&s->empty[stage]);
             umma_commit(&s->tmem_full[ks]);
             if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -491,8 +493,8 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           }
         }
         if (!ok) {  // after an abort MMAs may still be executing: wait (bounded) before TMEM goes away
-          umma_commit(&s->teardown);
-          mbar_wait_bounded(&s->teardown, 0, 20000000ull);
+          umma_commit(&s->teardown[half]);
+          mbar_wait_bounded(&s->teardown[half], 0, 20000000ull);
         }
       }
     }
