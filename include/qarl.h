@@ -165,7 +165,13 @@ typedef struct {
  * out: out_bf16 [M, H].
  * Limits: 1 <= k <= 32, 1 <= E <= 1024, M*k < 2^31.
  * workspace: at least qarl_moe_workspace_bytes(M, H, I, E, k) bytes, 256-byte aligned; the
- * call clears what must start at zero; calls sharing a workspace must not overlap. */
+ * call clears what must start at zero; calls sharing a workspace must not overlap.
+ * Launches: training-sized batches run the steps as separate kernels (grouping, activation
+ * quantization, gate_up, down, combine).  Decode-sized batches (M*k <= 2048 and M*k <= 32*E) run
+ * two: the grouping with the quantization, then the whole layer as one persistent kernel whose
+ * CTAs publish finished tiles to one another through counters in the workspace (every wait on
+ * them is bounded like the pipeline waits; expiry gives QARL_ERR_DEVICE_TIMEOUT).  The bytes of
+ * out_bf16 and of every dump are the same on both routes. */
 size_t qarl_moe_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k);
 int qarl_moe_fwd(qarl_ctx* ctx, const void* x_bf16, const int32_t* topk_ids,
                  const float* topk_weights, int64_t M, int64_t H, int64_t I, int64_t E,
