@@ -193,8 +193,10 @@ __device__ __forceinline__ void red_release_gpu_add(int* p, int v) {
 // orders this thread's generic-proxy accesses to global memory with its TMA (async-proxy) accesses
 __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
-// Bounded wait until *ctr >= target (acquire).  All CTAs of the launch are resident (at most one per
-// SM), and a counter only waits on tiles listed earlier, so the wait ends; the bound is for a broken run.
+// Bounded wait until *ctr >= target (acquire).  A counter only waits on tiles listed earlier, and a tile
+// is only ever held by a CTA that is running (tiles are drawn, not pre-assigned: a CTA of the grid that
+// has not been scheduled yet, e.g. behind another stream's kernel, holds none), so the wait ends whatever
+// part of the grid is resident; the bound is for a broken run.
 __device__ __forceinline__ bool counter_wait_or_abort(const int* ctr, int target, SmemTail* s, const DecodeParams& p) {
   if (ld_acquire_gpu(ctr) >= target) return true;
   const uint64_t t0 = globaltimer_ns();
