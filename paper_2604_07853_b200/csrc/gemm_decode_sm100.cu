@@ -891,8 +891,11 @@ int early_prefetch_tiles(const Launch& L, int kblocks) {
 }  // namespace
 
 bool gemm_decode_applies(const GemmArgs& a) {
-  // grouped calls whose groups average at most 32 rows (decode batches), K within the scale slab
-  return a.offsets != nullptr && a.rows_total <= static_cast<int64_t>(NT) * a.E && a.K / BK <= kMaxKB;
+  // grouped calls whose groups average at most 32 rows (decode batches) and dense calls of at most 64 rows
+  // (a decode step's projections: more CTAs stream the weight, none multiplies padding); K within the scale slab
+  if (a.K / BK > kMaxKB) return false;
+  if (a.offsets == nullptr) return a.E == 1 && a.rows_total <= 2 * NT;
+  return a.rows_total <= static_cast<int64_t>(NT) * a.E;
 }
 
 cudaError_t launch_gemm_decode(const Launch& L, EncodeTiledFn encode, const GemmArgs& a, CUresult* cu_err) {

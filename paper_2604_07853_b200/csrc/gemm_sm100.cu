@@ -664,7 +664,7 @@ cudaError_t launch_gemm(const Launch& L, EncodeTiledFn encode, const GemmArgs& a
   *cu_err = CUDA_SUCCESS;
   if (a.rows_total == 0) return cudaSuccess;
   // decode-sized groups: the swapped-operand kernel (bitwise the same rows, bound by the weight stream)
-  if (L.gemm_path == 2 ? (a.offsets != nullptr && a.K / BK <= 64) : (L.gemm_path == 0 && gemm_decode_applies(a)))
+  if (L.gemm_path == 2 ? ((a.offsets != nullptr || a.E == 1) && a.K / BK <= 64) : (L.gemm_path == 0 && gemm_decode_applies(a)))
     return launch_gemm_decode(L, encode, a, cu_err);
   CUtensorMap ta, tb;
   CUresult r = make_tmap(encode, &ta, a.a_codes, static_cast<uint64_t>(a.rows_total), static_cast<uint64_t>(a.K));
