@@ -84,3 +84,15 @@ def test_one_launch_layer_repeated_and_skewed(ctx, m, e, k, zipf):
         assert torch.equal(d_ref["down_f32"].view(torch.int32), d["down_f32"].view(torch.int32))
         assert torch.equal(ref, out)
         assert torch.equal(ref, _layer(ctx, c, 0, debug=False))
+
+
+@pytest.mark.parametrize("m,h,i,e,k", [(24, 4096, 1536, 16, 4), (40, 1024, 128, 300, 6), (17, 8192, 256, 4, 2)])
+def test_one_launch_layer_long_k_and_many_experts(ctx, m, h, i, e, k):
+    """K up to the scale slab's limit (64 K-blocks), an expert count that is no power of two and exceeds
+    one byte, a down projection of a single K-block."""
+    c = inputs.moe_case(91, m, h=h, i=i, e=e, k=k)
+    wide, d_w = _layer(ctx, c, 1)
+    out, d = _layer(ctx, c, 0)
+    for key in ("expert_offsets", "sorted_pair", "gate_up", "h", "h_codes", "h_scales", "down_f32"):
+        assert torch.equal(d_w[key].view(torch.uint8), d[key].view(torch.uint8)), key
+    assert torch.equal(wide, out)
