@@ -429,6 +429,10 @@ int qarl_router_fwd(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H,
                     const void* w_router_bf16, int64_t E, int64_t k, float* logits_f32,
                     int32_t* topk_ids, float* topk_weights, void* stream);
 
+/* Tracing: every entry point that launches kernels opens an NVTX range named after itself for the
+ * duration of the host call (header-only NVTX 3; a pointer check when no tool is attached), so a
+ * timeline profiler shows the library's calls among the caller's own ranges. */
+
 /* Stage timing (measurement aid, no paper counterpart).  Between qarl_profile_begin and
  * qarl_profile_end every call of this context brackets each of its kernels with CUDA events
  * on the caller's stream (events are created in qarl_profile_begin, none in the hot calls;

@@ -162,6 +162,7 @@ int qarl_quantize_weight(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int
 
 int qarl_quantize_weight_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_t N, int64_t K, uint8_t* codes,
                                  float* scales, uint8_t* pub_codes, float* pub_scales, void* stream) {
+  NvtxRange nvtx_range("qarl_quantize_weight_publish");
   if (!ctx || E < 0 || N < 0 || K < 0) return QARL_ERR_INVALID_ARG;
   if ((pub_codes == nullptr) != (pub_scales == nullptr)) return QARL_ERR_INVALID_ARG;
   if (!aligned16(pub_codes) || (reinterpret_cast<uintptr_t>(pub_scales) & 3u)) return QARL_ERR_MISALIGNED;
@@ -179,6 +180,7 @@ int qarl_quantize_weight_publish(qarl_ctx* ctx, const void* w, int64_t E, int64_
 
 int qarl_quantize_act(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* codes,
                       float* scales, void* stream) {
+  NvtxRange nvtx_range("qarl_quantize_act");
   if (!ctx || M < 0 || K < 0 || ldx < K) return QARL_ERR_INVALID_ARG;
   if (K % kBlock) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M * (K / kBlock) > (0x7FFFFFFFll << 5)) return QARL_ERR_UNSUPPORTED_SHAPE;
@@ -201,6 +203,7 @@ size_t qarl_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* xc, const float* xs, int64_t M, int64_t K, const uint8_t* wc,
                       const float* ws, int64_t N, void* y, float* y_f32, void* stream) {
+  NvtxRange nvtx_range("qarl_linear_fwd_q");
   if (!ctx || M < 0 || K <= 0 || N <= 0) return QARL_ERR_INVALID_ARG;
   if (N % kBlock || K % kBlock || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
@@ -228,6 +231,7 @@ int qarl_linear_fwd_q(qarl_ctx* ctx, const uint8_t* xc, const float* xs, int64_t
 
 int qarl_linear_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t K, const uint8_t* wc, const float* ws,
                     int64_t N, void* y, float* y_f32, void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("qarl_linear_fwd");
   if (!ctx || M < 0 || K <= 0 || N <= 0) return QARL_ERR_INVALID_ARG;
   if (N % kBlock || K % kBlock || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
@@ -253,6 +257,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
                  int64_t I, int64_t E, int64_t k, const uint8_t* w13c, const float* w13s, const uint8_t* w2c,
                  const float* w2s, void* out, void* workspace, size_t workspace_bytes, const qarl_moe_debug* dbg,
                  void* stream) {
+  NvtxRange nvtx_range("qarl_moe_fwd");
   if (!ctx || M < 0 || H <= 0 || I <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
   if (H % kBlock || I % kBlock || E > 1024 || M * k >= 0x7FFFFF00ll || E * 2 * I > 0x7FFFFF00ll)
     return QARL_ERR_UNSUPPORTED_SHAPE;

@@ -57,6 +57,7 @@ size_t qarl_moe_dispatch_workspace_bytes(int64_t M, int64_t E, int64_t k) {
 int qarl_moe_dispatch(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* wts, int64_t M, int64_t H,
                       int64_t E, int64_t k, uint8_t* codes_sorted, float* scales_sorted, float* weights_sorted,
                       int32_t* offsets, int32_t* pos_of_pair, void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_dispatch");
   if (!ctx || M < 0 || H <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
   if (H % kBlock || E > 1024 || M * k >= 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (!offsets) return QARL_ERR_INVALID_ARG;
@@ -98,6 +99,7 @@ int qarl_moe_experts_fwd(qarl_ctx* ctx, const uint8_t* codes, const float* scale
                          const int32_t* offsets, int64_t R, int64_t H, int64_t I, int64_t E_local,
                          const uint8_t* w13c, const float* w13s, const uint8_t* w2c, const float* w2s, void* contrib,
                          void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_experts_fwd");
   if (!ctx || R < 0 || H <= 0 || I <= 0 || E_local < 1) return QARL_ERR_INVALID_ARG;
   if (H % kBlock || I % kBlock || E_local > 1024 || R >= 0x7FFFFF00ll || E_local * 2 * I > 0x7FFFFF00ll)
     return QARL_ERR_UNSUPPORTED_SHAPE;
@@ -152,6 +154,7 @@ int qarl_moe_experts_fwd(qarl_ctx* ctx, const uint8_t* codes, const float* scale
 
 int qarl_moe_combine_sorted(qarl_ctx* ctx, const void* contrib_sorted, const int32_t* ids, const int32_t* pos_of_pair,
                             int64_t M, int64_t H, int64_t E, int64_t k, void* out, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_combine_sorted");
   if (!ctx || M < 0 || H <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
   if (H % 8 || M * k >= 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;

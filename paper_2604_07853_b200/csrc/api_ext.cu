@@ -250,6 +250,7 @@ int qarl_moe_fwd_w4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const f
                        int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w13z,
                        const uint8_t* w2p, const void* w2s, const uint8_t* w2z, void* out, void* workspace,
                        size_t workspace_bytes, const qarl_moe_debug* dbg, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_fwd_w4a16");
   return moe_w4(ctx, kFmtInt4, x, ids, wts, M, H, I, E, k, w13p, w13s, w13z, w2p, w2s, w2z, out, workspace,
                 workspace_bytes, dbg, stream);
 }
@@ -258,6 +259,7 @@ int qarl_moe_fwd_fp4a16(qarl_ctx* ctx, const void* x, const int32_t* ids, const 
                         int64_t I, int64_t E, int64_t k, const uint8_t* w13p, const void* w13s, const uint8_t* w2p,
                         const void* w2s, void* out, void* workspace, size_t workspace_bytes,
                         const qarl_moe_debug* dbg, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_fwd_fp4a16");
   return moe_w4(ctx, kFmtE2m1, x, ids, wts, M, H, I, E, k, w13p, w13s, nullptr, w2p, w2s, nullptr, out, workspace,
                 workspace_bytes, dbg, stream);
 }
@@ -269,6 +271,7 @@ size_t qarl_moe_w4a16_workspace_bytes(int64_t M, int64_t H, int64_t I, int64_t E
 
 int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w, int64_t M, int64_t N, int64_t K,
                     void* dx, float* dx_f32, float* dw_f32, void* stream) {
+  NvtxRange nvtx_range("qarl_linear_bwd");
   if (!ctx || M < 0 || N <= 0 || K <= 0) return QARL_ERR_INVALID_ARG;
   if (N % 8 || K % 8 || M > 0x7FFFFF00ll || N > 0x7FFFFF00ll || K > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
@@ -321,6 +324,7 @@ int qarl_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w,
 int qarl_grouped_linear_bwd(qarl_ctx* ctx, const void* dy, const void* x, const void* w, const int32_t* offsets,
                             int64_t P, int64_t N, int64_t K, int64_t E, void* dx, float* dx_f32, float* dw_f32,
                             void* stream) {
+  NvtxRange nvtx_range("qarl_grouped_linear_bwd");
   if (!ctx || P < 0 || N <= 0 || K <= 0 || E < 1) return QARL_ERR_INVALID_ARG;
   if (N % 64 || K % 8 || E > 1024 || P > 0x7FFFFF00ll || E * N > 0x7FFFFF00ll || E * K > 0x7FFFFF00ll)
     return QARL_ERR_UNSUPPORTED_SHAPE;
@@ -389,6 +393,7 @@ int qarl_moe_bwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
                  int64_t E, int64_t k, const void* w13, const void* w2, const void* gate_up, const void* h,
                  const void* dout, const float* down_f32, void* dx, float* dw13, float* dw2, float* dwts,
                  void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("qarl_moe_bwd");
   if (!ctx || M < 0 || H <= 0 || I <= 0 || E < 1 || k < 1 || k > 32) return QARL_ERR_INVALID_ARG;
   if (H % 64 || I % 32 || E > 1024 || M * k >= 0x7FFFFF00ll || E * 2 * I > 0x7FFFFF00ll || E * H > 0x7FFFFF00ll)
     return QARL_ERR_UNSUPPORTED_SHAPE;
@@ -524,6 +529,7 @@ int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learn
                    const int64_t* offsets, const float* adv, int64_t B, int64_t T, const qarl_tbpo_params* prm,
                    double* r_seq, double* w_seq, double* j_seq, int32_t* flags, float* grad, double* loss,
                    void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("qarl_tbpo_loss");
   if (!ctx || B < 0 || T < 0 || !prm || !loss) return QARL_ERR_INVALID_ARG;
   if (!(prm->cap > 1.0) || prm->eps_h < 0.0 || prm->delta_l < 0.0 || prm->delta_h < 0.0) return QARL_ERR_INVALID_ARG;
   if (B > 0x7FFFFF00ll || T / 2048 > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
@@ -558,6 +564,7 @@ int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learn
 
 int qarl_router_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, const void* wr, int64_t E, int64_t k,
                     float* logits, int32_t* ids, float* wts, void* stream) {
+  NvtxRange nvtx_range("qarl_router_fwd");
   if (!ctx || M < 0 || H <= 0 || E <= 0 || k < 1 || k > 32 || k > E) return QARL_ERR_INVALID_ARG;
   if (H % 8 || E % 8 || E > 1024 || M > 0x7FFFFF00ll) return QARL_ERR_UNSUPPORTED_SHAPE;
   if (M == 0) return QARL_OK;
