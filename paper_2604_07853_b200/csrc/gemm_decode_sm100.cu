@@ -68,7 +68,7 @@ constexpr int kMaxExperts = 1024;
 constexpr int kOutRowBytes = 2 * BW * 2 + 16;  // bf16 row of 256 outputs, padded
 constexpr uint32_t kOutBytes = NT * kOutRowBytes;
 constexpr int kModeLayer = 3;     // gate_up tiles + down tiles + combine in one launch (this file only)
-constexpr int kDepSlots = 32;     // the down tiles of expert e are listed with the gate_up tiles of expert e + kDepSlots
+constexpr int kDepSlots = 64;     // the down tiles of expert e are listed with the gate_up tiles of expert e + kDepSlots
 constexpr int kMaxTopK = 32;
 constexpr int kSchedSlots = 4;    // layer: tile numbers the producer has drawn and the other roles have not yet read
 
