@@ -38,7 +38,7 @@ MoePlan plan_moe(int64_t M, int64_t H, int64_t I, int64_t E, int64_t k) {
   p.h_codes = take(P * I);
   p.h_scales = take(P * (I / kBlock) * sizeof(float));
   p.contrib = take(P * H * sizeof(uint16_t));
-  p.sync = take((2 * E + 1) * sizeof(int32_t));  // counters of the one-launch decode layer
+  p.sync = take((2 * E + 2) * sizeof(int32_t));  // counters of the one-launch decode layer
   p.total = o;
   return p;
 }
@@ -289,7 +289,7 @@ int qarl_moe_fwd(qarl_ctx* ctx, const void* x, const int32_t* ids, const float* 
   if (prep_small) {
     // decode-sized: grouping + quantization + scatter in one launch (timed as the quantize_act stage)
     if ((e = launch_moe_prep_small(L, ids, M, k, E, pb, static_cast<const uint16_t*>(x), H, wts, a_codes, a_scales,
-                                   sorted_w, layer_sync, static_cast<int>(2 * E + 1))) != cudaSuccess)
+                                   sorted_w, layer_sync, static_cast<int>(2 * E + 2))) != cudaSuccess)
       return cuda_fail(ctx, e, "moe_prep");
     mark(ctx, L.stream, QARL_STAGE_QUANT_ACT);
   } else {

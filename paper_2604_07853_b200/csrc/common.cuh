@@ -160,7 +160,7 @@ cudaError_t launch_gemm_decode(const Launch& L, EncodeTiledFn encode, const Gemm
 // The decode-sized MoE layer after its grouping / quantization as ONE launch of that kernel: gate_up tiles,
 // down tiles (each waiting on a per-expert counter for the h rows it reads) and the k-sum of the
 // contributions.  `g` and `d` are the two projections as launch_gemm takes them (same groups);
-// `sync` is [1 + 2 E] int32 that must be zero when the kernel starts.  Same bytes as the separate launches.
+// `sync` is [2 + 2 E] int32 that must be zero when the kernel starts.  Same bytes as the separate launches.
 bool moe_decode_layer_applies(const GemmArgs& g, const GemmArgs& d);
 cudaError_t launch_moe_decode_layer(const Launch& L, EncodeTiledFn encode, const GemmArgs& g, const GemmArgs& d,
                                     const int32_t* ids, const int32_t* pos_of_pair, int64_t M, int64_t k, uint16_t* y,

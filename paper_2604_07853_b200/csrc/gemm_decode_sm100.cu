@@ -102,7 +102,7 @@ struct DecodeParams {
   uint16_t* y;                 // [M, H]
   int M, k;
   int* sync;                   // [0]: tiles handed out so far; [1 + e]: finished gate_up tiles of expert e;
-                               // [1 + E + e]: finished down tiles of expert e (all zero on entry)
+                               // [1 + E + e]: finished down tiles of expert e; [1 + 2E]: tokens handed out (all zero on entry)
   int* status;
   unsigned long long wait_limit_ns;
   int stop_after_stages;
@@ -131,6 +131,8 @@ struct __align__(8) SmemTail {
   int abort_flag;
   int ready_flag;
   int peek_T;
+  int token_T;
+  int pad_;
   int32_t order[1][kMaxTopK];  // combine: contribution row of the rank-th smallest expert id of a token
   int32_t off[kMaxExperts + 1];
   int32_t prefix[kMaxExperts + kDepSlots + 1];
@@ -771,14 +773,19 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (kLayer) {
       // ---- the combine --------------------------------------------------------------------------
       // out[t] = bf16( sum of the token's k bf16 contributions in ascending expert id, from 0.0f ).
-      // CTA b sums tokens b, b + grid, ... as soon as the down tiles of the token's k experts are all
-      // finished (their counters), so a CTA that runs out of tiles early sums while others still stream.
+      // A CTA that has run out of tiles draws tokens from a counter and sums each as soon as the down tiles
+      // of the token's k experts are all finished (their counters), while others still stream.
       ok = named_bar_all(4, kEpiThreads, ok);
       const int k = p.k, H = p.pj[1].N;
       const int64_t P = static_cast<int64_t>(p.M) * k;
       const int* dcount = p.sync + 1 + p.E;
       if (ok) {
-        for (int64_t t = blockIdx.x; t < p.M; t += gridDim.x) {
+        for (;;) {
+          // tokens are drawn like tiles: the CTAs that run out of tiles first sum the most tokens
+          if (et == 0) *reinterpret_cast<volatile int*>(&s->token_T) = atomicAdd(p.sync + 1 + 2 * p.E, 1);
+          named_bar_sync(4, kEpiThreads);
+          const int64_t t = *reinterpret_cast<volatile int*>(&s->token_T);
+          if (t >= p.M) break;
           // lane l < k of every warp holds the token's l-th pair: its rank among the token's expert ids
           // gives the position of its row in the sum; the lane also waits for its expert's down tiles
           const int mine = lane < k ? p.ids[t * k + lane] : 0x7FFFFFFF;
