@@ -43,15 +43,16 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const float* __restric
         }
       }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
-      const int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, o);
-      if (oe != 0x7FFFFFFF && (best_e == 0x7FFFFFFF || ob > best || (ob == best && oe < best_e))) {
-        best = ob;
-        best_e = oe;
-      }
-    }
+    // Warp arg-max in two reductions instead of a five-step butterfly on (value, id) pairs: the largest
+    // value through an order-preserving map of its bits to unsigned (-0 first folded onto +0, so equal
+    // values map to equal keys), then the lowest id among the lanes that hold it.
+    const uint32_t bits = __float_as_uint(best + 0.0f);
+    const uint32_t key = best_e == 0x7FFFFFFF ? 0u : ((bits & 0x80000000u) ? ~bits : (bits | 0x80000000u));
+    const uint32_t top = __reduce_max_sync(0xFFFFFFFFu, key);
+    const int win_e = static_cast<int>(__reduce_min_sync(0xFFFFFFFFu, key == top ? static_cast<uint32_t>(best_e) : 0x7FFFFFFFu));
+    const float win = __shfl_sync(0xFFFFFFFFu, best, win_e & 31);
+    best = win;
+    best_e = win_e;
     if ((best_e & 31) == lane) taken |= 1u << (best_e >> 5);
     if (lane == r) {
       sel = best;
