@@ -29,10 +29,11 @@
 // list holds the gate_up tiles and the down tiles of every expert, the down tiles of expert e
 // kDepSlots experts after its gate_up tiles, so the weight stream never stops between the two
 // projections; a down tile starts once a per-expert counter says the h rows it reads are written
-// (release by the writers, acquire + proxy fence by the readers, every spin bounded); a CTA that
-// has finished its tiles sums its share of the tokens -- a token's k contributions in ascending
-// expert id (the combine), read from L2 -- each as soon as the down tiles of its experts are done.  Tile arithmetic,
-// promotion chain and epilogues are the ones of the separate launches: the bytes are the same.
+// (release by the writers, acquire + proxy fence by the readers, every spin bounded); tiles are
+// drawn from a counter (they differ in size), and a CTA that has run out of tiles draws tokens
+// and sums each -- its k contributions in ascending expert id (the combine), read from L2 -- as
+// soon as the down tiles of the token's experts are done.  Tile arithmetic, promotion chain and
+// epilogues are the ones of the separate launches: the bytes are the same.
 #include <algorithm>
 #include <atomic>
 
