@@ -53,7 +53,8 @@ int qarl_harness_stop_producer_after(qarl_ctx* ctx, int64_t stages);
  * tiles, down tiles and the k-sum in one launch).  The library picks by size; this call forces one
  * (1 = wide, 2 = decode where it applies -- grouped calls with K <= 8192 --, one launch per projection
  * and a separate combine) or restores the automatic choice (0), so that a test can run one input
- * through each and compare.  Host side only, stored in the context. */
+ * through each and compare.  A value other than 0 also makes qarl_router_fwd take its two-launch form.
+ * Host side only, stored in the context. */
 int qarl_harness_set_gemm_path(qarl_ctx* ctx, int path);
 
 /* Roofline denominators measured with the library's own instructions (used by the benchmark; the

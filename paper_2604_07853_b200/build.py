@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqarl.so")
 SOURCES = ["api.cu", "quantize.cu", "permute.cu", "combine.cu", "gemm_sm100.cu", "gemm_decode_sm100.cu", "harness.cu", "linear_static.cu",
-           "gemm_w4a16_sm100.cu", "gemm_w4a16_decode_sm100.cu", "api_ext.cu", "api_ep.cu", "gemm_bf16_sm100.cu", "tbpo.cu", "router.cu", "moe_bwd.cu"]
+           "gemm_w4a16_sm100.cu", "gemm_w4a16_decode_sm100.cu", "api_ext.cu", "api_ep.cu", "gemm_bf16_sm100.cu", "tbpo.cu", "router.cu", "router_fused_sm100.cu", "moe_bwd.cu"]
 HEADERS = ["common.cuh", "quant_device.cuh", "w4_dequant.cuh", "ptx_sm100.cuh", "sched.cuh", "api_util.cuh", os.path.join("..", "..", "include", "qarl.h"),
            os.path.join("..", "..", "include", "qarl_harness.h")]
 

@@ -571,6 +571,19 @@ int qarl_router_fwd(qarl_ctx* ctx, const void* x, int64_t M, int64_t H, const vo
   if (!x || !wr || !logits || !ids || !wts) return QARL_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(wr) || !aligned16(logits)) return QARL_ERR_MISALIGNED;
   Launch L = make_launch(ctx, stream);
+  if (L.gemm_path == 0 && router_fused_applies(E, k)) {  // one launch: selection in the GEMM's epilogue
+    CUresult cu = CUDA_SUCCESS;
+    mark(ctx, L.stream, -1);
+    cudaError_t e = launch_router_fused(L, ctx->encode, static_cast<const uint16_t*>(x), M, H,
+                                        static_cast<const uint16_t*>(wr), E, k, logits, ids, wts, &cu);
+    if (cu != CUDA_SUCCESS) {
+      snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(cu));
+      return QARL_ERR_CUDA;
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "router");
+    mark(ctx, L.stream, QARL_STAGE_ROUTER);
+    return QARL_OK;
+  }
   GemmBf16Args a{};
   a.a = static_cast<const uint16_t*>(x);   // A(m, h) = x[m, h]
   a.b = static_cast<const uint16_t*>(wr);  // B(e, h) = W_r[e, h]

@@ -233,6 +233,11 @@ cudaError_t launch_pair_dot(const Launch& L, const uint16_t* dout, const float* 
 // fp32 logits [M, E] -> top-k ids (descending, ties to the lower id) and softmax weights over the selection
 cudaError_t launch_router_topk(const Launch& L, const float* logits, int64_t M, int64_t E, int64_t k, int32_t* ids,
                                float* wts);
+// One-launch router (logits tile on the tensor cores, selection and softmax in its epilogue) for E <= 128.
+bool router_fused_applies(int64_t E, int64_t k);
+cudaError_t launch_router_fused(const Launch& L, EncodeTiledFn encode, const uint16_t* x, int64_t M, int64_t H,
+                                const uint16_t* wr, int64_t E, int64_t k, float* logits, int32_t* ids, float* wts,
+                                CUresult* cu_err);
 
 // ---- TBPO sequence-level loss ------------------------------------------------------------------
 struct TbpoArgs {

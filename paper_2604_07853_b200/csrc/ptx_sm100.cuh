@@ -79,6 +79,20 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+// Tiled store shared -> global as a bulk async-group; rows and columns outside the tensor map's
+// extents are dropped.  x as for loads; never start a store at a negative coordinate.  The shared
+// memory was written through the generic proxy: fence_proxy_async_smem() by the writers first.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* smem_src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all groups of this thread have finished READING their shared-memory source (it may be rewritten)
+__device__ __forceinline__ void bulk_wait_group_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all groups of this thread are complete
+__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // L2 cache policies for loads: evict_first for data read once (streamed weights), evict_last for
 // small data that later kernels read again.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {

@@ -62,9 +62,8 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const float* __restric
   // softmax over the k selected logits, in double: exp(l - max) / sum, rounded to fp32
   const double mx = static_cast<double>(__shfl_sync(0xFFFFFFFFu, sel, 0));
   double ex = lane < k ? exp(static_cast<double>(sel) - mx) : 0.0;
-  double den = ex;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+  double den = 0.0;  // summed in selection order (the one-launch router adds them as it selects)
+  for (int j = 0; j < k; ++j) den += __shfl_sync(0xFFFFFFFFu, ex, j);
   if (lane < k) {
     ids[m * k + lane] = sel_id;
     wts[m * k + lane] = static_cast<float>(ex / den);

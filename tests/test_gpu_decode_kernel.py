@@ -96,3 +96,34 @@ def test_one_launch_layer_long_k_and_many_experts(ctx, m, h, i, e, k):
     for key in ("expert_offsets", "sorted_pair", "gate_up", "h", "h_codes", "h_scales", "down_f32"):
         assert torch.equal(d_w[key].view(torch.uint8), d[key].view(torch.uint8)), key
     assert torch.equal(wide, out)
+
+
+def test_decode_step_replays_from_a_cuda_graph(ctx):
+    """The decode-sized layer call allocates nothing and synchronizes nothing, so a stream capture
+    takes it whole (its launches keep their programmatic dependencies); replaying the graph gives the
+    bytes of the plain call, also after the output and the workspace were overwritten in between."""
+    c = inputs.moe_case(13, 256)
+    w13c, w13s = ctx.quantize_weight(bits_to_torch(c.w13))
+    w2c, w2s = ctx.quantize_weight(bits_to_torch(c.w2))
+    x, ids, wts = bits_to_torch(c.x), torch.from_numpy(c.ids).cuda(), torch.from_numpy(c.weights).cuda()
+    M, H = x.shape
+    out = torch.empty((M, H), dtype=torch.bfloat16, device=x.device)
+    ws = torch.empty(ctx.moe_workspace_bytes(M, H, w2c.shape[2], w13c.shape[0], ids.shape[1]), dtype=torch.uint8,
+                     device=x.device)
+    ref = ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s).clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, workspace=ws)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for _ in range(3):
+            ctx.moe_fwd(x, ids, wts, w13c, w13s, w2c, w2s, out=out, workspace=ws)
+    for _ in range(2):
+        out.zero_()
+        ws.fill_(0xA5)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref) and ctx.poll() == 0

@@ -74,6 +74,28 @@ def test_routing_does_not_depend_on_the_batch(ctx):
         assert torch.equal(l2, logits[rows]) and torch.equal(i2, ids[rows]) and torch.equal(w2, wts[rows])
 
 
+@pytest.mark.parametrize("m,h,e,k", [(1, 64, 8, 1), (300, 2048, 128, 8), (1000, 520, 40, 8), (129, 512, 128, 32),
+                                     (4133, 1024, 96, 6)])
+def test_one_launch_router_equals_the_two_launch_router(ctx, m, h, e, k):
+    """Up to 128 experts the selection runs in the epilogue of the logits GEMM (one launch); the harness
+    switch forces the separate selection kernel.  Logits, ids and weights must be the same bytes: the
+    same MMA sequence per row, the same selection rule, the softmax summed in the same order."""
+    rng = np.random.default_rng(900 + m)
+    x = bits_to_torch(inputs.act_bf16(rng, m, h))
+    wr_bits = inputs.weight_bf16(rng, e, h)
+    wr_bits[e - 1] = wr_bits[0]                              # a tie between the first and the last expert
+    wr = bits_to_torch(wr_bits)
+    fused = ctx.router_fwd(x, wr, k)
+    ctx.harness_set_gemm_path(1)
+    split = ctx.router_fwd(x, wr, k)
+    ctx.harness_set_gemm_path(0)
+    assert ctx.poll() == 0
+    for a, b in zip(fused, split):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    ids = fused[1].cpu().numpy()
+    assert ((ids >= 0) & (ids < e)).all() and all(len(set(r)) == k for r in ids[:: max(1, m // 50)].tolist())
+
+
 def test_o_proj_shape(ctx):
     """The attention output projection of the training configuration: K = 4096, N = 2048."""
     check_linear(ctx, inputs.linear_case(21, 200, 2048, 4096))
