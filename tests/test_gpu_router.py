@@ -75,7 +75,7 @@ def test_routing_does_not_depend_on_the_batch(ctx):
 
 
 @pytest.mark.parametrize("m,h,e,k", [(1, 64, 8, 1), (300, 2048, 128, 8), (1000, 520, 40, 8), (129, 512, 128, 32),
-                                     (4133, 1024, 96, 6)])
+                                     (4133, 1024, 96, 6), (3, 8, 8, 8), (129, 72, 24, 24), (40000, 128, 128, 8)])
 def test_one_launch_router_equals_the_two_launch_router(ctx, m, h, e, k):
     """Up to 128 experts the selection runs in the epilogue of the logits GEMM (one launch); the harness
     switch forces the separate selection kernel.  Logits, ids and weights must be the same bytes: the
@@ -94,6 +94,31 @@ def test_one_launch_router_equals_the_two_launch_router(ctx, m, h, e, k):
         assert torch.equal(a.view(torch.int32), b.view(torch.int32))
     ids = fused[1].cpu().numpy()
     assert ((ids >= 0) & (ids < e)).all() and all(len(set(r)) == k for r in ids[:: max(1, m // 50)].tolist())
+
+
+def test_router_with_non_finite_activations(ctx):
+    """Infinite and NaN activations give infinite and NaN logits; whatever the selection does with them, the
+    ids stay inside [0, E) and distinct, and both forms of the router do the same."""
+    rng = np.random.default_rng(77)
+    x = bits_to_torch(inputs.act_bf16(rng, 64, 256)).clone()
+    x[3, 5] = float("inf")
+    x[7, :] = float("nan")
+    x[9, 100] = float("-inf")
+    x[11, 1] = float("inf")
+    x[11, 2] = float("-inf")
+    wr = bits_to_torch(inputs.weight_bf16(rng, 32, 256))
+    fused = ctx.router_fwd(x, wr, 4)
+    ctx.harness_set_gemm_path(1)
+    split = ctx.router_fwd(x, wr, 4)
+    ctx.harness_set_gemm_path(0)
+    assert ctx.poll() == 0
+    ids = fused[1].cpu().numpy()
+    assert ((ids >= 0) & (ids < 32)).all() and all(len(set(r)) == 4 for r in ids.tolist())
+    assert torch.equal(fused[1], split[1])
+    assert torch.equal(fused[0].view(torch.int32), split[0].view(torch.int32))
+    assert torch.equal(fused[2].view(torch.int32), split[2].view(torch.int32))
+    o_ids, _ = oracle.router_topk(fused[0].cpu().numpy(), 4)
+    assert np.array_equal(ids, o_ids)
 
 
 def test_o_proj_shape(ctx):
