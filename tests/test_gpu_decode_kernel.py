@@ -127,3 +127,26 @@ def test_decode_step_replays_from_a_cuda_graph(ctx):
         g.replay()
         torch.cuda.synchronize()
         assert torch.equal(out, ref) and ctx.poll() == 0
+
+
+@pytest.mark.parametrize("m,n,k", [(64, 5120, 2048), (1, 256, 512), (31, 384, 128), (33, 128, 1024), (64, 2048, 4096),
+                                   (17, 640, 3968)])
+def test_dense_projection_decode_kernel_equals_wide_kernel(ctx, m, n, k):
+    """A dense projection of at most 64 rows runs on the swapped-operand kernel (automatic choice and
+    forced), larger ones on the wide-tile kernel: bf16 rows and fp32 accumulators must be the same bytes,
+    and a row's bytes must not depend on the batch around it."""
+    c = inputs.linear_case(300 + m, m, n, k)
+    wc, ws = ctx.quantize_weight(bits_to_torch(c.w))
+    x = bits_to_torch(c.x)
+    y0, f0 = ctx.linear_fwd(x, wc, ws, want_f32=True)
+    plain = ctx.linear_fwd(x, wc, ws).clone()
+    assert ctx.poll() == 0
+    for path in (1, 2):
+        ctx.harness_set_gemm_path(path)
+        y, f = ctx.linear_fwd(x, wc, ws, want_f32=True)
+        ctx.harness_set_gemm_path(0)
+        assert ctx.poll() == 0
+        assert torch.equal(y0, y) and torch.equal(f0.view(torch.int32), f.view(torch.int32)), path
+    assert torch.equal(plain, y0)
+    for rows in ([0], [m - 1], list(range(m // 2, m))):
+        assert torch.equal(ctx.linear_fwd(x[rows].contiguous(), wc, ws), y0[rows])
