@@ -28,8 +28,8 @@ int qarl_harness_rmsnorm(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H
  * qarl_poll_device_status reports (and clears) the error.  Nothing traps, faults or hangs. */
 int qarl_harness_wait_selftest(qarl_ctx* ctx, uint64_t limit_ns, void* stream);
 
-/* The two calls below exist so that a test can watch the FP8 GEMM's own pipeline give up on a wait
- * (the library never needs them).  Both only store a value in the context (host side, not
+/* The two calls below exist so that a test can watch the pipeline of the FP8 GEMMs and of the one-launch
+ * router give up on a wait (the library never needs them).  Both only store a value in the context (host side, not
  * synchronized with calls running on other threads); it applies to the GEMM kernels launched
  * through `ctx` afterwards.
  *

@@ -58,6 +58,7 @@ struct RouterParams {
   float* wts;
   int* status;
   unsigned long long wait_limit_ns;
+  int stop_after_stages;  // test harness only (< 0: off): the TMA producer stops arming stages after this many
 };
 
 struct __align__(8) SmemTail {
@@ -141,8 +142,11 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
       uint32_t phase = 0;
       uint32_t armed = 0, armed_parity = 0;
       bool ok = true;
+      int armed_total = 0;
       for (int T = blockIdx.x; ok && T < total_tiles; T += grid) {
         for (int ks = 0; ks < KS; ++ks) {
+          if (p.stop_after_stages >= 0 && armed_total >= p.stop_after_stages) { ok = false; break; }
+          ++armed_total;
           if (!wait_or_abort(&s->empty[stage], phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* a_dst = smem + static_cast<size_t>(stage) * kStageBytes;
           mbar_arrive_expect_tx(&s->full[stage], kStageBytes);
@@ -342,6 +346,7 @@ cudaError_t launch_router_fused(const Launch& L, EncodeTiledFn encode, const uin
   p.wts = wts;
   p.status = L.d_status;
   p.wait_limit_ns = L.wait_limit_ns ? L.wait_limit_ns : 2000000000ull;
+  p.stop_after_stages = L.stop_after_stages;
   // sticky per device; atomic: contexts on several host threads may launch at once (both would set the same value)
   static std::atomic<bool> attr_set_dev[64];
   std::atomic<bool>& attr_set = attr_set_dev[L.device & 63];

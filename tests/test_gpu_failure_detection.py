@@ -72,3 +72,31 @@ def test_gemm_pipeline_wait_expires_and_context_survives(stop_after):
     ctx.harness_set_wait_limit_ns(0)
     assert torch.equal(ctx.moe_fwd(*args), ref_moe) and ctx.poll() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("stop_after", [0, 1, 5])
+def test_router_pipeline_wait_expires_and_context_survives(stop_after):
+    """The same for the one-launch router: its TMA producer stops arming stages, the MMA role's bounded
+    wait (1 ms here) runs out, the CTA aborts (epilogue warps leave through the abort flag, logits
+    stores in flight are waited for, TMEM is freed), the status word says QARL_ERR_DEVICE_TIMEOUT and
+    the next call gives the reference bytes."""
+    build.build()
+    ctx = binding.Context(0)
+    rng = np.random.default_rng(8)
+    x = bits_to_torch(inputs.act_bf16(rng, 300, 512))       # 3 tiles of 8 contraction steps each
+    wr = bits_to_torch(inputs.weight_bf16(rng, 64, 512))
+    ref = [t.clone() for t in ctx.router_fwd(x, wr, 4)]
+    assert ctx.poll() == 0
+    ctx.harness_set_wait_limit_ns(1_000_000)
+    ctx.harness_stop_producer_after(stop_after)
+    t0 = time.perf_counter()
+    ctx.router_fwd(x, wr, 4)
+    assert ctx.poll() == -7
+    assert time.perf_counter() - t0 < 1.0
+    ctx.harness_stop_producer_after(-1)
+    ctx.harness_set_wait_limit_ns(0)
+    assert ctx.poll() == 0
+    for _ in range(2):
+        out = ctx.router_fwd(x, wr, 4)
+        assert all(torch.equal(a.view(torch.int32), b.view(torch.int32)) for a, b in zip(out, ref)) and ctx.poll() == 0
+    ctx.close()
