@@ -424,8 +424,8 @@ int qarl_tbpo_loss(qarl_ctx* ctx, const float* lp_cur, const float* lp_old_learn
  *      E <= 1024, 1 <= k <= min(E, 32).
  * out: logits_f32 [M, E] (required), topk_ids i32 [M, k], topk_weights f32 [M, k]; caller-owned.
  *      The outputs feed qarl_moe_fwd directly.
- * Up to 128 experts the call is one launch (the selection runs in the epilogue of the logits
- * GEMM); beyond that two (GEMM, then a selection kernel).  Both give the same bytes.
+ * Up to 128 experts and k <= 16 the call is one launch (the selection runs in the epilogue of the
+ * logits GEMM); beyond that two (GEMM, then a selection kernel).  Both give the same bytes.
  * A token's routing depends only on that token's row of x: bitwise the same for any M. */
 int qarl_router_fwd(qarl_ctx* ctx, const void* x_bf16, int64_t M, int64_t H,
                     const void* w_router_bf16, int64_t E, int64_t k, float* logits_f32,

@@ -96,6 +96,35 @@ def test_one_launch_router_equals_the_two_launch_router(ctx, m, h, e, k):
     assert ((ids >= 0) & (ids < e)).all() and all(len(set(r)) == k for r in ids[:: max(1, m // 50)].tolist())
 
 
+@pytest.mark.parametrize("e,k,hot", [(128, 16, range(0, 16)), (128, 16, range(16, 32)), (128, 8, range(120, 128)),
+                                     (40, 16, range(0, 16)), (128, 16, [0, 17, 33, 34, 35, 50, 66, 67, 82, 98, 99, 100, 113, 114, 126, 127])])
+def test_selection_concentrated_in_few_groups(ctx, e, k, hot):
+    """The one-launch router keeps one candidate per group of 16 experts and re-scans only the winner's group:
+    batches whose k largest logits all sit in one group (also the first, which then runs almost empty) or are
+    spread one per group must select what the oracle's plain scan selects on the same logits, in both forms."""
+    rng = np.random.default_rng(5 + e + k)
+    h = 256
+    u = rng.standard_normal(h).astype(np.float32)
+    x = (u[None, :] + 0.05 * rng.standard_normal((200, h))).astype(np.float32)
+    w = (0.02 * rng.standard_normal((e, h))).astype(np.float32)
+    for rank, ex in enumerate(hot):
+        w[ex] = (0.2 + 0.01 * ((rank * 7) % len(hot))) * u / np.linalg.norm(u)       # large, distinct, not in id order
+    w[hot[1]] = w[hot[0]]                                                            # and one exact tie
+    xt = torch.from_numpy(x).to(torch.bfloat16).cuda()
+    wt = torch.from_numpy(w).to(torch.bfloat16).cuda()
+    fused = ctx.router_fwd(xt, wt, k)
+    ctx.harness_set_gemm_path(1)
+    split = ctx.router_fwd(xt, wt, k)
+    ctx.harness_set_gemm_path(0)
+    assert ctx.poll() == 0
+    for a, b in zip(fused, split):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    o_ids, _ = oracle.router_topk(fused[0].cpu().numpy(), k)
+    ids = fused[1].cpu().numpy()
+    assert np.array_equal(ids, o_ids)
+    assert set(ids[0, :len(hot)].tolist()) == set(list(hot)[:k]) or len(hot) < k
+
+
 def test_router_with_non_finite_activations(ctx):
     """Infinite and NaN activations give infinite and NaN logits; whatever the selection does with them, the
     ids stay inside [0, E) and distinct, and both forms of the router do the same."""
