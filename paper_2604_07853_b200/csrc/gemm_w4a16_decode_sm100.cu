@@ -21,9 +21,10 @@
 // large as shared memory allows and every such thread has one job.
 // CTA = 768 threads: warps 0-3 epilogue (thread = weight row: TMEM -> SwiGLU / weighting -> bf16,
 // transposed through shared memory so that global stores are whole token rows), warps 4-11 / 12-19
-// dequantization of the tile's first / second weight block (two threads per weight row), warp 20
-// producer of the codes (bulk copies, streamed evict-first, a tile's codes pulled into L2 one tile
-// ahead), warp 21 producer of the token rows (TMA), warps 22 / 23 MMA issuers of the two blocks.
+// dequantization of the tile's first / second weight block (two threads per weight row; they read
+// their codes straight from global memory, three stages ahead, into registers), warp 21 producer of
+// the token rows (TMA), warps 22 / 23 MMA issuers of the two blocks (warp 20 only starts the CTA's
+// first tile's codes towards L2 while the kernel still waits for its predecessor).
 // Every barrier wait is bounded; an expired wait aborts the CTA cleanly.
 #include <algorithm>
 #include <atomic>
@@ -44,20 +45,18 @@ constexpr int BK = 64;             // bf16 elements per K-step (128 bytes)
 constexpr int kGK = 2;             // K-steps per stage: one 128-element quantization group
 constexpr int kEpiWarps = 4;       // warps 0-3
 constexpr int kDqHalfWarps = 8;    // warps 4-11 expand the tile's first block, warps 12-19 its second
-constexpr int kDqWarps = 2 * kDqHalfWarps;
 constexpr int kCodeWarp = 20;      // producer of the codes
 constexpr int kTokenWarp = 21;     // producer of the token rows
 constexpr int kMmaWarp0 = 22;      // MMA issuer of the first block (warp 23: of the second)
 constexpr int kThreads = 24 * 32;
 constexpr uint32_t kQStepBytes = BW * BK / 2;            // 4 KB: 128 rows x 32 bytes of codes (one K-step of one block)
 constexpr uint32_t kQHalfBytes = kGK * kQStepBytes;      // 8 KB: one block, one group
-constexpr uint32_t kQBytes = 2 * kQHalfBytes;            // 16 KB per stage
 constexpr uint32_t kXStepBytes = NT * BK * 2;            // 4 KB: 32 token rows x 64 bf16
 constexpr uint32_t kXBytes = kGK * kXStepBytes;          // 8 KB per stage
 constexpr uint32_t kDqStepBytes = BW * BK * 2;           // 16 KB: one expanded block, one K-step
 constexpr uint32_t kDqBytes = kGK * kDqStepBytes;        // 32 KB per stage and block
-constexpr int kQStages = 3;
-constexpr int kXStages = 2;
+constexpr int kCodeAhead = 3;       // stages whose codes a dequantization thread holds in registers ahead of use
+constexpr int kXStages = 4;
 constexpr int kDqStages = 2;       // per block
 constexpr int kAccBufs = 4;        // TMEM accumulators of 2 x NT columns
 constexpr uint32_t kTmemCols = 256;
@@ -87,8 +86,6 @@ struct W4DecodeParams {
 };
 
 struct __align__(8) SmemTail {
-  uint64_t q_full[kQStages];
-  uint64_t q_empty[kQStages];
   uint64_t x_full[kXStages];
   uint64_t x_empty[kXStages];
   uint64_t dq_full[2][kDqStages];
@@ -102,7 +99,7 @@ struct __align__(8) SmemTail {
   int32_t prefix[kMaxExperts + 1];
 };
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kQStages) * kQBytes + static_cast<size_t>(kXStages) * kXBytes +
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kXStages) * kXBytes +
                               2 * static_cast<size_t>(kDqStages) * kDqBytes + kOutBytes + sizeof(SmemTail);
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
@@ -165,18 +162,13 @@ gemm_w4a16_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const W4Decod
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* dq_base = smem;                                                   // [block][stage][K-step][16 KB], 1024-byte aligned
   uint8_t* x_base = dq_base + 2 * static_cast<size_t>(kDqStages) * kDqBytes;  // [stage][K-step][4 KB]
-  uint8_t* q_base = x_base + static_cast<size_t>(kXStages) * kXBytes;         // [stage][block][K-step][4 KB]
-  uint8_t* out_tile = q_base + static_cast<size_t>(kQStages) * kQBytes;
+  uint8_t* out_tile = x_base + static_cast<size_t>(kXStages) * kXBytes;
   SmemTail* s = reinterpret_cast<SmemTail*>(out_tile + kOutBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   // ---- set-up: barriers, TMEM, tile list ------------------------------------------------
   pdl_trigger();
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kQStages; ++i) {
-      mbar_init(&s->q_full[i], 1);
-      mbar_init(&s->q_empty[i], kDqWarps);        // every dequant warp, once its codes are in registers
-    }
     for (int i = 0; i < kXStages; ++i) {
       mbar_init(&s->x_full[i], 1);
       mbar_init(&s->x_empty[i], 2);               // the commits of the two MMA issuers
@@ -210,8 +202,7 @@ gemm_w4a16_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const W4Decod
     q_lo = p.b_packed + (static_cast<int64_t>(e) * NB + nb_lo) * KS * kQStepBytes;
     q_hi = p.b_packed + (static_cast<int64_t>(e) * NB + nb_hi) * KS * kQStepBytes;
   };
-  // The codes are the stream from HBM, and only three stages of them fit beside the expanded tiles:
-  // a whole tile's codes are pulled into L2 one tile ahead, so the ring only has to cover the L2 latency.
+  // pull a whole tile's codes towards L2 (used once, for the CTA's first tile, before the dependency wait)
   auto prefetch_tile = [&](int e, int j) {
     const uint8_t *q_lo, *q_hi;
     tile_codes(e, j, q_lo, q_hi);
@@ -238,40 +229,7 @@ gemm_w4a16_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const W4Decod
   const int first_tile = blockIdx.x;
 
   if (warp == kCodeWarp) {
-    // =============================== producer of the codes ============================
-    if (lane == 0) {
-      int qs = 0, cur_e = 0, cur_n = 0;
-      uint32_t q_phase = 0, q_armed = 0, q_armed_parity = 0;
-      bool ok = true;
-      // the codes are read once per call: evict-first keeps them from pushing the layer's small shared data out of L2
-      const uint64_t stream_once = l2_policy_evict_first();
-      for (int T = first_tile; ok && T < total_tiles; T += num_ctas) {
-        const TileCoord c = decode_tile(s->off, s->prefix, NT, T, cur_e);
-        if (T + num_ctas < total_tiles) {
-          cur_n = max(cur_n, cur_e);
-          const TileCoord cn = decode_tile(s->off, s->prefix, NT, T + num_ctas, cur_n);
-          prefetch_tile(cn.e, cn.n_tile);
-        }
-        const uint8_t *q_lo, *q_hi;
-        tile_codes(c.e, c.n_tile, q_lo, q_hi);
-        for (int g = 0; g < KG; ++g) {
-          if (!wait_or_abort(&s->q_empty[qs], q_phase ^ 1, s, p)) { ok = false; break; }
-          uint8_t* q_dst = q_base + static_cast<size_t>(qs) * kQBytes;
-          mbar_arrive_expect_tx(&s->q_full[qs], kQBytes);
-          // consecutive K-steps of a block are consecutive 4 KB chunks of the tile-major storage: one copy per block
-          bulk_load_1d_hint(q_dst, q_lo + static_cast<int64_t>(g) * kQHalfBytes, kQHalfBytes, &s->q_full[qs], stream_once);
-          bulk_load_1d_hint(q_dst + kQHalfBytes, q_hi + static_cast<int64_t>(g) * kQHalfBytes, kQHalfBytes, &s->q_full[qs],
-                            stream_once);
-          q_armed |= 1u << qs;
-          q_armed_parity = (q_armed_parity & ~(1u << qs)) | (q_phase << qs);
-          if (++qs == kQStages) { qs = 0; q_phase ^= 1; }
-        }
-      }
-      if (!ok) {  // let copies in flight land before the CTA's shared memory is released
-        for (int i = 0; i < kQStages; ++i)
-          if (q_armed & (1u << i)) mbar_wait_bounded(&s->q_full[i], (q_armed_parity >> i) & 1u, 20000000ull);
-      }
-    }
+    // (this warp only started the first tile's codes on their way to L2, above)
   } else if (warp == kTokenWarp) {
     // =============================== producer of the token rows =======================
     if (lane == 0) {
@@ -354,6 +312,39 @@ gemm_w4a16_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const W4Decod
       const int row = min((h ? nb_hi : nb_lo) * BW + nr, p.N - 1);
       return (static_cast<int64_t>(c.e) * KG + g) * p.N + row;
     };
+    // The codes come straight from global memory, three stages ahead of their use, in registers: no
+    // shared-memory ring and no hand-off between a producer thread and these warps stands between the
+    // memory and the expansion.  Consecutive threads read consecutive 16-byte pieces of a 4 KB chunk
+    // ([word quad 0..1][row][16 bytes]); the data are read once (streaming loads).  (Pulling a tile's codes
+    // into L2 a tile ahead as well was measured and costs 7 % here.)
+    int pfT = first_tile, pfg = 0, pf_e = 0;
+    const uint8_t* pf_base = nullptr;  // this thread's piece of group 0 of tile pfT
+    auto pf_set_tile = [&]() {
+      if (pfT < total_tiles) {
+        const TileCoord t = decode_tile(s->off, s->prefix, NT, pfT, pf_e);
+        const uint8_t *q_lo, *q_hi;
+        tile_codes(t.e, t.n_tile, q_lo, q_hi);
+        pf_base = (h ? q_hi : q_lo) + u * kQStepBytes + nr * 16;
+      }
+    };
+    auto pf_load = [&](uint4& a, uint4& b) {
+      if (pfT < total_tiles) {
+        const uint4* src = reinterpret_cast<const uint4*>(pf_base + static_cast<int64_t>(pfg) * kQHalfBytes);
+        a = __ldcs(src);
+        b = __ldcs(src + kQStepBytes / 32);
+        if (++pfg == KG) {
+          pfg = 0;
+          pfT += num_ctas;
+          pf_set_tile();
+        }
+      }
+    };
+    uint4 qa0 = make_uint4(0, 0, 0, 0), qa1 = qa0, qb0 = qa0, qb1 = qa0, qc0 = qa0, qc1 = qa0;
+    static_assert(kCodeAhead == 3, "three register sets");
+    pf_set_tile();
+    pf_load(qa0, qa1);
+    pf_load(qb0, qb1);
+    pf_load(qc0, qc1);
     int T = first_tile;
     if (T < total_tiles) {
       TileCoord c = decode_tile(s->off, s->prefix, NT, T, cur_e);
@@ -379,15 +370,13 @@ gemm_w4a16_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const W4Decod
           }
           s_next = __ldg(p.b_scales + sz);
           if constexpr (FMT == kFmtInt4) z_next = __ldg(p.b_zeros + sz);
-          const uint32_t qs = stage % kQStages, q_phase = (stage / kQStages) & 1u;
           const uint32_t ds = stage % kDqStages, dq_phase = (stage / kDqStages) & 1u;
-          if (!warp_wait_or_abort(&s->q_full[qs], q_phase, s, p)) { ok = false; break; }
-          // a chunk is [word quad 0..1][row][16 bytes]: consecutive threads read consecutive pieces
-          const uint4* q_src = reinterpret_cast<const uint4*>(q_base + static_cast<size_t>(qs) * kQBytes + h * kQHalfBytes +
-                                                              u * kQStepBytes + nr * 16);
-          const uint4 q0 = q_src[0], q1 = q_src[kQStepBytes / 32];
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&s->q_empty[qs]);  // the codes are in registers
+          const uint4 q0 = qa0, q1 = qa1;  // this stage's codes; the sets move up and the third one is refilled
+          qa0 = qb0;
+          qa1 = qb1;
+          qb0 = qc0;
+          qb1 = qc1;
+          pf_load(qc0, qc1);
           if (!warp_wait_or_abort(&s->dq_empty[h][ds], dq_phase ^ 1, s, p)) { ok = false; break; }
           uint8_t* row_dst = dq_base + (static_cast<size_t>(h) * kDqStages + ds) * kDqBytes + u * kDqStepBytes + nr * 128;
           const uint32_t words[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
