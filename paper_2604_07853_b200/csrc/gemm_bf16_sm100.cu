@@ -73,6 +73,7 @@ struct Bf16Params {
   int E;
   int rows_total;           // grouped contraction: P
   int a3d, b3d;             // MN-major operand staged by one 3-D TMA box (64 columns x 64 rows x blocks)
+  int col_fastest;          // dense: consecutive tiles walk the column tiles of a row tile (else the row tiles of a column tile)
   const int32_t* out_rows;  // grouped rows: output row of each sorted row (nullptr: the row itself)
   uint16_t* c_bf16;   // [Mo, No] or nullptr
   float* c_f32;       // [Mo, No] or nullptr
@@ -186,8 +187,17 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     Tile t{};
     t.last_valid = BK;
     if (GROUP == kDense) {
-      t.i0 = (T % m_tiles) * TM;
-      t.j0 = (T / m_tiles) * BN;
+      // CTAs that run at the same time take consecutive T.  Walking the column tiles of one row tile
+      // together (col_fastest) lets a wave of CTAs read each block of A once and share it through L2;
+      // walking the row tiles of one column tile together does the same for B.  The host picks the
+      // order that re-reads the smaller operand.
+      if (p.col_fastest) {
+        t.i0 = (T / n_tiles) * TM;
+        t.j0 = (T % n_tiles) * BN;
+      } else {
+        t.i0 = (T % m_tiles) * TM;
+        t.j0 = (T / m_tiles) * BN;
+      }
       t.KS = (p.Kc + BK - 1) / BK;  // a ragged last step reads zeros (TMA out-of-range fill)
       t.row_end = p.Mo;
     } else if (GROUP == kGroupedRows) {
@@ -480,6 +490,7 @@ cudaError_t launch_gemm_bf16(const Launch& L, EncodeTiledFn encode, const GemmBf
   p.out_rows = a.out_rows;
   p.a3d = a3d;
   p.b3d = b3d;
+  p.col_fastest = a.group == 0 && a.Mo >= a.No;  // A (Mo x Kc) is the larger operand: re-read B, not A
   p.c_bf16 = a.c_bf16;
   p.c_f32 = a.c_f32;
   p.status = L.d_status;
