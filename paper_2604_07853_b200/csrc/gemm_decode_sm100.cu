@@ -17,12 +17,12 @@
 //
 // A tile = (expert e, pair of weight blocks j, chunk of <= 32 rows of the expert's group):
 //   gate_up: blocks j (gate rows) and j + I/128 (the matching up rows); down/linear: blocks 2j, 2j+1.
-// CTA = 384 threads in three warpgroups (registers re-allocated with setmaxnreg): warps 0-3 promotion
-// (thread = weight row, 2 x 32 accumulators; at the end of a tile they round to bf16 -- down: after
-// the multiplication by the pair's combine weight -- and transpose the tile through shared memory),
-// warps 4-7 epilogue (a warp per token row while the promotion warps run the next tile: gate_up =
-// SwiGLU, 1x128 amax / scale / e4m3 codes; down / linear = whole-row stores), warp 8 TMA producer,
-// warps 9 and 10 MMA issuers (one per weight block of the pair).
+// CTA = 512 threads, 128 registers each: warps 0-7 promotion (two threads per weight row -- warps w
+// and w + 4 read the same TMEM lanes, token columns 0-15 and 16-31 --, 2 x 16 accumulators each; at the
+// end of a tile they round to bf16 -- down: after the multiplication by the pair's combine weight --
+// and transpose the tile through shared memory), warps 8-11 epilogue (a warp per token row while the
+// promotion warps run the next tile: gate_up = SwiGLU, 1x128 amax / scale / e4m3 codes; down / linear =
+// whole-row stores), warp 12 TMA producer, warps 13 and 14 MMA issuers (one per weight block of the pair).
 // Every barrier wait is bounded as in the wide kernel; an expired wait aborts the CTA cleanly.
 //
 // The whole decode-sized MoE layer also runs as ONE launch of this kernel (kModeLayer): the tile
@@ -51,15 +51,14 @@ constexpr int NT = 32;            // token rows per tile (UMMA N)
 constexpr int BK = 128;
 constexpr int kStages = 5;         // 36 KB each: 180 KB of loads in flight per SM (2, 3, 5 stages: 99, 92, 87 us at decode)
 constexpr int kAccBufs = 8;       // TMEM accumulators of 2 x NT columns
-constexpr int kPromoWarps = 4;     // warps 0-3 (warpgroup 0)
-constexpr int kEpiWarps = 4;       // warps 4-7 (warpgroup 1)
-constexpr int kTmaWarp = 8;        // warpgroup 2: warp 11 idle (setmaxnreg works on whole warpgroups)
-constexpr int kMmaWarp = 9;         // and 10: one issuer per weight block of the pair
-constexpr int kThreads = 12 * 32;
-// register re-allocation: 128 x (232 + 128 + 96) = 58368 <= 384 x 168 (the launch allocation)
-constexpr int kPromoRegs = 232;
-constexpr int kEpiRegs = 128;
-constexpr int kAuxRegs = 96;
+constexpr int kPromoWarps = 8;     // warps 0-7: TMEM lane quadrant = warp % 4, token half = warp / 4
+constexpr int kEpiWarps = 4;       // warps 8-11
+constexpr int kTmaWarp = 12;
+constexpr int kMmaWarp = 13;        // and 14: one issuer per weight block of the pair; warp 15 idle
+constexpr int kThreads = 16 * 32;
+constexpr int NTH = NT / 2;        // token columns per promotion thread
+// 512 threads: 128 registers each, which every role fits (a promotion thread holds 2 x 16 accumulators and
+// 2 x 16 partial sums in flight); no re-allocation between warpgroups
 constexpr uint32_t kABytes = 2 * BW * BK;   // two weight blocks
 constexpr uint32_t kBBytes = NT * BK;       // token codes
 constexpr uint32_t kStageBytes = kABytes + kBBytes;  // 36 KB
@@ -398,7 +397,6 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 
 
   if (warp >= kPromoWarps + kEpiWarps) {
-    setmaxnreg_dec<kAuxRegs>();
     if (warp == kTmaWarp) {
       // =============================== TMA producer =======================================
       if (lane == 0) {
@@ -505,11 +503,13 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     }
   } else if (warp < kPromoWarps) {
     // =============================== promotion warps ====================================
-    setmaxnreg_inc<kPromoRegs>();
-    const int wr = warp * 32 + lane;  // weight row within a block = TMEM lane
-    const int pt = threadIdx.x;       // 0..127
+    // Two threads per weight row: warps w and w + 4 read the same TMEM lanes, the first the partial sums
+    // of token columns 0-15, the second those of columns 16-31 (of both weight blocks).
+    const int wr = (warp & 3) * 32 + lane;  // weight row within a block = TMEM lane
+    const int tb = (warp >> 2) * NTH;       // first token column of this thread
+    const int pt = threadIdx.x;             // 0..255
     constexpr uint32_t kPromoThreads = kPromoWarps * 32;
-    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int ks = 0, cur = 0, sb = 0;
     uint32_t acc_phase = 0, tile_iter = 0;
     bool ok = true;
@@ -616,17 +616,17 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const int pi = proj_of<MODE>(c.mode);
         const int KB = p.pj[pi].kblocks, N = p.pj[pi].N;
 
-        float acc_lo[NT], acc_hi[NT];
+        float acc_lo[NTH], acc_hi[NTH];
 #pragma unroll
-        for (int t = 0; t < NT; ++t) acc_lo[t] = acc_hi[t] = 0.0f;
+        for (int t = 0; t < NTH; ++t) acc_lo[t] = acc_hi[t] = 0.0f;
 
         for (int kb = 0; kb < KB; ++kb) {
           if (!warp_wait_or_abort(&s->tmem_full[ks], acc_phase, s, p)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(ks) * (2 * NT);
-          uint32_t vl[NT], vh[NT];
-          tmem_ld_x32(t0, vl);
-          tmem_ld_x32(t0 + NT, vh);
+          const uint32_t t0 = tmem_base + lane_addr + static_cast<uint32_t>(ks) * (2 * NT) + static_cast<uint32_t>(tb);
+          uint32_t vl[NTH], vh[NTH];
+          tmem_ld_x16(t0, vl);
+          tmem_ld_x16(t0 + NT, vh);
           tmem_ld_wait();
           tc_fence_before_sync();
           __syncwarp();
@@ -634,8 +634,8 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           if (++ks == kAccBufs) { ks = 0; acc_phase ^= 1; }
           const float2 sw = *reinterpret_cast<const float2*>(sl.sw[kb]);
 #pragma unroll
-          for (int t4 = 0; t4 < NT; t4 += 4) {
-            const float4 sx = *reinterpret_cast<const float4*>(&sl.sx[kb][t4]);  // same address in every lane: broadcast
+          for (int t4 = 0; t4 < NTH; t4 += 4) {
+            const float4 sx = *reinterpret_cast<const float4*>(&sl.sx[kb][tb + t4]);  // same address in every lane: broadcast
             const float sxs[4] = {sx.x, sx.y, sx.z, sx.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -649,9 +649,9 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if (ok && c.mode != kModeGateUp && p.out_f32) {  // debug dump of the fp32 accumulators
           const int col_lo = 2 * c.j * BW + wr, col_hi = col_lo + BW;
 #pragma unroll
-          for (int t = 0; t < NT; ++t) {
-            if (t < rows) {
-              float* d = p.out_f32 + static_cast<int64_t>(c.m0 + t) * N;
+          for (int t = 0; t < NTH; ++t) {
+            if (tb + t < rows) {
+              float* d = p.out_f32 + static_cast<int64_t>(c.m0 + tb + t) * N;
               d[col_lo] = acc_lo[t];
               if (col_hi < N) d[col_hi] = acc_hi[t];
             }
@@ -661,15 +661,15 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if (ok) {
           uint16_t* T16 = reinterpret_cast<uint16_t*>(out_tile);
 #pragma unroll
-          for (int t = 0; t < NT; ++t) {
+          for (int t = 0; t < NTH; ++t) {
             float lo = acc_lo[t], hi = acc_hi[t];
             if (c.mode == kModeDown) {  // contribution = bf16( fl(w * y) )
-              const float w = sl.w[t];
+              const float w = sl.w[tb + t];
               lo = __fmul_rn(w, lo);
               hi = __fmul_rn(w, hi);
             }
-            T16[t * (kOutRowBytes / 2) + wr] = static_cast<uint16_t>(f32_to_bf16_bits(lo));
-            T16[t * (kOutRowBytes / 2) + BW + wr] = static_cast<uint16_t>(f32_to_bf16_bits(hi));
+            T16[(tb + t) * (kOutRowBytes / 2) + wr] = static_cast<uint16_t>(f32_to_bf16_bits(lo));
+            T16[(tb + t) * (kOutRowBytes / 2) + BW + wr] = static_cast<uint16_t>(f32_to_bf16_bits(hi));
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&s->out_full);  // release: the epilogue warps see the tile after their wait
@@ -689,11 +689,10 @@ gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     cp_async_wait_all();
   } else {
     // =============================== epilogue warps =====================================
-    setmaxnreg_dec<kEpiRegs>();
     // They finish the staged bf16 tile per token row while the promotion warps are already in the
     // next tile: gate_up = SwiGLU, 1x128 amax / scale / e4m3 codes; down / linear = row stores.
     const int ew = warp - kPromoWarps;
-    const int et = threadIdx.x - kPromoWarps * 32;  // 0..127
+    const int et = threadIdx.x - kPromoWarps * 32;  // 0..127 (the epilogue's threads)
     constexpr uint32_t kEpiThreads = kEpiWarps * 32;
     int cur = 0, sslot = 0;
     uint32_t sphase = 0, tile_iter = 0;
